@@ -1,0 +1,241 @@
+/*
+ * libdeco — the data-parallel hot path of DD-EF-SGD / DeCo-SGD on one NVIDIA B200 (sm_100a).
+ *
+ * For n workers simulated on one GPU the library runs, per training iteration t
+ * (Algorithm 1 of the paper, "DD-EF-SGD"):
+ *
+ *   worker i :  a       = e_i + gamma * g_i
+ *               Delta_i = C_delta(a)        Top-k: the k largest-|a| entries, as (index, value)
+ *               e_i     = a - Delta_i
+ *   server   :  S_t     = sum_i Delta_i     kept in a cache (ring) of stale aggregates
+ *               x       = x - (1/n) * S_{t - tau}
+ *
+ * and, on the host, the DeCo decision (Algorithm 3) that picks (tau, delta) from the
+ * measured bandwidth and latency, with the iteration-time model of Theorem 3.
+ *
+ * Conventions
+ *   - Plain C ABI.  Pointers are marked HOST or DEVICE.  No allocation is visible to the
+ *     caller except through deco_init / deco_destroy.
+ *   - Every device operation is enqueued on the CUDA stream the caller passes
+ *     (a cudaStream_t cast to void*; NULL = the default stream) and returns without
+ *     waiting.  Argument and state errors are found on the host before anything is
+ *     launched and leave the context unchanged.
+ *   - Every function returns a deco_status; nothing throws, aborts or traps.  Anomalies seen
+ *     by a kernel (an index out of range, a count that does not add up) are latched in a
+ *     device status word and reported by deco_get_stats.
+ *   - One context is used from one host thread at a time, on one stream at a time.
+ *   - There is no CPU fallback: without a CUDA device deco_init fails with DECO_ERR_CUDA.
+ *
+ * Fixed readings where the paper is silent
+ *   - "largest" compares |a| through the IEEE-754 bit pattern with the sign cleared
+ *     (so +0 == -0, and NaN > Inf > finite, deterministically); equal magnitudes are
+ *     taken in order of increasing index.
+ *   - k = ceil(delta * d) clamped to [1, d] (delta*d within 1e-6 of an integer is that
+ *     integer); Top-k is over the whole flat vector, not per layer.
+ *   - iterations count from 0; update t applies S_{t-tau} iff t - tau >= 0.  If tau changes
+ *     at run time the cache is drained exactly once, oldest first: update t applies every
+ *     cached aggregate whose step is <= t - tau.
+ *   - state is fp32; each arithmetic statement is one fused multiply-add (round to nearest
+ *     even, no flush to zero); the n messages are summed in fp32 in worker order 0..n-1.
+ */
+#ifndef DECO_H_
+#define DECO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct deco_ctx deco_ctx;            /* opaque, owned by the library */
+
+typedef enum {
+    DECO_OK = 0,
+    DECO_ERR_INVALID_ARG = 1,   /* NULL pointer, d == 0, delta outside (0,1], misaligned buffer ... */
+    DECO_ERR_OOM = 2,           /* device or host allocation failed */
+    DECO_ERR_CUDA = 3,          /* a CUDA runtime call failed (no device, launch error ...) */
+    DECO_ERR_STATE = 4,         /* calls out of order (compress -> aggregate -> apply) */
+    DECO_ERR_CAPACITY = 5,      /* tau > tau_max, or k(delta) > k(delta_max) */
+    DECO_ERR_TIMEOUT = 6,       /* reserved: a bounded device-side wait ran out */
+    DECO_ERR_DEVICE_CHECK = 7   /* a kernel's self-check latched an anomaly */
+} deco_status;
+
+typedef enum { DECO_F32 = 0, DECO_BF16 = 1 } deco_dtype;
+
+/* One element of a compressed update Delta (what a worker would send): 8 bytes. */
+typedef struct { uint32_t idx; float val; } deco_pair;
+
+/* idx value of an unused position inside a cached aggregate (see deco_get_aggregate). */
+#define DECO_NO_INDEX 0xFFFFFFFFu
+
+typedef enum {
+    DECO_SELECT_AUTO = 0,       /* sampled threshold + one streaming pass; exact multi-pass
+                                   selection only for the workers where the sample fails */
+    DECO_SELECT_EXACT_PASSES = 1 /* always the multi-pass radix selection (no sampling) */
+} deco_select_mode;
+
+/* Options of deco_init.  A zero-filled struct selects every default. */
+typedef struct {
+    int32_t  grad_dtype;     /* deco_dtype of the gradients handed to deco_ef_compress; default F32 */
+    uint32_t tau_max;        /* largest staleness deco_set_policy may ask for; 0 -> the initial tau */
+    double   delta_max;      /* largest ratio deco_set_policy may ask for; 0 -> the initial delta */
+    int32_t  lr_at_server;   /* 0: paper form, a = e + gamma*g and update scale 1/n;
+                                1: a = e + g and update scale gamma/n */
+    float   *params;         /* DEVICE, [d] fp32, 16-byte aligned, caller-owned; NULL -> the library
+                                allocates a zero-filled vector and frees it in deco_destroy */
+    int32_t  device;         /* CUDA device ordinal */
+    int32_t  select_mode;    /* deco_select_mode */
+    uint32_t reserved[8];    /* must be zero */
+} deco_options;
+
+typedef struct {
+    uint64_t step;                 /* iterations completed (t of the next compress) */
+    uint64_t k;                    /* entries kept per worker at the current delta */
+    double   delta;
+    uint32_t tau;
+    uint32_t device_status;        /* 0, or a deco_status latched by a kernel */
+    uint64_t exact_pass_workers;   /* worker-iterations that needed the multi-pass selection */
+    uint64_t cached_aggregates;    /* aggregates sent but not yet applied */
+    uint64_t device_bytes;         /* device memory held by the context */
+} deco_stats;
+
+/* ------------------------------------------------------------------ life cycle */
+
+/*
+ * Create the state of Algorithm 1 ("Initialize x_0, e_0^i = 0"): error terms e[n][d] = 0, an
+ * empty cache of stale aggregates, iteration counter 0, and the inputs n, gamma (lr), delta,
+ * tau.  d < 2^32 - 1, n >= 1, 0 < delta <= 1.  Allocates all device memory the context will
+ * ever use (sized by delta_max and tau_max).  *out is set only on success.
+ */
+deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double delta, uint32_t tau,
+                      float lr, const deco_options *opt /* HOST, may be NULL */);
+
+/* Free the context and everything it owns (waits for the device first).  NULL is allowed. */
+void deco_destroy(deco_ctx *ctx);
+
+/* Back to the state right after deco_init (e = 0, cache empty, t = 0; library-owned
+ * parameters are zeroed, caller-owned ones are left alone).  Enqueued on `stream`. */
+deco_status deco_reset(deco_ctx *ctx, void *stream);
+
+/* ------------------------------------------------------- the iteration (hot path) */
+
+/*
+ * Worker side of iteration t for all n workers (Algorithm 1: "Delta = C_delta(e + gamma g)",
+ * "e = e + gamma g - Delta").
+ *   grads  DEVICE, [n][d] row-major without padding, dtype = grad_dtype, read-only; the base
+ *          must be 16-byte aligned.  Rows that are not 16-byte aligned (d*sizeof(g) % 16 != 0)
+ *          are accepted and read with narrower loads.  May be reused once the stream has
+ *          passed this call.
+ * Afterwards (in stream order) the message buffer holds, per worker, exactly k pairs sorted
+ * by increasing index, val being the selected entry of a verbatim, and e holds a with +0
+ * at the selected positions.
+ */
+deco_status deco_ef_compress(deco_ctx *ctx, const void *grads, void *stream);
+
+/*
+ * Server side, arrival of iteration t's messages (Algorithm 1: the sum inside
+ * "x = x - (1/n) sum_i Delta_{t-tau}^i", kept in the server's cache of stale updates):
+ * S_t[j] = sum over workers, in worker order, of the values sent for index j, stored sparsely
+ * in cache slot t mod (tau_max + 1).  Must follow deco_ef_compress of the same iteration.
+ */
+deco_status deco_aggregate_stale(deco_ctx *ctx, void *stream);
+
+/*
+ * Server update of iteration t (Algorithm 1: "x_{t+1} = x_t - (1/n) sum_i Delta_{t-tau}^i"):
+ * x[j] = fma(-scale, S_s[j], x[j]) for every cached aggregate with s <= t - tau, oldest
+ * first (normally exactly one; none while t < tau), scale = 1/n (or gamma/n with
+ * lr_at_server).  Then t advances.  Must follow deco_aggregate_stale.
+ */
+deco_status deco_apply_update(deco_ctx *ctx, void *stream);
+
+/* The three calls above in order, for callers that do not interleave other work. */
+deco_status deco_step(deco_ctx *ctx, const void *grads /* DEVICE */, void *stream);
+
+/*
+ * One iteration with HOST buffers: copies grads_host ([n][d], grad_dtype) to the device,
+ * runs deco_step, and copies back what a deployment would move: the n messages
+ * (msg_host_out, [n][k] pairs, may be NULL) and the parameters (params_host_out, [d] fp32,
+ * may be NULL).  Copies are asynchronous on `stream`; use pinned host memory and
+ * synchronise the stream before reading the outputs.
+ */
+deco_status deco_step_host(deco_ctx *ctx, const void *grads_host, deco_pair *msg_host_out,
+                           float *params_host_out, void *stream);
+
+/* ------------------------------------------------------------- policy (Algorithms 2, 3) */
+
+/*
+ * Algorithm 2: "Broadcast new tau and delta".  Takes effect from the next deco_ef_compress;
+ * may only be called between iterations.  tau > tau_max or k(delta) > k(delta_max) gives
+ * DECO_ERR_CAPACITY and changes nothing.
+ */
+deco_status deco_set_policy(deco_ctx *ctx, double delta, uint32_t tau);
+
+/* New stepsize gamma from the next iteration on. */
+deco_status deco_set_lr(deco_ctx *ctx, float lr);
+
+/*
+ * Algorithm 3 (DeCo), pure host arithmetic in double: walk tau from
+ * ceil((b + V_g/a_bar)/T_comp) down to ceil(b/T_comp), delta = delta*(tau) =
+ * min{(tau T_comp - b) a_bar / V_g, T_comp a_bar / V_g, 1}, keep the pair with the smallest
+ * phi = (1-delta)/(delta (1-delta/2)^tau) (phi' = phi/delta when non_iid != 0); equal phi
+ * goes to the smaller tau; candidates with delta <= 0 are skipped; if none is feasible
+ * tau = ceil(b/T_comp) + 1.  Finally tau is clamped to tau_cap (delta recomputed for the
+ * clamped tau) when tau_cap != 0.
+ *   V_g_bits > 0, a_bar_bps > 0, b_s >= 0, T_comp_s > 0;  tau_out, delta_out HOST.
+ */
+deco_status deco_policy_select(double V_g_bits, double a_bar_bps, double b_s, double T_comp_s,
+                               uint32_t tau_cap, int32_t non_iid,
+                               uint32_t *tau_out, double *delta_out);
+
+/* Theorem 3: T_avg ~ max{(T_comp + b + delta V_g/a_bar)/(tau+1), delta V_g/a_bar, T_comp}.
+ * Returns a negative value for invalid arguments. */
+double deco_t_avg(double delta, uint32_t tau, double V_g_bits, double a_bar_bps, double b_s,
+                  double T_comp_s);
+
+/* k kept for ratio delta on a length-d vector (0 for invalid arguments). */
+uint64_t deco_k_from_delta(double delta, uint64_t d);
+
+/* --------------------------------------------------------------------- inspection */
+
+deco_status deco_get_k(const deco_ctx *ctx, uint64_t *k /* HOST */);
+
+/*
+ * Device pointers of the library-owned state (any out-pointer may be NULL):
+ *   e       [n][e_stride] fp32, error terms; columns >= d are padding
+ *   msg     [n][k_cap] pairs, the messages of the last deco_ef_compress (first k valid)
+ *   params  [d] fp32
+ */
+deco_status deco_get_buffers(deco_ctx *ctx, float **e, uint64_t *e_stride, deco_pair **msg,
+                             uint64_t *k_cap, float **params);
+
+/*
+ * The cached aggregate of iteration `step` (must still be in the cache): DEVICE pointer to
+ * `positions` pairs; positions with idx == DECO_NO_INDEX are unused, the others hold each
+ * touched index once (increasing) with its fp32 sum.
+ */
+deco_status deco_get_aggregate(deco_ctx *ctx, uint64_t step, const deco_pair **entries,
+                               uint64_t *positions);
+
+/*
+ * Per-worker facts about the last deco_ef_compress (waits for `stream`); each HOST array has
+ * n entries and may be NULL:
+ *   threshold_key  magnitude key (bit pattern, sign cleared) of the k-th largest |a|
+ *   n_greater      entries strictly above it
+ *   exact_passes   1 if the worker went through the multi-pass selection in that call
+ */
+deco_status deco_get_select_info(deco_ctx *ctx, void *stream, uint32_t *threshold_key,
+                                 uint32_t *n_greater, uint32_t *exact_passes);
+
+/* Waits for `stream`, then fills *out (HOST); returns DECO_ERR_DEVICE_CHECK if a kernel
+ * latched an anomaly since the context was created or reset. */
+deco_status deco_get_stats(deco_ctx *ctx, void *stream, deco_stats *out);
+
+/* Number of kernels and memset/memcpy nodes the library has enqueued so far. */
+uint64_t deco_launch_count(const deco_ctx *ctx);
+
+const char *deco_status_string(deco_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DECO_H_ */

@@ -1,0 +1,273 @@
+"""ctypes binding of libdeco: one Python function per C entry point, same names.
+
+Argument marshalling only — every step of the path runs in the library's CUDA kernels.
+Tensors are passed as raw device pointers (``tensor.data_ptr()``) and the current PyTorch
+stream's handle; PyTorch is used for device memory and streams, nothing else.  There is no
+fallback: if ``libdeco.so`` is missing or no CUDA device is present the calls raise.
+"""
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdeco.so")
+
+DECO_OK = 0
+DECO_ERR_INVALID_ARG = 1
+DECO_ERR_OOM = 2
+DECO_ERR_CUDA = 3
+DECO_ERR_STATE = 4
+DECO_ERR_CAPACITY = 5
+DECO_ERR_TIMEOUT = 6
+DECO_ERR_DEVICE_CHECK = 7
+
+DECO_F32 = 0
+DECO_BF16 = 1
+DECO_NO_INDEX = 0xFFFFFFFF
+DECO_SELECT_AUTO = 0
+DECO_SELECT_EXACT_PASSES = 1
+
+
+class deco_pair(ctypes.Structure):
+    _fields_ = [("idx", ctypes.c_uint32), ("val", ctypes.c_float)]
+
+
+class deco_options(ctypes.Structure):
+    _fields_ = [("grad_dtype", ctypes.c_int32),
+                ("tau_max", ctypes.c_uint32),
+                ("delta_max", ctypes.c_double),
+                ("lr_at_server", ctypes.c_int32),
+                ("params", ctypes.c_void_p),
+                ("device", ctypes.c_int32),
+                ("select_mode", ctypes.c_int32),
+                ("reserved", ctypes.c_uint32 * 8)]
+
+
+class deco_stats(ctypes.Structure):
+    _fields_ = [("step", ctypes.c_uint64),
+                ("k", ctypes.c_uint64),
+                ("delta", ctypes.c_double),
+                ("tau", ctypes.c_uint32),
+                ("device_status", ctypes.c_uint32),
+                ("exact_pass_workers", ctypes.c_uint64),
+                ("cached_aggregates", ctypes.c_uint64),
+                ("device_bytes", ctypes.c_uint64)]
+
+
+class DecoError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__("%s: %s (%d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+_vp, _u64, _u32, _i32, _f32, _f64 = (ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32,
+                                     ctypes.c_int32, ctypes.c_float, ctypes.c_double)
+_P = ctypes.POINTER
+
+# name -> (restype, argtypes); the list mirrors include/deco.h
+SIGNATURES = {
+    "deco_init": (_i32, [_P(_vp), _u64, _u32, _f64, _u32, _f32, _P(deco_options)]),
+    "deco_destroy": (None, [_vp]),
+    "deco_reset": (_i32, [_vp, _vp]),
+    "deco_ef_compress": (_i32, [_vp, _vp, _vp]),
+    "deco_aggregate_stale": (_i32, [_vp, _vp]),
+    "deco_apply_update": (_i32, [_vp, _vp]),
+    "deco_step": (_i32, [_vp, _vp, _vp]),
+    "deco_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp]),
+    "deco_set_policy": (_i32, [_vp, _f64, _u32]),
+    "deco_set_lr": (_i32, [_vp, _f32]),
+    "deco_policy_select": (_i32, [_f64, _f64, _f64, _f64, _u32, _i32, _P(_u32), _P(_f64)]),
+    "deco_t_avg": (_f64, [_f64, _u32, _f64, _f64, _f64, _f64]),
+    "deco_k_from_delta": (_u64, [_f64, _u64]),
+    "deco_get_k": (_i32, [_vp, _P(_u64)]),
+    "deco_get_buffers": (_i32, [_vp, _P(_vp), _P(_u64), _P(_vp), _P(_u64), _P(_vp)]),
+    "deco_get_aggregate": (_i32, [_vp, _u64, _P(_vp), _P(_u64)]),
+    "deco_get_select_info": (_i32, [_vp, _vp, _vp, _vp, _vp]),
+    "deco_get_stats": (_i32, [_vp, _vp, _P(deco_stats)]),
+    "deco_launch_count": (_u64, [_vp]),
+    "deco_status_string": (ctypes.c_char_p, [_i32]),
+}
+
+
+def load():
+    """Load libdeco.so (built in-tree by ``build.py``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise OSError("libdeco.so not built: run `python -m paper_2507_17346_b200.build` "
+                          "(expected at %s)" % LIB_PATH)
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def deco_status_string(status):
+    return load().deco_status_string(int(status)).decode()
+
+
+status_string = deco_status_string
+
+
+def _check(status, where):
+    if status != DECO_OK:
+        raise DecoError(status, where)
+
+
+def _ptr(x):
+    """Raw address of a torch tensor / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+# ------------------------------------------------------------------ entry points
+
+def deco_init(d, n, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0, delta_max=0.0,
+              lr_at_server=False, params=None, device=0, select_mode=DECO_SELECT_AUTO):
+    """-> opaque context handle (int).  `params`: optional fp32 CUDA tensor of length d."""
+    opt = deco_options()
+    opt.grad_dtype = grad_dtype
+    opt.tau_max = tau_max
+    opt.delta_max = delta_max
+    opt.lr_at_server = int(bool(lr_at_server))
+    opt.params = _ptr(params)
+    opt.device = device
+    opt.select_mode = select_mode
+    ctx = _vp()
+    _check(load().deco_init(ctypes.byref(ctx), d, n, delta, tau, lr, ctypes.byref(opt)),
+           "deco_init")
+    return ctx.value
+
+
+def deco_destroy(ctx):
+    load().deco_destroy(ctx)
+
+
+def deco_reset(ctx, stream=None):
+    _check(load().deco_reset(ctx, _stream(stream)), "deco_reset")
+
+
+def deco_ef_compress(ctx, grads, stream=None):
+    _check(load().deco_ef_compress(ctx, _ptr(grads), _stream(stream)), "deco_ef_compress")
+
+
+def deco_aggregate_stale(ctx, stream=None):
+    _check(load().deco_aggregate_stale(ctx, _stream(stream)), "deco_aggregate_stale")
+
+
+def deco_apply_update(ctx, stream=None):
+    _check(load().deco_apply_update(ctx, _stream(stream)), "deco_apply_update")
+
+
+def deco_step(ctx, grads, stream=None):
+    _check(load().deco_step(ctx, _ptr(grads), _stream(stream)), "deco_step")
+
+
+def deco_step_host(ctx, grads_host, msg_host_out=None, params_host_out=None, stream=None):
+    _check(load().deco_step_host(ctx, _ptr(grads_host), _ptr(msg_host_out),
+                                 _ptr(params_host_out), _stream(stream)), "deco_step_host")
+
+
+def deco_set_policy(ctx, delta, tau):
+    _check(load().deco_set_policy(ctx, delta, tau), "deco_set_policy")
+
+
+def deco_set_lr(ctx, lr):
+    _check(load().deco_set_lr(ctx, lr), "deco_set_lr")
+
+
+def deco_policy_select(V_g_bits, a_bar_bps, b_s, T_comp_s, tau_cap=0, non_iid=False):
+    """Algorithm 3 -> (tau, delta)."""
+    tau, delta = _u32(), _f64()
+    _check(load().deco_policy_select(V_g_bits, a_bar_bps, b_s, T_comp_s, tau_cap,
+                                     int(bool(non_iid)), ctypes.byref(tau),
+                                     ctypes.byref(delta)), "deco_policy_select")
+    return tau.value, delta.value
+
+
+def deco_t_avg(delta, tau, V_g_bits, a_bar_bps, b_s, T_comp_s):
+    return load().deco_t_avg(delta, tau, V_g_bits, a_bar_bps, b_s, T_comp_s)
+
+
+def deco_k_from_delta(delta, d):
+    return load().deco_k_from_delta(delta, d)
+
+
+def deco_get_k(ctx):
+    k = _u64()
+    _check(load().deco_get_k(ctx, ctypes.byref(k)), "deco_get_k")
+    return k.value
+
+
+def deco_get_buffers(ctx):
+    """-> dict of raw device addresses and sizes: e, e_stride, msg, k_cap, params."""
+    e, msg, params = _vp(), _vp(), _vp()
+    stride, k_cap = _u64(), _u64()
+    _check(load().deco_get_buffers(ctx, ctypes.byref(e), ctypes.byref(stride), ctypes.byref(msg),
+                                   ctypes.byref(k_cap), ctypes.byref(params)),
+           "deco_get_buffers")
+    return {"e": e.value, "e_stride": stride.value, "msg": msg.value, "k_cap": k_cap.value,
+            "params": params.value}
+
+
+def deco_get_aggregate(ctx, step):
+    """-> (device address of the pairs, number of positions) of a cached aggregate."""
+    entries, positions = _vp(), _u64()
+    _check(load().deco_get_aggregate(ctx, step, ctypes.byref(entries), ctypes.byref(positions)),
+           "deco_get_aggregate")
+    return entries.value, positions.value
+
+
+def deco_get_select_info(ctx, n, stream=None):
+    """-> (threshold_key[n], n_greater[n], exact_passes[n]) as Python lists."""
+    thr, gt, ex = (_u32 * n)(), (_u32 * n)(), (_u32 * n)()
+    _check(load().deco_get_select_info(ctx, _stream(stream), thr, gt, ex),
+           "deco_get_select_info")
+    return list(thr), list(gt), list(ex)
+
+
+def deco_get_stats(ctx, stream=None):
+    st = deco_stats()
+    _check(load().deco_get_stats(ctx, _stream(stream), ctypes.byref(st)), "deco_get_stats")
+    return {f: getattr(st, f) for f, _ in deco_stats._fields_}
+
+
+def deco_launch_count(ctx):
+    return load().deco_launch_count(ctx)
+
+
+# ------------------------------------------------------------- device views (plumbing)
+
+class _DevArray:
+    """Minimal __cuda_array_interface__ holder so torch can view library-owned memory."""
+
+    def __init__(self, addr, shape, typestr, strides=None):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr,
+                                         "data": (int(addr), False), "version": 2,
+                                         "strides": strides}
+
+
+def view_f32(addr, shape, device=0):
+    import torch
+    return torch.as_tensor(_DevArray(addr, shape, "<f4"), device="cuda:%d" % device)
+
+
+def view_i32(addr, shape, device=0):
+    import torch
+    return torch.as_tensor(_DevArray(addr, shape, "<i4"), device="cuda:%d" % device)

@@ -1,0 +1,419 @@
+// Host side of libdeco: context, memory, iteration state machine, cache (ring) bookkeeping.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "deco_internal.h"
+
+using namespace deco;
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+template <typename T>
+deco_status dev_alloc(deco_ctx *c, T **p, uint64_t count)
+{
+    const uint64_t bytes = (count ? count : 1) * sizeof(T);
+    void *q = nullptr;
+    cudaError_t err = cudaMalloc(&q, bytes);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return err == cudaErrorMemoryAllocation ? DECO_ERR_OOM : DECO_ERR_CUDA;
+    }
+    *p = static_cast<T *>(q);
+    c->device_bytes += bytes;
+    return DECO_OK;
+}
+
+void free_all(deco_ctx *c)
+{
+    cudaFree(c->e);
+    if (c->own_params) cudaFree(c->params);
+    cudaFree(c->msg);
+    cudaFree(c->slots);
+    cudaFree(c->stage);
+    cudaFree(c->hist);
+    cudaFree(c->sel);
+    cudaFree(c->tile_gt);
+    cudaFree(c->tile_eq);
+    cudaFree(c->tile_take);
+    cudaFree(c->tile_start);
+    cudaFree(c->tile_off);
+    cudaFree(c->tile_cnt);
+    cudaFree(c->sample_keys);
+    cudaFree(c->dev_status);
+    cudaFree(c->grads_staging);
+}
+
+deco_status zero_state(deco_ctx *c, cudaStream_t s)
+{
+    cudaError_t err = cudaMemsetAsync(c->e, 0, sizeof(float) * c->n * c->e_stride, s);
+    if (err == cudaSuccess && c->own_params)
+        err = cudaMemsetAsync(c->params, 0, sizeof(float) * c->d, s);
+    if (err == cudaSuccess) err = cudaMemsetAsync(c->sel, 0, sizeof(SelectState) * c->n, s);
+    if (err == cudaSuccess) err = cudaMemsetAsync(c->dev_status, 0, sizeof(uint32_t) * 4, s);
+    if (err == cudaSuccess)
+        err = cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n * (c->ntiles + 1), s);
+    c->launches += 5;
+    c->t = 0;
+    c->phase = 0;
+    for (auto &sl : c->slot_info) sl = Slot();
+    return err == cudaSuccess ? DECO_OK : DECO_ERR_CUDA;
+}
+
+inline cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
+
+}  // namespace
+
+extern "C" const char *deco_status_string(deco_status s)
+{
+    switch (s) {
+    case DECO_OK: return "ok";
+    case DECO_ERR_INVALID_ARG: return "invalid argument";
+    case DECO_ERR_OOM: return "out of memory";
+    case DECO_ERR_CUDA: return "CUDA runtime error";
+    case DECO_ERR_STATE: return "call out of order";
+    case DECO_ERR_CAPACITY: return "beyond the capacity fixed at deco_init";
+    case DECO_ERR_TIMEOUT: return "device-side wait ran out";
+    case DECO_ERR_DEVICE_CHECK: return "a kernel self-check failed";
+    }
+    return "unknown status";
+}
+
+extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double delta,
+                                 uint32_t tau, float lr, const deco_options *opt)
+{
+    if (!out) return DECO_ERR_INVALID_ARG;
+    deco_options o;
+    std::memset(&o, 0, sizeof o);
+    if (opt) o = *opt;
+    for (uint32_t r : o.reserved)
+        if (r != 0) return DECO_ERR_INVALID_ARG;
+    if (d == 0 || d >= 0xFFFFFFFFull - TILE || n == 0 || n > 65535) return DECO_ERR_INVALID_ARG;
+    if (!(delta > 0.0) || !(delta <= 1.0) || !(lr == lr)) return DECO_ERR_INVALID_ARG;
+    if (o.grad_dtype != DECO_F32 && o.grad_dtype != DECO_BF16) return DECO_ERR_INVALID_ARG;
+    if (o.select_mode != DECO_SELECT_AUTO && o.select_mode != DECO_SELECT_EXACT_PASSES)
+        return DECO_ERR_INVALID_ARG;
+    if (o.delta_max != 0.0 && (!(o.delta_max <= 1.0) || o.delta_max < delta))
+        return DECO_ERR_INVALID_ARG;
+    if (o.tau_max != 0 && o.tau_max < tau) return DECO_ERR_INVALID_ARG;
+    if (o.tau_max > (1u << 20) || tau > (1u << 20)) return DECO_ERR_INVALID_ARG;
+    if (o.params && (reinterpret_cast<uintptr_t>(o.params) & 15u)) return DECO_ERR_INVALID_ARG;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) {
+        cudaGetLastError();
+        return DECO_ERR_CUDA;
+    }
+    if (o.device < 0 || o.device >= ndev) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(o.device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+
+    deco_ctx *c = new (std::nothrow) deco_ctx();
+    if (!c) return DECO_ERR_OOM;
+    c->d = d;
+    c->n = n;
+    c->delta = delta;
+    c->delta_max = o.delta_max != 0.0 ? o.delta_max : delta;
+    c->tau = tau;
+    c->tau_max = o.tau_max != 0 ? o.tau_max : tau;
+    c->lr = lr;
+    c->grad_dtype = o.grad_dtype;
+    c->lr_at_server = o.lr_at_server;
+    c->select_mode = o.select_mode;
+    c->device = o.device;
+    c->k = deco_k_from_delta(delta, d);
+    c->k_cap = deco_k_from_delta(c->delta_max, d);
+    c->ntiles = static_cast<uint32_t>((d + TILE - 1) / TILE);
+    c->e_stride = static_cast<uint64_t>(c->ntiles) * TILE;
+    c->ring = c->tau_max + 1;
+    // staged candidates per worker: four times the message capacity plus slack, at most d
+    c->stage_cap = 4 * c->k_cap + 65536;
+    if (c->stage_cap > c->e_stride) c->stage_cap = c->e_stride;
+    try {
+        c->slot_info.resize(c->ring);
+    } catch (...) {
+        delete c;
+        return DECO_ERR_OOM;
+    }
+
+    deco_status st = DECO_OK;
+    auto need = [&](deco_status s) { if (st == DECO_OK) st = s; };
+    need(dev_alloc(c, &c->e, static_cast<uint64_t>(n) * c->e_stride));
+    if (o.params) {
+        c->params = o.params;
+    } else {
+        need(dev_alloc(c, &c->params, d));
+        c->own_params = (st == DECO_OK);
+    }
+    need(dev_alloc(c, &c->msg, static_cast<uint64_t>(n) * c->k_cap));
+    need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * n * c->k_cap));
+    need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
+    need(dev_alloc(c, &c->hist, static_cast<uint64_t>(n) * RADIX_LEVELS * RADIX_BINS));
+    need(dev_alloc(c, &c->sel, n));
+    need(dev_alloc(c, &c->tile_gt, static_cast<uint64_t>(n) * c->ntiles));
+    need(dev_alloc(c, &c->tile_eq, static_cast<uint64_t>(n) * c->ntiles));
+    need(dev_alloc(c, &c->tile_take, static_cast<uint64_t>(n) * c->ntiles));
+    need(dev_alloc(c, &c->tile_start, static_cast<uint64_t>(n) * (c->ntiles + 1)));
+    need(dev_alloc(c, &c->tile_off, static_cast<uint64_t>(n) * c->ntiles));
+    need(dev_alloc(c, &c->tile_cnt, static_cast<uint64_t>(n) * c->ntiles));
+    need(dev_alloc(c, &c->dev_status, 4));
+    if (st == DECO_OK) st = zero_state(c, nullptr);
+    if (st == DECO_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = DECO_ERR_CUDA;
+    if (st != DECO_OK) {
+        free_all(c);
+        delete c;
+        cudaGetLastError();
+        return st;
+    }
+    *out = c;
+    return DECO_OK;
+}
+
+extern "C" void deco_destroy(deco_ctx *c)
+{
+    if (!c) return;
+    DeviceGuard guard(c->device);
+    cudaDeviceSynchronize();
+    free_all(c);
+    delete c;
+}
+
+extern "C" deco_status deco_reset(deco_ctx *c, void *stream)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    return zero_state(c, as_stream(stream));
+}
+
+extern "C" deco_status deco_ef_compress(deco_ctx *c, const void *grads, void *stream)
+{
+    if (!c || !grads) return DECO_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(grads) & 15u) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    cudaStream_t s = as_stream(stream);
+    c->k_of_msg = c->k;
+    cudaError_t err = launch_begin_step(c, s);
+    if (err == cudaSuccess) err = launch_accumulate(c, grads, s);
+    if (err == cudaSuccess) err = launch_exact_selection(c, s);
+    if (err != cudaSuccess) return DECO_ERR_CUDA;
+    c->phase = 1;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_aggregate_stale(deco_ctx *c, void *stream)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 1) return DECO_ERR_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    const uint32_t si = static_cast<uint32_t>(c->t % c->ring);
+    Slot &sl = c->slot_info[si];
+    if (sl.valid) return DECO_ERR_STATE;    // cannot happen while tau <= tau_max
+    deco_pair *slot = c->slots + static_cast<uint64_t>(si) * c->n * c->k_cap;
+    if (launch_aggregate(c, slot, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    sl.step = c->t;
+    sl.positions = static_cast<uint64_t>(c->n) * c->k_of_msg;
+    sl.valid = true;
+    c->phase = 2;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_apply_update(deco_ctx *c, void *stream)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 2) return DECO_ERR_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    const float beta = c->lr_at_server ? c->lr : 1.0f;
+    const float neg_scale = -(beta / static_cast<float>(c->n));
+    if (c->t >= c->tau) {
+        const uint64_t due = c->t - c->tau;
+        // oldest first: step ids still cached lie in (t - ring, t]
+        const uint64_t lo = c->t + 1 >= c->ring ? c->t + 1 - c->ring : 0;
+        for (uint64_t s = lo; s <= due; ++s) {
+            Slot &sl = c->slot_info[s % c->ring];
+            if (!sl.valid || sl.step != s) continue;
+            const deco_pair *slot = c->slots + (s % c->ring) * c->n * c->k_cap;
+            if (launch_apply(c, slot, sl.positions, neg_scale, as_stream(stream)) != cudaSuccess)
+                return DECO_ERR_CUDA;
+            sl.valid = false;
+        }
+    }
+    c->t += 1;
+    c->phase = 0;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_step(deco_ctx *c, const void *grads, void *stream)
+{
+    deco_status st = deco_ef_compress(c, grads, stream);
+    if (st == DECO_OK) st = deco_aggregate_stale(c, stream);
+    if (st == DECO_OK) st = deco_apply_update(c, stream);
+    return st;
+}
+
+extern "C" deco_status deco_step_host(deco_ctx *c, const void *grads_host, deco_pair *msg_out,
+                                      float *params_out, void *stream)
+{
+    if (!c || !grads_host) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    cudaStream_t s = as_stream(stream);
+    const uint64_t gbytes = static_cast<uint64_t>(c->n) * c->d * (c->grad_dtype == DECO_BF16 ? 2 : 4);
+    if (!c->grads_staging) {
+        void *q = nullptr;
+        cudaError_t err = cudaMalloc(&q, gbytes);
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            return err == cudaErrorMemoryAllocation ? DECO_ERR_OOM : DECO_ERR_CUDA;
+        }
+        c->grads_staging = q;
+        c->device_bytes += gbytes;
+    }
+    if (cudaMemcpyAsync(c->grads_staging, grads_host, gbytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    c->launches += 1;
+    deco_status st = deco_step(c, c->grads_staging, stream);
+    if (st != DECO_OK) return st;
+    if (msg_out) {
+        // rows of k pairs, packed: [n][k]
+        if (cudaMemcpy2DAsync(msg_out, c->k_of_msg * sizeof(deco_pair), c->msg,
+                              c->k_cap * sizeof(deco_pair), c->k_of_msg * sizeof(deco_pair), c->n,
+                              cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        c->launches += 1;
+    }
+    if (params_out) {
+        if (cudaMemcpyAsync(params_out, c->params, sizeof(float) * c->d, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        c->launches += 1;
+    }
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_set_policy(deco_ctx *c, double delta, uint32_t tau)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    if (!(delta > 0.0) || !(delta <= 1.0)) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    const uint64_t k = deco_k_from_delta(delta, c->d);
+    if (tau > c->tau_max || k > c->k_cap) return DECO_ERR_CAPACITY;
+    c->delta = delta;
+    c->tau = tau;
+    c->k = k;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_set_lr(deco_ctx *c, float lr)
+{
+    if (!c || !(lr == lr)) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    c->lr = lr;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_get_k(const deco_ctx *c, uint64_t *k)
+{
+    if (!c || !k) return DECO_ERR_INVALID_ARG;
+    *k = c->k;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_get_buffers(deco_ctx *c, float **e, uint64_t *e_stride,
+                                        deco_pair **msg, uint64_t *k_cap, float **params)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    if (e) *e = c->e;
+    if (e_stride) *e_stride = c->e_stride;
+    if (msg) *msg = c->msg;
+    if (k_cap) *k_cap = c->k_cap;
+    if (params) *params = c->params;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_get_aggregate(deco_ctx *c, uint64_t step, const deco_pair **entries,
+                                          uint64_t *positions)
+{
+    if (!c || !entries || !positions) return DECO_ERR_INVALID_ARG;
+    const Slot &sl = c->slot_info[step % c->ring];
+    if (!sl.valid || sl.step != step) return DECO_ERR_STATE;
+    *entries = c->slots + (step % c->ring) * c->n * c->k_cap;
+    *positions = sl.positions;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_get_select_info(deco_ctx *c, void *stream, uint32_t *threshold_key,
+                                            uint32_t *n_greater, uint32_t *exact_passes)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    std::vector<SelectState> h;
+    try {
+        h.resize(c->n);
+    } catch (...) {
+        return DECO_ERR_OOM;
+    }
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    if (cudaMemcpy(h.data(), c->sel, sizeof(SelectState) * c->n, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    for (uint32_t i = 0; i < c->n; ++i) {
+        if (threshold_key) threshold_key[i] = h[i].threshold;
+        if (n_greater) n_greater[i] = h[i].n_greater;
+        if (exact_passes) exact_passes[i] = h[i].exact;
+    }
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_get_stats(deco_ctx *c, void *stream, deco_stats *out)
+{
+    if (!c || !out) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    uint32_t st[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(st, c->dev_status, sizeof st, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    std::vector<SelectState> h;
+    try {
+        h.resize(c->n);
+    } catch (...) {
+        return DECO_ERR_OOM;
+    }
+    if (cudaMemcpy(h.data(), c->sel, sizeof(SelectState) * c->n, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    std::memset(out, 0, sizeof *out);
+    out->step = c->t;
+    out->k = c->k;
+    out->delta = c->delta;
+    out->tau = c->tau;
+    out->device_status = st[0];
+    for (uint32_t i = 0; i < c->n; ++i) out->exact_pass_workers += h[i].exact_total;
+    for (const Slot &sl : c->slot_info) out->cached_aggregates += sl.valid ? 1 : 0;
+    out->device_bytes = c->device_bytes;
+    if (st[0] != 0) {
+        std::fprintf(stderr, "libdeco: device check %u (site 0x%x, detail %u)\n", st[0], st[1], st[2]);
+        return DECO_ERR_DEVICE_CHECK;
+    }
+    return DECO_OK;
+}
+
+extern "C" uint64_t deco_launch_count(const deco_ctx *c) { return c ? c->launches : 0; }

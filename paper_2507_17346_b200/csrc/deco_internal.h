@@ -1,0 +1,107 @@
+// Internal declarations shared by the host API and the kernel translation units of libdeco.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "deco.h"
+
+namespace deco {
+
+// Geometry of one streaming tile.  A tile is TILE consecutive entries of one worker's
+// vector, processed by one CTA of BLOCK threads; warp w owns the WARP_ELEMS consecutive
+// entries [w*WARP_ELEMS, (w+1)*WARP_ELEMS) of the tile, so that every warp-level load
+// instruction is one contiguous 512-byte request and entry order is (warp, round, lane,
+// component).  Tiles are also the index blocks of the message directory.
+constexpr int TILE = 8192;
+constexpr int BLOCK = 256;
+constexpr int WARPS = BLOCK / 32;
+constexpr int WARP_ELEMS = TILE / WARPS;   // 1024
+
+// Radix levels over the 31-bit magnitude key: 12 + 12 + 7 bits, most significant first.
+constexpr int RADIX_BINS = 4096;
+constexpr int RADIX_LEVELS = 3;
+
+// Per-worker selection record (device).  One 64-byte line per worker.
+struct SelectState {
+    uint32_t prefix;        // key bits resolved so far (right-aligned)
+    uint32_t k_rem;         // entries still to take among keys matching `prefix`
+    uint32_t n_greater;     // entries known to be strictly above the threshold
+    uint32_t threshold;     // final: key of the k-th largest magnitude
+    uint32_t ties_take;     // final: how many entries equal to `threshold` are taken (by index)
+    uint32_t exact;         // 1: this worker runs the multi-pass selection over e this step
+    uint32_t spec_key;      // speculative lower bound used by the streaming pass (or DISABLED)
+    uint32_t n_staged;      // candidates staged by the streaming pass
+    uint32_t exact_total;   // cumulative count of steps that took the multi-pass path
+    uint32_t pad[7];
+};
+static_assert(sizeof(SelectState) == 64, "one line per worker");
+
+constexpr uint32_t SPEC_DISABLED = 0x80000000u;   // above every 31-bit key
+
+struct Slot {
+    uint64_t step = 0;
+    uint64_t positions = 0;
+    bool valid = false;
+};
+
+}  // namespace deco
+
+struct deco_ctx {
+    // problem
+    uint64_t d = 0;
+    uint32_t n = 0;
+    double delta = 0, delta_max = 0;
+    uint32_t tau = 0, tau_max = 0;
+    float lr = 0;
+    int grad_dtype = DECO_F32;
+    int lr_at_server = 0;
+    int select_mode = DECO_SELECT_AUTO;
+    int device = 0;
+    // derived
+    uint64_t k = 0, k_cap = 0;
+    uint64_t e_stride = 0;      // floats per worker row of e (multiple of TILE)
+    uint32_t ntiles = 0;
+    uint32_t ring = 0;          // tau_max + 1 slots
+    uint64_t stage_cap = 0;     // staged candidates per worker
+    // device memory
+    float *e = nullptr;
+    float *params = nullptr;
+    bool own_params = false;
+    deco_pair *msg = nullptr;
+    deco_pair *slots = nullptr;         // [ring][n * k_cap]
+    deco_pair *stage = nullptr;         // [n][stage_cap]
+    uint32_t *hist = nullptr;           // [n][RADIX_LEVELS][RADIX_BINS]
+    deco::SelectState *sel = nullptr;   // [n]
+    uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
+    uint32_t *tile_eq = nullptr;        // [n][ntiles]  entries equal to it per tile
+    uint32_t *tile_take = nullptr;      // [n][ntiles]  ties taken per tile
+    uint32_t *tile_start = nullptr;     // [n][ntiles + 1] message position of each tile
+    uint32_t *tile_off = nullptr;       // [n][ntiles]  staging offset of each tile's candidates
+    uint32_t *tile_cnt = nullptr;       // [n][ntiles]  staged candidates per tile
+    uint32_t *sample_keys = nullptr;    // [n][sample_cap]
+    uint32_t *dev_status = nullptr;     // [4]: status, detail words
+    void *grads_staging = nullptr;      // device copy of host gradients (deco_step_host)
+    uint64_t device_bytes = 0;
+    // host bookkeeping
+    uint64_t t = 0;
+    int phase = 0;                      // 0: expect compress, 1: aggregate, 2: apply
+    std::vector<deco::Slot> slot_info;
+    uint64_t launches = 0;
+    uint64_t k_of_msg = 0;              // k used by the last compress
+};
+
+namespace deco {
+
+// --- kernel launchers (deco_compress.cu) -------------------------------------------------
+cudaError_t launch_begin_step(deco_ctx *c, cudaStream_t s);
+cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s);
+cudaError_t launch_exact_selection(deco_ctx *c, cudaStream_t s);
+// --- kernel launchers (deco_server.cu) ---------------------------------------------------
+cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s);
+cudaError_t launch_apply(deco_ctx *c, const deco_pair *slot, uint64_t positions, float neg_scale,
+                         cudaStream_t s);
+
+}  // namespace deco

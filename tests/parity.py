@@ -1,0 +1,117 @@
+"""Shared driver of the GPU parity tests: runs libdeco (through the C-ABI binding) and the
+CPU oracle side by side on the same seeded gradients and compares every output.
+
+Acceptance (written here once, used by every parity test):
+  * selected indices per worker: identical arrays (both sides store them ascending);
+  * message values and the residual e: identical bit patterns;
+  * aggregated values and parameters: identical bit patterns are expected because both sides
+    sum in worker order; the stated bar is |a-b| <= rtol*max(|a|,|b|) + rtol*A with
+    rtol = 1e-6 (fp32 gradients) or 1e-2 (bf16 gradients) against the float64 shadow, where
+    A is the mean magnitude of the summed terms (guards cancellation).
+"""
+import numpy as np
+import torch
+
+from oracle import dd_ef_sgd as O
+from paper_2507_17346_b200 import binding as B
+from paper_2507_17346_b200 import workloads as W
+
+
+def read_messages(ctx, n, k, device=0):
+    buf = B.deco_get_buffers(ctx)
+    raw = B.view_i32(buf["msg"], (n, buf["k_cap"], 2), device)[:, :k, :].cpu().numpy()
+    idx = raw[:, :, 0].view(np.uint32)
+    val = np.ascontiguousarray(raw[:, :, 1]).view(np.float32)
+    return idx, val
+
+
+def read_e(ctx, n, d, device=0):
+    buf = B.deco_get_buffers(ctx)
+    full = B.view_f32(buf["e"], (n, buf["e_stride"]), device)
+    pad = full[:, d:]
+    assert pad.numel() == 0 or bool((pad == 0).all()), "padding of e must stay zero"
+    return full[:, :d].cpu().numpy()
+
+
+def read_params(ctx, d, device=0):
+    buf = B.deco_get_buffers(ctx)
+    return B.view_f32(buf["params"], (d,), device).cpu().numpy()
+
+
+def read_aggregate(ctx, step, device=0):
+    addr, positions = B.deco_get_aggregate(ctx, step)
+    raw = B.view_i32(addr, (positions, 2), device).cpu().numpy()
+    idx = raw[:, 0].view(np.uint32)
+    val = np.ascontiguousarray(raw[:, 1]).view(np.float32)
+    keep = idx != np.uint32(B.DECO_NO_INDEX)
+    return idx[keep], val[keep]
+
+
+def bits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def close(a, b64, scale_terms, rtol):
+    a = a.astype(np.float64)
+    return np.all(np.abs(a - b64) <= rtol * np.maximum(np.abs(a), np.abs(b64)) + rtol * scale_terms)
+
+
+def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mode=None,
+               policy_plan=None, lr_at_server=False, tau_max=0, delta_max=0.0, device=0,
+               check_every=1, expect_exact=None):
+    """grad_fn(step) -> torch CUDA tensor [n, d] (float32 or bfloat16).
+
+    policy_plan: {step: (delta, tau)} applied before that step on both sides."""
+    rtol = 1e-6 if grad_dtype == "f32" else 1e-2
+    mode = B.DECO_SELECT_AUTO if select_mode is None else select_mode
+    ctx = B.deco_init(d, n, delta, tau, lr,
+                      grad_dtype=B.DECO_F32 if grad_dtype == "f32" else B.DECO_BF16,
+                      tau_max=tau_max, delta_max=delta_max, lr_at_server=lr_at_server,
+                      device=device, select_mode=mode)
+    try:
+        orc = O.DDEFSGD(d, n, delta, tau, lr, lr_in_compress=not lr_at_server)
+        assert B.deco_get_k(ctx) == orc.k
+        for t in range(steps):
+            if policy_plan and t in policy_plan:
+                B.deco_set_policy(ctx, *policy_plan[t])
+                orc.set_policy(*policy_plan[t])
+                assert B.deco_get_k(ctx) == orc.k
+            g = grad_fn(t)
+            assert g.is_cuda and g.shape == (n, d)
+            ref = orc.step(W.to_numpy_bits(g))
+            k = ref["k"]
+            B.deco_ef_compress(ctx, g)
+            check = (t % check_every == 0) or t == steps - 1
+            if check:
+                idx, val = read_messages(ctx, n, k, device)
+                for i, (sel, vals) in enumerate(ref["msgs"]):
+                    assert np.array_equal(idx[i], sel), "step %d worker %d: index set" % (t, i)
+                    assert np.array_equal(bits(val[i]), bits(vals)), \
+                        "step %d worker %d: message values" % (t, i)
+                e = read_e(ctx, n, d, device)
+                assert np.array_equal(bits(e), bits(orc.e)), "step %d: residual" % t
+                if expect_exact is not None:
+                    _, _, ex = B.deco_get_select_info(ctx, n)
+                    assert all(bool(x) == expect_exact for x in ex), (t, ex)
+            B.deco_aggregate_stale(ctx)
+            if check:
+                aidx, aval = read_aggregate(ctx, t, device)
+                touched = np.unique(np.concatenate([s for s, _ in ref["msgs"]]))
+                assert np.array_equal(aidx, touched), "step %d: aggregate index set" % t
+                terms = np.zeros(d)
+                for s, v in ref["msgs"]:
+                    terms[s] += np.abs(v.astype(np.float64))
+                assert close(aval, ref["S64"][touched], terms[touched] / n, rtol)
+                assert np.array_equal(bits(aval), bits(ref["S"][touched])), \
+                    "step %d: aggregate not the worker-order fp32 sum" % t
+            B.deco_apply_update(ctx)
+            if check:
+                x = read_params(ctx, d, device)
+                assert close(x, orc.x64, np.abs(orc.x64) * 0 + float(np.abs(orc.x64).mean()), rtol)
+                assert np.array_equal(bits(x), bits(orc.x)), "step %d: parameters" % t
+        st = B.deco_get_stats(ctx)
+        assert st["device_status"] == 0 and st["step"] == steps
+        assert st["cached_aggregates"] == len(orc.in_flight())
+        return st
+    finally:
+        B.deco_destroy(ctx)

@@ -1,0 +1,176 @@
+"""GPU parity: libdeco (through the C-ABI) against the CPU oracle, element by element, on the
+same seeded inputs.  Sizes span several tiles of 8192 entries plus ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_17346_b200 import binding as B
+from paper_2507_17346_b200 import workloads as W
+from tests.parity import run_parity
+
+pytestmark = pytest.mark.gpu
+
+MODES = [B.DECO_SELECT_EXACT_PASSES, B.DECO_SELECT_AUTO]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2507_17346_b200 import build
+    build.build()
+    B.load()
+
+
+def _values(kind, n, d, step, dtype):
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1000 * step + d + 7 * n)
+    if kind == "normal":
+        x = torch.randn((n, d), generator=g, device="cuda")
+    elif kind == "all_equal":
+        x = torch.full((n, d), -1.5, device="cuda")
+    elif kind == "all_zero":
+        x = torch.zeros((n, d), device="cuda")
+    elif kind == "two_valued":
+        x = torch.where(torch.rand((n, d), generator=g, device="cuda") < 0.3, 2.0, -0.25)
+    elif kind == "signed_zero":
+        r = torch.rand((n, d), generator=g, device="cuda")
+        x = torch.where(r < 0.4, 0.0, torch.where(r < 0.8, -0.0, 1.0))
+    elif kind == "coarse":                                  # few distinct magnitudes
+        x = torch.randint(-8, 9, (n, d), generator=g, device="cuda").float() / 8.0
+    else:
+        raise KeyError(kind)
+    return x.to(dtype).contiguous()
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("kind", ["normal", "all_equal", "all_zero", "two_valued",
+                                  "signed_zero", "coarse"])
+def test_tiny_and_ragged_shapes(kind, mode):
+    for d, n, delta in [(1, 1, 1.0), (3, 2, 0.5), (31, 3, 0.1), (4097, 2, 0.01),
+                        (8192, 1, 0.3), (8193, 3, 0.02), (20001, 2, 1.0), (24576, 2, 1e-9)]:
+        for dtype, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+            run_parity(d, n, delta, 1, 0.1, lambda t: _values(kind, n, d, t, dtype), steps=3,
+                       grad_dtype=name, select_mode=mode)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_flat_1m_all_steps(mode):
+    wl = W.make_workload("flat_1m")
+    run_parity(wl.d, wl.n, wl.delta, wl.tau, wl.lr, lambda t: W.gradients(wl, t, "cuda"),
+               steps=wl.steps, grad_dtype=wl.grad_dtype, select_mode=mode)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("name,scale,steps", [("resnet18", 0.25, 8), ("gpt2_small", 0.08, 6),
+                                              ("decoder_1b", 0.03, 6)])
+def test_scaled_workloads(name, scale, steps, mode):
+    wl = W.make_workload(name, scale)
+    run_parity(wl.d, wl.n, wl.delta, wl.tau, wl.lr, lambda t: W.gradients(wl, t, "cuda"),
+               steps=steps, grad_dtype=wl.grad_dtype, select_mode=mode)
+
+
+def test_resnet18_full_size():
+    wl = W.make_workload("resnet18")
+    assert wl.d == 11_689_512 and len(wl.tensors) == 62
+    run_parity(wl.d, wl.n, wl.delta, wl.tau, wl.lr, lambda t: W.gradients(wl, t, "cuda"),
+               steps=6, grad_dtype=wl.grad_dtype)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_policy_changes_at_run_time(mode):
+    d, n = 300_000, 4
+    plan = {3: (0.05, 1), 6: (0.001, 4), 9: (0.1, 0), 12: (0.0001, 2)}
+    wl = W.make_workload("sweep_100m", 0.003)
+    assert wl.d == d
+    run_parity(d, n, 0.01, 2, 0.1, lambda t: W.gradients(wl, t, "cuda"), steps=16,
+               policy_plan=plan, tau_max=4, delta_max=0.1, select_mode=mode)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_degradation_to_dsgd_and_stepsize_at_server(mode):
+    d, n = 50_000, 4
+    wl = W.make_workload("sweep_100m", 0.0005)
+    assert wl.d == d
+    run_parity(d, n, 1.0, 0, 0.1, lambda t: W.gradients(wl, t, "cuda"), steps=4,
+               select_mode=mode)                                    # delta = 1, tau = 0: D-SGD
+    run_parity(d, n, 1.0, 3, 0.1, lambda t: W.gradients(wl, t, "cuda"), steps=6,
+               select_mode=mode)                                    # delayed aggregation only
+    run_parity(d, n, 0.02, 2, 0.25, lambda t: W.gradients(wl, t, "cuda"), steps=6,
+               lr_at_server=True, select_mode=mode)
+
+
+def test_call_order_and_capacity_errors():
+    d, n = 10_000, 2
+    ctx = B.deco_init(d, n, 0.01, 1, 0.1, tau_max=2, delta_max=0.05)
+    try:
+        g = torch.randn((n, d), device="cuda")
+        with pytest.raises(B.DecoError) as e:
+            B.deco_aggregate_stale(ctx)
+        assert e.value.status == B.DECO_ERR_STATE
+        with pytest.raises(B.DecoError) as e:
+            B.deco_apply_update(ctx)
+        assert e.value.status == B.DECO_ERR_STATE
+        B.deco_ef_compress(ctx, g)
+        with pytest.raises(B.DecoError) as e:
+            B.deco_ef_compress(ctx, g)
+        assert e.value.status == B.DECO_ERR_STATE
+        with pytest.raises(B.DecoError) as e:
+            B.deco_set_policy(ctx, 0.02, 1)
+        assert e.value.status == B.DECO_ERR_STATE
+        B.deco_aggregate_stale(ctx)
+        B.deco_apply_update(ctx)
+        for delta, tau in ((0.06, 1), (0.01, 3)):
+            with pytest.raises(B.DecoError) as e:
+                B.deco_set_policy(ctx, delta, tau)
+            assert e.value.status == B.DECO_ERR_CAPACITY
+        assert B.deco_get_k(ctx) == 100                              # unchanged
+        B.deco_set_policy(ctx, 0.05, 2)
+        assert B.deco_get_k(ctx) == 500
+        with pytest.raises(B.DecoError) as e:
+            B.deco_ef_compress(ctx, g[:, 1:])                        # misaligned base pointer
+        assert e.value.status == B.DECO_ERR_INVALID_ARG
+        assert B.deco_get_stats(ctx)["step"] == 1
+    finally:
+        B.deco_destroy(ctx)
+
+
+def test_two_runs_give_the_same_bits():
+    wl = W.make_workload("resnet18", 0.25)
+    outs = []
+    for _ in range(2):
+        ctx = B.deco_init(wl.d, wl.n, wl.delta, wl.tau, wl.lr)
+        try:
+            for t in range(6):
+                B.deco_step(ctx, W.gradients(wl, t, "cuda"))
+            buf = B.deco_get_buffers(ctx)
+            outs.append((B.view_i32(buf["e"], (wl.n, buf["e_stride"])).clone(),
+                         B.view_i32(buf["params"], (wl.d,)).clone(),
+                         B.view_i32(buf["msg"], (wl.n, buf["k_cap"], 2)).clone()))
+            assert B.deco_get_stats(ctx)["device_status"] == 0
+        finally:
+            B.deco_destroy(ctx)
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_host_buffer_step_matches_device_step():
+    wl = W.make_workload("resnet18", 0.25)
+    k = B.deco_k_from_delta(wl.delta, wl.d)
+    a = B.deco_init(wl.d, wl.n, wl.delta, wl.tau, wl.lr)
+    b = B.deco_init(wl.d, wl.n, wl.delta, wl.tau, wl.lr)
+    try:
+        msg_host = torch.empty((wl.n, k, 2), dtype=torch.int32).pin_memory()
+        x_host = torch.empty(wl.d, dtype=torch.float32).pin_memory()
+        for t in range(6):
+            g = W.gradients(wl, t, "cuda")
+            g_host = g.cpu().pin_memory()
+            B.deco_step(a, g)
+            B.deco_step_host(b, g_host, msg_host, x_host)
+            torch.cuda.synchronize()
+            buf = B.deco_get_buffers(a)
+            want_msg = B.view_i32(buf["msg"], (wl.n, buf["k_cap"], 2))[:, :k].cpu()
+            want_x = B.view_f32(buf["params"], (wl.d,)).cpu()
+            assert torch.equal(msg_host, want_msg)
+            assert torch.equal(x_host.view(torch.int32), want_x.view(torch.int32))
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
