@@ -7,7 +7,7 @@ Acceptance (written here once, used by every parity test):
   * aggregated values and parameters: identical bit patterns are expected because both sides
     sum in worker order; the stated bar is |a-b| <= rtol*max(|a|,|b|) + rtol*A with
     rtol = 1e-6 (fp32 gradients) or 1e-2 (bf16 gradients) against the float64 shadow, where
-    A is the mean magnitude of the summed terms (guards cancellation).
+    A is the magnitude of the summed terms (per-entry sum of |term|; guards cancellation).
 """
 import numpy as np
 import torch
@@ -71,6 +71,8 @@ def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mo
     try:
         orc = O.DDEFSGD(d, n, delta, tau, lr, lr_in_compress=not lr_at_server)
         assert B.deco_get_k(ctx) == orc.k
+        abs_S, mass = {}, np.zeros(d)
+        scale = float(np.float32(1.0 if not lr_at_server else lr) / np.float32(n))
         for t in range(steps):
             if policy_plan and t in policy_plan:
                 B.deco_set_policy(ctx, *policy_plan[t])
@@ -94,6 +96,9 @@ def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mo
                     _, _, ex = B.deco_get_select_info(ctx, n)
                     assert all(bool(x) == expect_exact for x in ex), (t, ex)
             B.deco_aggregate_stale(ctx)
+            terms = np.zeros(d)                                # per-entry sum of |term|
+            for s, v in ref["msgs"]:
+                terms[s] += np.abs(v.astype(np.float64))
             if check:
                 aidx, aval = read_aggregate(ctx, t, device)
                 touched = np.unique(np.concatenate([s for s, _ in ref["msgs"]]))
@@ -105,9 +110,12 @@ def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mo
                 assert np.array_equal(bits(aval), bits(ref["S"][touched])), \
                     "step %d: aggregate not the worker-order fp32 sum" % t
             B.deco_apply_update(ctx)
+            abs_S[t] = terms
+            for s_applied in ref["applied"]:
+                mass += scale * abs_S.pop(s_applied)          # magnitude of the summed terms
             if check:
                 x = read_params(ctx, d, device)
-                assert close(x, orc.x64, np.abs(orc.x64) * 0 + float(np.abs(orc.x64).mean()), rtol)
+                assert close(x, orc.x64, mass, rtol), "step %d: parameters vs float64" % t
                 assert np.array_equal(bits(x), bits(orc.x)), "step %d: parameters" % t
         st = B.deco_get_stats(ctx)
         assert st["device_status"] == 0 and st["step"] == steps
