@@ -230,6 +230,18 @@ deco_status deco_get_select_info(deco_ctx *ctx, void *stream, uint32_t *threshol
  * latched an anomaly since the context was created or reset. */
 deco_status deco_get_stats(deco_ctx *ctx, void *stream, deco_stats *out);
 
+/*
+ * Optional device timing with CUDA events recorded on the caller's stream around the parts of
+ * an iteration.  While enabled (up to 4096 iterations are kept) every iteration records
+ * events around: [0] the streaming accumulate kernel, [1] the rest of deco_ef_compress
+ * (selection and message build), [2] deco_aggregate_stale, [3] deco_apply_update.
+ * deco_get_kernel_timing waits for `stream`, returns the summed milliseconds per part in
+ * ms_sum[4] (HOST) and the number of iterations they cover, and clears the record.
+ */
+deco_status deco_set_kernel_timing(deco_ctx *ctx, int32_t enabled);
+deco_status deco_get_kernel_timing(deco_ctx *ctx, void *stream, double *ms_sum /* [4] */,
+                                   uint64_t *iterations);
+
 /* Number of kernels and memset/memcpy nodes the library has enqueued so far. */
 uint64_t deco_launch_count(const deco_ctx *ctx);
 

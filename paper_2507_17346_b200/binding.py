@@ -85,6 +85,8 @@ SIGNATURES = {
     "deco_get_aggregate": (_i32, [_vp, _u64, _P(_vp), _P(_u64)]),
     "deco_get_select_info": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "deco_get_stats": (_i32, [_vp, _vp, _P(deco_stats)]),
+    "deco_set_kernel_timing": (_i32, [_vp, _i32]),
+    "deco_get_kernel_timing": (_i32, [_vp, _vp, _P(_f64), _P(_u64)]),
     "deco_launch_count": (_u64, [_vp]),
     "deco_status_string": (ctypes.c_char_p, [_i32]),
 }
@@ -246,6 +248,19 @@ def deco_get_stats(ctx, stream=None):
     st = deco_stats()
     _check(load().deco_get_stats(ctx, _stream(stream), ctypes.byref(st)), "deco_get_stats")
     return {f: getattr(st, f) for f, _ in deco_stats._fields_}
+
+
+def deco_set_kernel_timing(ctx, enabled):
+    _check(load().deco_set_kernel_timing(ctx, int(bool(enabled))), "deco_set_kernel_timing")
+
+
+def deco_get_kernel_timing(ctx, stream=None):
+    """-> ({'accumulate','select','aggregate','apply'}: summed ms, iterations covered)."""
+    ms = (_f64 * 4)()
+    it = _u64()
+    _check(load().deco_get_kernel_timing(ctx, _stream(stream), ms, ctypes.byref(it)),
+           "deco_get_kernel_timing")
+    return dict(zip(("accumulate", "select", "aggregate", "apply"), list(ms))), it.value
 
 
 def deco_launch_count(ctx):

@@ -53,9 +53,11 @@ void free_all(deco_ctx *c)
     cudaFree(c->tile_start);
     cudaFree(c->tile_off);
     cudaFree(c->tile_cnt);
-    cudaFree(c->sample_keys);
+    cudaFree(c->done);
     cudaFree(c->dev_status);
     cudaFree(c->grads_staging);
+    for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
+    c->events.clear();
 }
 
 deco_status zero_state(deco_ctx *c, cudaStream_t s)
@@ -75,6 +77,21 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
 }
 
 inline cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
+
+constexpr size_t MAX_TIMED_ITERS = 4096;
+
+// Record event `which` (0..7) of the iteration being timed, if timing is on and there is room.
+void mark(deco_ctx *c, int which, cudaStream_t s)
+{
+    if (!c->timing || c->timed_iters >= MAX_TIMED_ITERS) return;
+    const size_t need = (c->timed_iters + 1) * 8;
+    while (c->events.size() < need) {
+        cudaEvent_t ev = nullptr;
+        if (cudaEventCreate(&ev) != cudaSuccess) { c->timing = false; return; }
+        c->events.push_back(ev);
+    }
+    cudaEventRecord(c->events[c->timed_iters * 8 + which], s);
+}
 
 }  // namespace
 
@@ -140,8 +157,8 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     c->ntiles = static_cast<uint32_t>((d + TILE - 1) / TILE);
     c->e_stride = static_cast<uint64_t>(c->ntiles) * TILE;
     c->ring = c->tau_max + 1;
-    // staged candidates per worker: four times the message capacity plus slack, at most d
-    c->stage_cap = 4 * c->k_cap + 65536;
+    // staged candidates per worker: six times the message capacity plus slack, at most d
+    c->stage_cap = 6 * c->k_cap + 65536;
     if (c->stage_cap > c->e_stride) c->stage_cap = c->e_stride;
     try {
         c->slot_info.resize(c->ring);
@@ -162,7 +179,8 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->msg, static_cast<uint64_t>(n) * c->k_cap));
     need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * n * c->k_cap));
     need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
-    need(dev_alloc(c, &c->hist, static_cast<uint64_t>(n) * RADIX_LEVELS * RADIX_BINS));
+    need(dev_alloc(c, &c->hist, static_cast<uint64_t>(n) * 2 * RADIX_LEVELS * RADIX_BINS));
+    need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * RADIX_LEVELS));
     need(dev_alloc(c, &c->sel, n));
     need(dev_alloc(c, &c->tile_gt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_eq, static_cast<uint64_t>(n) * c->ntiles));
@@ -171,6 +189,7 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->tile_off, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_cnt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->dev_status, 4));
+    if (st == DECO_OK && query_fallback_grid(c) != cudaSuccess) st = DECO_ERR_CUDA;
     if (st == DECO_OK) st = zero_state(c, nullptr);
     if (st == DECO_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = DECO_ERR_CUDA;
     if (st != DECO_OK) {
@@ -209,9 +228,12 @@ extern "C" deco_status deco_ef_compress(deco_ctx *c, const void *grads, void *st
     if (!guard.ok) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);
     c->k_of_msg = c->k;
-    cudaError_t err = launch_begin_step(c, s);
+    cudaError_t err = launch_begin_step(c, grads, s);
+    mark(c, 0, s);
     if (err == cudaSuccess) err = launch_accumulate(c, grads, s);
-    if (err == cudaSuccess) err = launch_exact_selection(c, s);
+    mark(c, 1, s);
+    if (err == cudaSuccess) err = launch_selection(c, s);
+    mark(c, 2, s);
     if (err != cudaSuccess) return DECO_ERR_CUDA;
     c->phase = 1;
     return DECO_OK;
@@ -227,7 +249,9 @@ extern "C" deco_status deco_aggregate_stale(deco_ctx *c, void *stream)
     Slot &sl = c->slot_info[si];
     if (sl.valid) return DECO_ERR_STATE;    // cannot happen while tau <= tau_max
     deco_pair *slot = c->slots + static_cast<uint64_t>(si) * c->n * c->k_cap;
+    mark(c, 3, as_stream(stream));
     if (launch_aggregate(c, slot, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    mark(c, 4, as_stream(stream));
     sl.step = c->t;
     sl.positions = static_cast<uint64_t>(c->n) * c->k_of_msg;
     sl.valid = true;
@@ -243,6 +267,7 @@ extern "C" deco_status deco_apply_update(deco_ctx *c, void *stream)
     if (!guard.ok) return DECO_ERR_CUDA;
     const float beta = c->lr_at_server ? c->lr : 1.0f;
     const float neg_scale = -(beta / static_cast<float>(c->n));
+    mark(c, 5, as_stream(stream));
     if (c->t >= c->tau) {
         const uint64_t due = c->t - c->tau;
         // oldest first: step ids still cached lie in (t - ring, t]
@@ -256,8 +281,42 @@ extern "C" deco_status deco_apply_update(deco_ctx *c, void *stream)
             sl.valid = false;
         }
     }
+    mark(c, 6, as_stream(stream));
+    if (c->timing && c->timed_iters < MAX_TIMED_ITERS) c->timed_iters += 1;
     c->t += 1;
     c->phase = 0;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_set_kernel_timing(deco_ctx *c, int32_t enabled)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    c->timing = enabled != 0;
+    c->timed_iters = 0;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_get_kernel_timing(deco_ctx *c, void *stream, double *ms_sum,
+                                              uint64_t *iterations)
+{
+    if (!c || !ms_sum || !iterations) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    static const int pairs[4][2] = {{0, 1}, {1, 2}, {3, 4}, {5, 6}};
+    for (int p = 0; p < 4; ++p) ms_sum[p] = 0.0;
+    for (size_t it = 0; it < c->timed_iters; ++it)
+        for (int p = 0; p < 4; ++p) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, c->events[it * 8 + pairs[p][0]],
+                                     c->events[it * 8 + pairs[p][1]]) != cudaSuccess)
+                return DECO_ERR_CUDA;
+            ms_sum[p] += ms;
+        }
+    *iterations = c->timed_iters;
+    c->timed_iters = 0;
     return DECO_OK;
 }
 

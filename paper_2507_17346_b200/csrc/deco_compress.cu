@@ -1,22 +1,55 @@
 // Worker side of Algorithm 1 on the device: a = e + gamma*g, exact Top-k of |a| with ties to
 // the lower index, messages as packed (index, value) pairs sorted by index, residual in e.
 //
-// Kernels in this file
-//   ef_accumulate_kernel   streaming pass: reads e and g once, writes a into e
-//   radix_hist_e_kernel    histogram of one radix level of the magnitude keys of a
-//   radix_pick_kernel      walks a histogram from the top and fixes the next key bits
-//   tile_count_e_kernel    per tile: entries above / equal to the threshold
-//   tile_scan_kernel       per worker: prefix sums over tiles -> message position of each tile
-//   emit_e_kernel          ordered compaction of the selected entries, zeroing them in e
+// Two routes give the same bits.
+//
+// Streaming route (DECO_SELECT_AUTO): a small sample of a fixes, per worker, a lower bound
+// `spec_key` that is below the k-th largest magnitude with overwhelming probability.  One pass
+// reads e and g, writes a into e and stages every entry whose key reaches the bound (a few
+// times k pairs, each tile's entries in index order).  The exact threshold is then found by
+// a three-level radix selection over the staged pairs only, and the message is an ordered
+// filter of them.  The count of staged pairs proves the bound was valid (>= k of them); if it
+// was not, or the staging area overflowed, that worker takes the second route in the same
+// call.
+//
+// Multi-pass route (DECO_SELECT_EXACT_PASSES, and the fallback of the first): three radix
+// histogram passes over e fix the threshold key, one pass counts per tile, one pass emits.
+// It handles any input (all entries equal, all zero, k = d ...).
+//
+// Entry order inside a tile is (warp, round, lane, component): warp w owns WARP_ELEMS
+// consecutive entries, and in round u lane l owns V consecutive ones, so each warp-level
+// load is one contiguous 512-byte request.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include "deco_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace deco {
 
 namespace {
 
 constexpr uint32_t FULL = 0xFFFFFFFFu;
+
+// Everything the selection kernels need, passed by value.
+struct Sel {
+    float *e;
+    uint64_t e_stride;
+    uint64_t d;
+    uint32_t n;
+    uint32_t ntiles;
+    uint32_t k;
+    SelectState *sel;
+    uint32_t *hist;          // [n][2][RADIX_LEVELS][RADIX_BINS]: 0 = staged route, 1 = multi-pass
+    uint32_t *done;          // [n][RADIX_LEVELS] CTA arrival counters of the staged route
+    uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt;
+    deco_pair *msg;
+    uint64_t k_cap;
+    deco_pair *stage;
+    uint64_t stage_cap;
+    uint32_t *status;        // [0] latched status, [1..2] detail, [3] "some worker needs the multi-pass route"
+};
 
 __device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
 
@@ -26,6 +59,11 @@ __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t 
         status[1] = a;
         status[2] = b;
     }
+}
+
+__device__ __forceinline__ uint32_t *hist_of(const Sel &p, uint32_t i, int route, int level)
+{
+    return p.hist + ((static_cast<size_t>(i) * 2 + route) * RADIX_LEVELS + level) * RADIX_BINS;
 }
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v)
@@ -68,15 +106,30 @@ __device__ __forceinline__ void ordered_prefix(const uint32_t (&cnt)[U], uint32_
     __syncthreads();
 }
 
+// Exclusive scan over the CTA (any multiple of 32 threads up to 1024); s_w has 33 words.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_w, uint32_t &total)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int nw = blockDim.x >> 5;
+    const uint32_t incl = warp_incl_scan(v);
+    if (lane == 31) s_w[w] = incl;
+    __syncthreads();
+    if (w == 0) {
+        const uint32_t x = lane < nw ? s_w[lane] : 0u;
+        const uint32_t xi = warp_incl_scan(x);
+        s_w[lane] = xi - x;
+        if (lane == 31) s_w[32] = xi;
+    }
+    __syncthreads();
+    const uint32_t out = s_w[w] + incl - v;
+    total = s_w[32];
+    __syncthreads();
+    return out;
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// ------------------------------------------------------------------------------------------
-// Streaming pass.  GT = 0: fp32 gradients, 4 entries per thread and round; GT = 1: bfloat16
-// gradients, 8 entries per thread and round.  ALIGNED: every gradient row starts on a
-// 16-byte boundary, so whole tiles are read with 128-bit loads; otherwise (and in the tile
-// that contains the end of the vector) gradients are read entry by entry.
-// ------------------------------------------------------------------------------------------
 template <int GT>
 struct Geo {
     static constexpr int V = GT ? 8 : 4;                 // entries per thread and round
@@ -93,6 +146,200 @@ __device__ __forceinline__ float load_g(const void *grow, uint64_t j)
     return reinterpret_cast<const float *>(grow)[j];
 }
 
+// ------------------------------------------------------------------------------------------
+// Radix helpers shared by both routes: 31-bit key = 12 + 12 + 7 bits.
+// ------------------------------------------------------------------------------------------
+template <int LEVEL>
+__device__ __forceinline__ void radix_bin(uint32_t key, uint32_t prefix, uint32_t *h)
+{
+    if (LEVEL == 0) {
+        atomicAdd(&h[key >> 19], 1u);
+    } else if (LEVEL == 1) {
+        if ((key >> 19) == prefix) atomicAdd(&h[(key >> 7) & 0xFFFu], 1u);
+    } else {
+        if ((key >> 7) == prefix) atomicAdd(&h[key & 0x7Fu], 1u);
+    }
+}
+
+// One CTA (BLOCK threads).  Finds the bin b with  count(bins > b) < k_rem <= count(bins >= b)
+// in histogram h and appends it to the key prefix of s.  After the last level the prefix is
+// the threshold key.  suf: BLOCK + 1 words of shared memory.
+template <int LEVEL>
+__device__ __forceinline__ void pick_body(SelectState &s, const uint32_t *h, uint32_t *suf,
+                                          uint32_t *status, uint32_t i)
+{
+    constexpr int BITS = (LEVEL == 2) ? 7 : 12;
+    constexpr int PER = RADIX_BINS / BLOCK;   // 16 bins per thread
+    const uint32_t k_rem = s.k_rem;
+    const int t = threadIdx.x;
+    uint32_t loc[PER], sum = 0;
+#pragma unroll
+    for (int b = 0; b < PER; ++b) {
+        loc[b] = __ldcg(&h[t * PER + b]);
+        sum += loc[b];
+    }
+    suf[t] = sum;
+    if (t == 0) suf[BLOCK] = 0;
+    __syncthreads();
+    for (int o = 1; o < BLOCK; o <<= 1) {      // inclusive suffix sums over threads
+        const uint32_t v = (t + o < BLOCK) ? suf[t + o] : 0u;
+        __syncthreads();
+        suf[t] += v;
+        __syncthreads();
+    }
+    const uint32_t s_here = suf[t], s_above = suf[t + 1];
+    if (t == 0 && s_here < k_rem) latch(status, DECO_ERR_DEVICE_CHECK, 0x100u + LEVEL, i);
+    if (s_here >= k_rem && s_above < k_rem) {
+        uint32_t acc = s_above;
+        int bin = t * PER;
+#pragma unroll
+        for (int b = PER - 1; b >= 0; --b) {
+            if (acc + loc[b] >= k_rem) {
+                bin = t * PER + b;
+                break;
+            }
+            acc += loc[b];
+        }
+        s.n_greater += acc;
+        s.k_rem = k_rem - acc;
+        const uint32_t prefix = (s.prefix << BITS) | static_cast<uint32_t>(bin);
+        s.prefix = prefix;
+        if (LEVEL == 2) {
+            s.threshold = prefix;
+            s.ties_take = k_rem - acc;
+        }
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------
+// Start of an iteration: one CTA per worker re-arms the selection record, clears the
+// histograms and, on the streaming route, draws the sample that fixes spec_key.
+// ------------------------------------------------------------------------------------------
+constexpr int BEGIN_BLOCK = 1024;
+constexpr int SAMPLE_CHUNKS = 8192;                        // 4 consecutive entries each
+constexpr int SAMPLE_PER_THREAD = SAMPLE_CHUNKS / BEGIN_BLOCK;   // 8 chunks = 32 keys
+
+template <int GT>
+__global__ void __launch_bounds__(BEGIN_BLOCK)
+begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t exact_all)
+{
+    const uint32_t i = blockIdx.x;
+    const int t = threadIdx.x;
+    SelectState &s = p.sel[i];
+    uint32_t *hz = hist_of(p, i, 0, 0);
+    for (int q = t; q < 2 * RADIX_LEVELS * RADIX_BINS; q += BEGIN_BLOCK) hz[q] = 0;
+    if (t < RADIX_LEVELS) p.done[i * RADIX_LEVELS + t] = 0;
+    if (i == 0 && t == 0) p.status[3] = exact_all;
+    if (t == 0) {
+        s.prefix = 0;
+        s.k_rem = p.k;
+        s.n_greater = 0;
+        s.threshold = 0;
+        s.ties_take = 0;
+        s.exact = exact_all;
+        s.spec_key = SPEC_DISABLED;
+        s.n_staged = 0;
+        if (exact_all) s.exact_total += 1;
+    }
+    if (exact_all) return;
+
+    // ---- sample: SAMPLE_CHUNKS groups of 4 consecutive entries, evenly spread over [0, d)
+    __shared__ uint32_t h[RADIX_BINS];
+    __shared__ uint32_t s_w[33];
+    __shared__ uint32_t s_pick[2];
+    const float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+    const char *grow = reinterpret_cast<const char *>(grads) +
+                       static_cast<size_t>(i) * p.d * (GT ? 2 : 4);
+    const uint64_t nchunks = (p.d + 3) >> 2;
+    const uint32_t S = nchunks < SAMPLE_CHUNKS ? static_cast<uint32_t>(nchunks) : SAMPLE_CHUNKS;
+    uint32_t keys[SAMPLE_PER_THREAD * 4];
+    uint32_t valid = 0;
+#pragma unroll
+    for (int q = 0; q < SAMPLE_PER_THREAD; ++q) {
+        const uint32_t sidx = q * BEGIN_BLOCK + t;
+        uint64_t j = 0;
+        const bool on = sidx < S;
+        if (on) j = ((static_cast<uint64_t>(sidx) * nchunks) / S) << 2;
+        float4 ev = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (on) ev = *reinterpret_cast<const float4 *>(erow + j);
+        const float es[4] = {ev.x, ev.y, ev.z, ev.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const bool in = on && (j + c < p.d);
+            uint32_t key = 0xFFFFFFFFu;                      // marks "not a sample"
+            if (in) key = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
+            keys[q * 4 + c] = key;
+            valid += in ? 1u : 0u;
+        }
+    }
+    uint32_t m_total;
+    block_excl_scan(valid, s_w, m_total);
+    // rank inside the sample: mean + 5 sigma + 2 of a binomial with p = k/d (exact when the
+    // sample is the whole vector)
+    uint32_t R;
+    if (m_total >= p.d) {
+        R = p.k;
+    } else {
+        const double mean = static_cast<double>(p.k) * m_total / static_cast<double>(p.d);
+        const double r = mean + 5.0 * sqrt(mean) + 2.0;
+        R = r >= static_cast<double>(m_total) ? m_total + 1u : static_cast<uint32_t>(r) + 1u;
+    }
+    if (R > m_total) {                         // the sample cannot bound the threshold
+        if (t == 0) s.spec_key = 0;            // stage everything: the count check decides
+        return;
+    }
+    uint32_t prefix = 0, rem = R;
+#pragma unroll 1
+    for (int level = 0; level < 2; ++level) {
+        for (int q = t; q < RADIX_BINS; q += BEGIN_BLOCK) h[q] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < SAMPLE_PER_THREAD * 4; ++q) {
+            const uint32_t key = keys[q];
+            if (key == 0xFFFFFFFFu) continue;
+            if (level == 0) atomicAdd(&h[key >> 19], 1u);
+            else if ((key >> 19) == prefix) atomicAdd(&h[(key >> 7) & 0xFFFu], 1u);
+        }
+        __syncthreads();
+        // suffix pick with 4 bins per thread
+        uint32_t loc[4], sum = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            loc[b] = h[t * 4 + b];
+            sum += loc[b];
+        }
+        uint32_t tot;
+        const uint32_t below = block_excl_scan(sum, s_w, tot);   // bins below this thread's
+        const uint32_t s_here = tot - below, s_above = tot - below - sum;
+        if (s_here >= rem && s_above < rem) {
+            uint32_t acc = s_above;
+            int bin = t * 4;
+#pragma unroll
+            for (int b = 3; b >= 0; --b) {
+                if (acc + loc[b] >= rem) {
+                    bin = t * 4 + b;
+                    break;
+                }
+                acc += loc[b];
+            }
+            s_pick[0] = static_cast<uint32_t>(bin);
+            s_pick[1] = rem - acc;
+        }
+        __syncthreads();
+        prefix = (prefix << 12) | s_pick[0];
+        rem = s_pick[1];
+        __syncthreads();
+    }
+    if (t == 0) s.spec_key = prefix << 7;      // lower edge of the 24-bit bin
+}
+
+// ------------------------------------------------------------------------------------------
+// Streaming pass.  GT = 0: fp32 gradients; GT = 1: bfloat16 gradients.  ALIGNED: every
+// gradient row starts on a 16-byte boundary, so whole tiles are read with 128-bit loads;
+// otherwise (and in the tile that holds the end of the vector) gradients are read entry by
+// entry.  SPEC: stage the entries whose key reaches sel[i].spec_key.
+// ------------------------------------------------------------------------------------------
 template <int GT, bool ALIGNED, bool SPEC>
 __global__ void __launch_bounds__(BLOCK)
 ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
@@ -206,126 +453,185 @@ ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__res
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint64_t j = wbase + u * (32 * V) + lane * V;
-            uint32_t p = pos[u];
+            uint32_t q = pos[u];
 #pragma unroll
             for (int c = 0; c < V; ++c)
                 if (m[u] & (1u << c)) {
                     deco_pair pr;
                     pr.idx = static_cast<uint32_t>(j + c);
                     pr.val = x[u][c];
-                    out[p++] = pr;
+                    out[q++] = pr;
                 }
         }
     }
 }
 
 // ------------------------------------------------------------------------------------------
-// Multi-pass exact selection over e (workers with sel[i].exact != 0).
+// Streaming route: exact selection among the staged pairs.
 // ------------------------------------------------------------------------------------------
+// Histogram of one radix level over the staged pairs of each worker; the last CTA of a worker
+// to arrive (counted with an atomic after a fence, no waiting) does the pick.  At level 0 the
+// pick first checks that the staged set is valid: n_staged in [k, stage_cap].  If not, the
+// worker is handed to the multi-pass route.
 template <int LEVEL>
-__device__ __forceinline__ void radix_bin(uint32_t key, uint32_t prefix, uint32_t *h)
+__global__ void __launch_bounds__(BLOCK)
+stage_hist_pick_kernel(Sel p)
 {
-    if (LEVEL == 0) {
-        atomicAdd(&h[key >> 19], 1u);
-    } else if (LEVEL == 1) {
-        if ((key >> 19) == prefix) atomicAdd(&h[(key >> 7) & 0xFFFu], 1u);
-    } else {
-        if ((key >> 7) == prefix) atomicAdd(&h[key & 0x7Fu], 1u);
+    const uint32_t i = blockIdx.y;
+    SelectState &s = p.sel[i];
+    if (s.exact) return;
+    __shared__ uint32_t h[RADIX_BINS];
+    __shared__ uint32_t suf[BLOCK + 1];
+    __shared__ uint32_t s_last;
+    const uint32_t n_staged = s.n_staged;
+    const bool valid = n_staged >= p.k && n_staged <= p.stage_cap;
+    if (valid) {
+        for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
+        __syncthreads();
+        const uint32_t prefix = s.prefix;
+        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
+        for (uint32_t q = blockIdx.x * BLOCK + threadIdx.x; q < n_staged; q += gridDim.x * BLOCK)
+            radix_bin<LEVEL>(mag_key(src[q].val), prefix, h);
+        __syncthreads();
+        uint32_t *out = hist_of(p, i, 0, LEVEL);
+        for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
+            if (h[b]) atomicAdd(&out[b], h[b]);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0)
+        s_last = (atomicAdd(&p.done[i * RADIX_LEVELS + LEVEL], 1u) == gridDim.x - 1) ? 1u : 0u;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (!valid) {
+        if (threadIdx.x == 0) {
+            s.exact = 1;
+            s.exact_total += 1;
+            p.status[3] = 1;
+        }
+        return;
+    }
+    pick_body<LEVEL>(s, hist_of(p, i, 0, LEVEL), suf, p.status, i);
+}
+
+// One warp per tile: entries above / equal to the threshold among the tile's staged pairs.
+__global__ void __launch_bounds__(BLOCK)
+tile_count_stage_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.y;
+    if (p.sel[i].exact) return;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t tile = blockIdx.x * WARPS + w;
+    if (tile >= p.ntiles) return;
+    const uint32_t T = p.sel[i].threshold;
+    const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
+    const uint32_t cnt = p.tile_cnt[ti];
+    uint32_t gt = 0, eq = 0;
+    if (cnt) {
+        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + p.tile_off[ti];
+        for (uint32_t q = lane; q < cnt; q += 32) {
+            const uint32_t key = mag_key(src[q].val);
+            gt += key > T;
+            eq += key == T;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            gt += __shfl_down_sync(FULL, gt, o);
+            eq += __shfl_down_sync(FULL, eq, o);
+        }
+    }
+    if (lane == 0) {
+        p.tile_gt[ti] = gt;
+        p.tile_eq[ti] = eq;
     }
 }
 
-template <int LEVEL>
+// One warp per tile: ordered filter of the tile's staged pairs into the message; the selected
+// entries become +0 in e.
 __global__ void __launch_bounds__(BLOCK)
-radix_hist_e_kernel(const float *__restrict__ e, uint64_t e_stride, uint64_t d,
-                    const SelectState *__restrict__ sel, uint32_t *__restrict__ hist)
+emit_stage_kernel(Sel p)
 {
     const uint32_t i = blockIdx.y;
-    if (!sel[i].exact) return;
-    __shared__ uint32_t h[RADIX_BINS];
+    if (p.sel[i].exact) return;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t tile = blockIdx.x * WARPS + w;
+    if (tile >= p.ntiles) return;
+    const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
+    const uint32_t cnt = p.tile_cnt[ti];
+    if (cnt == 0) return;
+    const uint32_t start = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile];
+    const uint32_t want = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile + 1] - start;
+    if (want == 0) return;
+    const uint32_t T = p.sel[i].threshold;
+    const uint32_t take = p.tile_take[ti];
+    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + p.tile_off[ti];
+    deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
+    float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+    uint32_t written = 0, ties_seen = 0;
+    for (uint32_t base = 0; base < cnt; base += 32) {
+        const uint32_t q = base + lane;
+        deco_pair pr;
+        pr.idx = 0;
+        pr.val = 0.f;
+        bool gt = false, eq = false;
+        if (q < cnt) {
+            pr = src[q];
+            const uint32_t key = mag_key(pr.val);
+            gt = key > T;
+            eq = key == T;
+        }
+        const uint32_t eq_mask = __ballot_sync(FULL, eq);
+        const uint32_t rank = ties_seen + __popc(eq_mask & ((1u << lane) - 1u));
+        const bool pick = gt || (eq && rank < take);
+        const uint32_t pick_mask = __ballot_sync(FULL, pick);
+        if (pick) {
+            const uint32_t pos = start + written + __popc(pick_mask & ((1u << lane) - 1u));
+            if (pos < p.k && pr.idx < p.d) {
+                out[pos] = pr;
+                erow[pr.idx] = 0.0f;
+            } else {
+                latch(p.status, DECO_ERR_DEVICE_CHECK, 0x310u, tile);
+            }
+        }
+        written += __popc(pick_mask);
+        ties_seen += __popc(eq_mask);
+    }
+    if (lane == 0 && written != want) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x311u, tile);
+}
+
+// ------------------------------------------------------------------------------------------
+// Multi-pass route: bodies written for one CTA of BLOCK threads working on (worker, part).
+// ------------------------------------------------------------------------------------------
+template <int LEVEL>
+__device__ __forceinline__ void hist_e_body(const Sel &p, uint32_t i, uint32_t part,
+                                            uint32_t nparts, uint32_t *h)
+{
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
     __syncthreads();
-    const uint32_t prefix = sel[i].prefix;
-    const float4 *row = reinterpret_cast<const float4 *>(e + static_cast<size_t>(i) * e_stride);
-    const uint64_t nvec = (d + 3) >> 2;
-    for (uint64_t v = static_cast<uint64_t>(blockIdx.x) * BLOCK + threadIdx.x; v < nvec;
-         v += static_cast<uint64_t>(gridDim.x) * BLOCK) {
+    const uint32_t prefix = p.sel[i].prefix;
+    const float4 *row = reinterpret_cast<const float4 *>(p.e + static_cast<size_t>(i) * p.e_stride);
+    const uint64_t nvec = (p.d + 3) >> 2;
+    for (uint64_t v = static_cast<uint64_t>(part) * BLOCK + threadIdx.x; v < nvec;
+         v += static_cast<uint64_t>(nparts) * BLOCK) {
         const float4 q = row[v];
         const uint64_t j = v << 2;
         radix_bin<LEVEL>(mag_key(q.x), prefix, h);
-        if (j + 1 < d) radix_bin<LEVEL>(mag_key(q.y), prefix, h);
-        if (j + 2 < d) radix_bin<LEVEL>(mag_key(q.z), prefix, h);
-        if (j + 3 < d) radix_bin<LEVEL>(mag_key(q.w), prefix, h);
+        if (j + 1 < p.d) radix_bin<LEVEL>(mag_key(q.y), prefix, h);
+        if (j + 2 < p.d) radix_bin<LEVEL>(mag_key(q.z), prefix, h);
+        if (j + 3 < p.d) radix_bin<LEVEL>(mag_key(q.w), prefix, h);
     }
     __syncthreads();
-    uint32_t *out = hist + (static_cast<size_t>(i) * RADIX_LEVELS + LEVEL) * RADIX_BINS;
+    uint32_t *out = hist_of(p, i, 1, LEVEL);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
         if (h[b]) atomicAdd(&out[b], h[b]);
-}
-
-// One CTA per worker.  Finds the bin b with  count(bins > b) < k_rem <= count(bins >= b)
-// and appends it to the key prefix.  After the last level the prefix is the threshold key.
-template <int LEVEL>
-__global__ void __launch_bounds__(BLOCK)
-radix_pick_kernel(SelectState *__restrict__ sel, const uint32_t *__restrict__ hist,
-                  uint32_t want_exact, uint32_t *__restrict__ status)
-{
-    constexpr int BITS = (LEVEL == 2) ? 7 : 12;
-    constexpr int PER = RADIX_BINS / BLOCK;   // 16 bins per thread
-    const uint32_t i = blockIdx.x;
-    if (sel[i].exact != want_exact) return;
-    const uint32_t k_rem = sel[i].k_rem;
-    const uint32_t *h = hist + (static_cast<size_t>(i) * RADIX_LEVELS + LEVEL) * RADIX_BINS;
-    __shared__ uint32_t suf[BLOCK + 1];
-    const int t = threadIdx.x;
-    uint32_t loc[PER], sum = 0;
-#pragma unroll
-    for (int b = 0; b < PER; ++b) {
-        loc[b] = h[t * PER + b];
-        sum += loc[b];
-    }
-    suf[t] = sum;
-    if (t == 0) suf[BLOCK] = 0;
     __syncthreads();
-    for (int o = 1; o < BLOCK; o <<= 1) {      // inclusive suffix sums over threads
-        const uint32_t v = (t + o < BLOCK) ? suf[t + o] : 0u;
-        __syncthreads();
-        suf[t] += v;
-        __syncthreads();
-    }
-    const uint32_t s_here = suf[t], s_above = suf[t + 1];
-    if (t == 0 && s_here < k_rem) latch(status, DECO_ERR_DEVICE_CHECK, 0x100u + LEVEL, i);
-    if (s_here >= k_rem && s_above < k_rem) {
-        uint32_t acc = s_above;
-        int bin = t * PER;
-#pragma unroll
-        for (int b = PER - 1; b >= 0; --b) {
-            if (acc + loc[b] >= k_rem) {
-                bin = t * PER + b;
-                break;
-            }
-            acc += loc[b];
-        }
-        SelectState &s = sel[i];
-        s.n_greater += acc;
-        s.k_rem = k_rem - acc;
-        const uint32_t prefix = (s.prefix << BITS) | static_cast<uint32_t>(bin);
-        s.prefix = prefix;
-        if (LEVEL == 2) {
-            s.threshold = prefix;
-            s.ties_take = k_rem - acc;
-        }
-    }
 }
 
-__global__ void __launch_bounds__(BLOCK)
-tile_count_e_kernel(const float *__restrict__ e, uint64_t e_stride, uint64_t d,
-                    const SelectState *__restrict__ sel, uint32_t *__restrict__ tile_gt,
-                    uint32_t *__restrict__ tile_eq, uint32_t ntiles)
+__device__ __forceinline__ void count_e_tile(const Sel &p, uint32_t i, uint32_t tile,
+                                             uint32_t *s_a /*[WARPS]*/, uint32_t *s_b /*[WARPS]*/)
 {
-    const uint32_t tile = blockIdx.x, i = blockIdx.y;
-    if (!sel[i].exact) return;
-    const uint32_t T = sel[i].threshold;
-    const float *row = e + static_cast<size_t>(i) * e_stride;
+    const uint32_t T = p.sel[i].threshold;
+    const float *row = p.e + static_cast<size_t>(i) * p.e_stride;
     const uint64_t base = static_cast<uint64_t>(tile) * TILE;
     uint32_t gt = 0, eq = 0;
 #pragma unroll
@@ -336,72 +642,45 @@ tile_count_e_kernel(const float *__restrict__ e, uint64_t e_stride, uint64_t d,
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             const uint32_t key = mag_key(xs[c]);
-            const bool in = j + c < d;
+            const bool in = j + c < p.d;
             gt += (in && key > T);
             eq += (in && key == T);
         }
     }
-    __shared__ uint32_t s_gt[WARPS], s_eq[WARPS];
     for (int o = 16; o > 0; o >>= 1) {
         gt += __shfl_down_sync(FULL, gt, o);
         eq += __shfl_down_sync(FULL, eq, o);
     }
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     if (lane == 0) {
-        s_gt[w] = gt;
-        s_eq[w] = eq;
+        s_a[w] = gt;
+        s_b[w] = eq;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         uint32_t a = 0, b = 0;
         for (int ww = 0; ww < WARPS; ++ww) {
-            a += s_gt[ww];
-            b += s_eq[ww];
+            a += s_a[ww];
+            b += s_b[ww];
         }
-        tile_gt[static_cast<size_t>(i) * ntiles + tile] = a;
-        tile_eq[static_cast<size_t>(i) * ntiles + tile] = b;
-    }
-}
-
-// Exclusive scan over SCAN_BLOCK threads; returns the prefix of `v`, total in `total`.
-constexpr int SCAN_BLOCK = 1024;
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *s_w /*[33]*/,
-                                                    uint32_t &total)
-{
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t incl = warp_incl_scan(v);
-    if (lane == 31) s_w[w] = incl;
-    __syncthreads();
-    if (w == 0) {
-        const uint32_t x = s_w[lane];
-        const uint32_t xi = warp_incl_scan(x);
-        s_w[lane] = xi - x;
-        if (lane == 31) s_w[32] = xi;
+        p.tile_gt[static_cast<size_t>(i) * p.ntiles + tile] = a;
+        p.tile_eq[static_cast<size_t>(i) * p.ntiles + tile] = b;
     }
     __syncthreads();
-    const uint32_t out = s_w[w] + incl - v;
-    total = s_w[32];
-    __syncthreads();
-    return out;
 }
 
-// One CTA per worker: ties are granted to tiles in index order until ties_take are used up,
-// then every tile gets its position in the message.
-__global__ void __launch_bounds__(SCAN_BLOCK)
-tile_scan_kernel(const SelectState *__restrict__ sel, const uint32_t *__restrict__ tile_gt,
-                 const uint32_t *__restrict__ tile_eq, uint32_t *__restrict__ tile_take,
-                 uint32_t *__restrict__ tile_start, uint32_t ntiles, uint32_t k,
-                 uint32_t *__restrict__ status)
+// One CTA per worker (any block size): ties are granted to tiles in index order until
+// ties_take are used up, then every tile gets its position in the message.
+__device__ __forceinline__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w /*[33]*/)
 {
-    const uint32_t i = blockIdx.x;
-    __shared__ uint32_t s_w[33];
-    const uint32_t *gt = tile_gt + static_cast<size_t>(i) * ntiles;
-    const uint32_t *eq = tile_eq + static_cast<size_t>(i) * ntiles;
-    uint32_t *take = tile_take + static_cast<size_t>(i) * ntiles;
-    uint32_t *start = tile_start + static_cast<size_t>(i) * (ntiles + 1);
-    const uint32_t ties = sel[i].ties_take;
-    const uint32_t per = (ntiles + SCAN_BLOCK - 1) / SCAN_BLOCK;
-    const uint32_t lo = min(ntiles, threadIdx.x * per), hi = min(ntiles, lo + per);
+    const uint32_t nt = blockDim.x;
+    const uint32_t *gt = p.tile_gt + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t *eq = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
+    uint32_t *take = p.tile_take + static_cast<size_t>(i) * p.ntiles;
+    uint32_t *start = p.tile_start + static_cast<size_t>(i) * (p.ntiles + 1);
+    const uint32_t ties = p.sel[i].ties_take;
+    const uint32_t per = (p.ntiles + nt - 1) / nt;
+    const uint32_t lo = min(p.ntiles, threadIdx.x * per), hi = min(p.ntiles, lo + per);
     uint32_t eq_sum = 0;
     for (uint32_t t = lo; t < hi; ++t) eq_sum += eq[t];
     uint32_t eq_total;
@@ -422,31 +701,25 @@ tile_scan_kernel(const SelectState *__restrict__ sel, const uint32_t *__restrict
         pos += gt[t] + take[t];
     }
     if (threadIdx.x == 0) {
-        start[ntiles] = sel_total;
-        if (sel_total != k) latch(status, DECO_ERR_DEVICE_CHECK, 0x200u, i);
+        start[p.ntiles] = sel_total;
+        if (sel_total != p.k) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x200u, i);
     }
+    __syncthreads();
 }
 
-__global__ void __launch_bounds__(BLOCK)
-emit_e_kernel(float *__restrict__ e, uint64_t e_stride, uint64_t d,
-              const SelectState *__restrict__ sel, const uint32_t *__restrict__ tile_eq,
-              const uint32_t *__restrict__ tile_take, const uint32_t *__restrict__ tile_start,
-              deco_pair *__restrict__ msg, uint64_t k_cap, uint32_t k, uint32_t ntiles,
-              uint32_t *__restrict__ status)
+__device__ __forceinline__ void emit_e_tile(const Sel &p, uint32_t i, uint32_t tile,
+                                            uint32_t *s_w /*[WARPS]*/)
 {
     constexpr int V = 4, U = WARP_ELEMS / (32 * V);
-    const uint32_t tile = blockIdx.x, i = blockIdx.y;
-    if (!sel[i].exact) return;
-    const uint32_t start = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-    const uint32_t count = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1] - start;
+    const uint32_t start = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile];
+    const uint32_t count = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile + 1] - start;
     if (count == 0) return;
-    const uint32_t T = sel[i].threshold;
-    const uint32_t take = tile_take[static_cast<size_t>(i) * ntiles + tile];
-    const uint32_t n_eq = tile_eq[static_cast<size_t>(i) * ntiles + tile];
+    const uint32_t T = p.sel[i].threshold;
+    const uint32_t take = p.tile_take[static_cast<size_t>(i) * p.ntiles + tile];
+    const uint32_t n_eq = p.tile_eq[static_cast<size_t>(i) * p.ntiles + tile];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    float *erow = e + static_cast<size_t>(i) * e_stride;
+    float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     const uint64_t wbase = static_cast<uint64_t>(tile) * TILE + static_cast<uint64_t>(w) * WARP_ELEMS;
-    __shared__ uint32_t s_w[WARPS];
 
     float x[U][V];
     uint32_t gt[U], eq[U];
@@ -459,7 +732,7 @@ emit_e_kernel(float *__restrict__ e, uint64_t e_stride, uint64_t d,
 #pragma unroll
         for (int c = 0; c < V; ++c) {
             const uint32_t key = mag_key(x[u][c]);
-            if (j + c < d) {
+            if (j + c < p.d) {
                 gt[u] |= (key > T) ? (1u << c) : 0u;
                 eq[u] |= (key == T) ? (1u << c) : 0u;
             }
@@ -490,46 +763,158 @@ emit_e_kernel(float *__restrict__ e, uint64_t e_stride, uint64_t d,
     for (int u = 0; u < U; ++u) cnt[u] = __popc(m[u]);
     ordered_prefix<U>(cnt, pos, s_w, total);
     if (total != count) {
-        if (threadIdx.x == 0) latch(status, DECO_ERR_DEVICE_CHECK, 0x300u, tile);
+        if (threadIdx.x == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x300u, tile);
         return;
     }
-    deco_pair *out = msg + static_cast<size_t>(i) * k_cap;
+    deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         if (!m[u]) continue;
         const uint64_t j = wbase + u * 128 + lane * 4;
-        uint32_t p = start + pos[u];
+        uint32_t q = start + pos[u];
 #pragma unroll
         for (int c = 0; c < V; ++c)
             if (m[u] & (1u << c)) {
-                if (p < k) {
+                if (q < p.k) {
                     deco_pair pr;
                     pr.idx = static_cast<uint32_t>(j + c);
                     pr.val = x[u][c];
-                    out[p] = pr;
+                    out[q] = pr;
                 }
-                ++p;
+                ++q;
                 x[u][c] = 0.0f;
             }
         *reinterpret_cast<float4 *>(erow + j) = make_float4(x[u][0], x[u][1], x[u][2], x[u][3]);
     }
 }
 
-// Per step: clear the histograms and (re)arm the per-worker selection records.
-__global__ void begin_step_kernel(SelectState *sel, uint32_t n, uint32_t k, uint32_t exact_all)
+// ---- dedicated kernels of the multi-pass route (every worker takes it) --------------------
+template <int LEVEL>
+__global__ void __launch_bounds__(BLOCK) radix_hist_e_kernel(Sel p)
 {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    SelectState &s = sel[i];
-    s.prefix = 0;
-    s.k_rem = k;
-    s.n_greater = 0;
-    s.threshold = 0;
-    s.ties_take = 0;
-    s.exact = exact_all;
-    s.spec_key = SPEC_DISABLED;
-    s.n_staged = 0;
-    if (exact_all) s.exact_total += 1;
+    const uint32_t i = blockIdx.y;
+    if (!p.sel[i].exact) return;
+    __shared__ uint32_t h[RADIX_BINS];
+    hist_e_body<LEVEL>(p, i, blockIdx.x, gridDim.x, h);
+}
+
+template <int LEVEL>
+__global__ void __launch_bounds__(BLOCK) radix_pick_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.x;
+    if (!p.sel[i].exact) return;
+    __shared__ uint32_t suf[BLOCK + 1];
+    pick_body<LEVEL>(p.sel[i], hist_of(p, i, 1, LEVEL), suf, p.status, i);
+}
+
+__global__ void __launch_bounds__(BLOCK) tile_count_e_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.y;
+    if (!p.sel[i].exact) return;
+    __shared__ uint32_t s_a[WARPS], s_b[WARPS];
+    count_e_tile(p, i, blockIdx.x, s_a, s_b);
+}
+
+// exact_only: 1 = scan the workers on the multi-pass route, 0 = those on the streaming route
+constexpr int SCAN_BLOCK = 1024;
+__global__ void __launch_bounds__(SCAN_BLOCK) tile_scan_kernel(Sel p, uint32_t exact_only)
+{
+    const uint32_t i = blockIdx.x;
+    if ((p.sel[i].exact != 0) != (exact_only != 0)) return;
+    __shared__ uint32_t s_w[33];
+    scan_tiles_body(p, i, s_w);
+}
+
+__global__ void __launch_bounds__(BLOCK) emit_e_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.y;
+    if (!p.sel[i].exact) return;
+    __shared__ uint32_t s_w[WARPS];
+    emit_e_tile(p, i, blockIdx.x, s_w);
+}
+
+// ---- fallback of the streaming route: the whole multi-pass route in one cooperative launch.
+// Leaves at once unless some worker's staged set was rejected.  All CTAs take every
+// grid-wide barrier: the decision to leave is the same for the whole grid.
+__global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
+{
+    if (__ldcg(&p.status[3]) == 0) return;
+    cg::grid_group grid = cg::this_grid();
+    __shared__ uint32_t h[RADIX_BINS];
+    __shared__ uint32_t suf[BLOCK + 1];
+    __shared__ uint32_t s_a[33], s_b[WARPS];
+    const uint32_t cta = blockIdx.x, ncta = gridDim.x;
+    for (int level = 0; level < RADIX_LEVELS; ++level) {
+        for (uint32_t i = 0; i < p.n; ++i) {
+            if (!p.sel[i].exact) continue;
+            if (level == 0) hist_e_body<0>(p, i, cta, ncta, h);
+            else if (level == 1) hist_e_body<1>(p, i, cta, ncta, h);
+            else hist_e_body<2>(p, i, cta, ncta, h);
+        }
+        __threadfence();
+        grid.sync();
+        for (uint32_t i = cta; i < p.n; i += ncta) {
+            if (!p.sel[i].exact) continue;
+            if (level == 0) pick_body<0>(p.sel[i], hist_of(p, i, 1, 0), suf, p.status, i);
+            else if (level == 1) pick_body<1>(p.sel[i], hist_of(p, i, 1, 1), suf, p.status, i);
+            else pick_body<2>(p.sel[i], hist_of(p, i, 1, 2), suf, p.status, i);
+        }
+        __threadfence();
+        grid.sync();
+    }
+    for (uint32_t i = 0; i < p.n; ++i) {
+        if (!p.sel[i].exact) continue;
+        for (uint32_t tile = cta; tile < p.ntiles; tile += ncta) count_e_tile(p, i, tile, s_a, s_b);
+    }
+    __threadfence();
+    grid.sync();
+    for (uint32_t i = cta; i < p.n; i += ncta) {
+        if (!p.sel[i].exact) continue;
+        scan_tiles_body(p, i, s_a);
+    }
+    __threadfence();
+    grid.sync();
+    for (uint32_t i = 0; i < p.n; ++i) {
+        if (!p.sel[i].exact) continue;
+        for (uint32_t tile = cta; tile < p.ntiles; tile += ncta) {
+            emit_e_tile(p, i, tile, s_b);
+            __syncthreads();
+        }
+    }
+}
+
+Sel make_sel(const deco_ctx *c)
+{
+    Sel p;
+    p.e = c->e;
+    p.e_stride = c->e_stride;
+    p.d = c->d;
+    p.n = c->n;
+    p.ntiles = c->ntiles;
+    p.k = static_cast<uint32_t>(c->k);
+    p.sel = c->sel;
+    p.hist = c->hist;
+    p.done = c->done;
+    p.tile_gt = c->tile_gt;
+    p.tile_eq = c->tile_eq;
+    p.tile_take = c->tile_take;
+    p.tile_start = c->tile_start;
+    p.tile_off = c->tile_off;
+    p.tile_cnt = c->tile_cnt;
+    p.msg = c->msg;
+    p.k_cap = c->k_cap;
+    p.stage = c->stage;
+    p.stage_cap = c->stage_cap;
+    p.status = c->dev_status;
+    return p;
+}
+
+uint32_t part_blocks(const deco_ctx *c, uint64_t items_per_worker, uint32_t items_per_cta)
+{
+    // enough CTAs per worker to fill the machine, never more than there is work for
+    const uint64_t want = (items_per_worker + items_per_cta - 1) / items_per_cta;
+    const uint64_t cap = (148ull * 8 + c->n - 1) / c->n;
+    return static_cast<uint32_t>(want < 1 ? 1 : (want < cap ? want : cap));
 }
 
 }  // namespace
@@ -537,15 +922,17 @@ __global__ void begin_step_kernel(SelectState *sel, uint32_t n, uint32_t k, uint
 // ------------------------------------------------------------------------------------------
 // Launchers
 // ------------------------------------------------------------------------------------------
-cudaError_t launch_begin_step(deco_ctx *c, cudaStream_t s)
+bool streaming_route(const deco_ctx *c) { return c->select_mode == DECO_SELECT_AUTO; }
+
+cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s)
 {
-    cudaError_t err = cudaMemsetAsync(
-        c->hist, 0, sizeof(uint32_t) * c->n * RADIX_LEVELS * RADIX_BINS, s);
-    if (err != cudaSuccess) return err;
-    const uint32_t exact_all = 1;   // speculative path not wired yet
-    begin_step_kernel<<<(c->n + 127) / 128, 128, 0, s>>>(c->sel, c->n,
-                                                          static_cast<uint32_t>(c->k), exact_all);
-    c->launches += 2;
+    const float alpha = c->lr_at_server ? 1.0f : c->lr;
+    const uint32_t exact_all = streaming_route(c) ? 0u : 1u;
+    if (c->grad_dtype == DECO_BF16)
+        begin_step_kernel<1><<<c->n, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
+    else
+        begin_step_kernel<0><<<c->n, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
+    c->launches += 1;
     return cudaGetLastError();
 }
 
@@ -553,9 +940,14 @@ template <int GT, bool ALIGNED>
 static void launch_acc(deco_ctx *c, const void *grads, float alpha, cudaStream_t s)
 {
     dim3 grid(c->ntiles, c->n);
-    ef_accumulate_kernel<GT, ALIGNED, false><<<grid, BLOCK, 0, s>>>(
-        c->e, c->e_stride, grads, c->d, alpha, c->sel, c->stage, c->stage_cap, c->tile_off,
-        c->tile_cnt, c->ntiles);
+    if (streaming_route(c))
+        ef_accumulate_kernel<GT, ALIGNED, true><<<grid, BLOCK, 0, s>>>(
+            c->e, c->e_stride, grads, c->d, alpha, c->sel, c->stage, c->stage_cap, c->tile_off,
+            c->tile_cnt, c->ntiles);
+    else
+        ef_accumulate_kernel<GT, ALIGNED, false><<<grid, BLOCK, 0, s>>>(
+            c->e, c->e_stride, grads, c->d, alpha, c->sel, c->stage, c->stage_cap, c->tile_off,
+            c->tile_cnt, c->ntiles);
 }
 
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s)
@@ -574,35 +966,55 @@ cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s)
     return cudaGetLastError();
 }
 
-static uint32_t hist_blocks(const deco_ctx *c)
+cudaError_t query_fallback_grid(deco_ctx *c)
 {
-    // enough CTAs to fill the machine, never more than there are 128-bit words per CTA round
-    const uint64_t nvec = (c->d + 3) / 4;
-    const uint64_t want = (nvec + BLOCK * 8 - 1) / (BLOCK * 8);
-    const uint64_t cap = (148ull * 8 + c->n - 1) / c->n;
-    return static_cast<uint32_t>(want < 1 ? 1 : (want < cap ? want : cap));
+    int per_sm = 0, sms = 0;
+    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, exact_fallback_kernel,
+                                                                    BLOCK, 0);
+    if (err != cudaSuccess) return err;
+    err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+    if (per_sm > 4) per_sm = 4;
+    c->fallback_grid = static_cast<uint32_t>(per_sm * sms);
+    return cudaSuccess;
 }
 
-cudaError_t launch_exact_selection(deco_ctx *c, cudaStream_t s)
+cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
 {
-    dim3 hgrid(hist_blocks(c), c->n);
+    Sel p = make_sel(c);
     dim3 tgrid(c->ntiles, c->n);
-    const uint32_t k = static_cast<uint32_t>(c->k);
-    radix_hist_e_kernel<0><<<hgrid, BLOCK, 0, s>>>(c->e, c->e_stride, c->d, c->sel, c->hist);
-    radix_pick_kernel<0><<<c->n, BLOCK, 0, s>>>(c->sel, c->hist, 1u, c->dev_status);
-    radix_hist_e_kernel<1><<<hgrid, BLOCK, 0, s>>>(c->e, c->e_stride, c->d, c->sel, c->hist);
-    radix_pick_kernel<1><<<c->n, BLOCK, 0, s>>>(c->sel, c->hist, 1u, c->dev_status);
-    radix_hist_e_kernel<2><<<hgrid, BLOCK, 0, s>>>(c->e, c->e_stride, c->d, c->sel, c->hist);
-    radix_pick_kernel<2><<<c->n, BLOCK, 0, s>>>(c->sel, c->hist, 1u, c->dev_status);
-    tile_count_e_kernel<<<tgrid, BLOCK, 0, s>>>(c->e, c->e_stride, c->d, c->sel, c->tile_gt,
-                                                c->tile_eq, c->ntiles);
-    tile_scan_kernel<<<c->n, SCAN_BLOCK, 0, s>>>(c->sel, c->tile_gt, c->tile_eq, c->tile_take,
-                                                 c->tile_start, c->ntiles, k, c->dev_status);
-    emit_e_kernel<<<tgrid, BLOCK, 0, s>>>(c->e, c->e_stride, c->d, c->sel, c->tile_eq,
-                                          c->tile_take, c->tile_start, c->msg, c->k_cap, k,
-                                          c->ntiles, c->dev_status);
-    c->launches += 9;
-    return cudaGetLastError();
+    if (!streaming_route(c)) {
+        dim3 hgrid(part_blocks(c, (c->d + 3) / 4, BLOCK * 8), c->n);
+        radix_hist_e_kernel<0><<<hgrid, BLOCK, 0, s>>>(p);
+        radix_pick_kernel<0><<<c->n, BLOCK, 0, s>>>(p);
+        radix_hist_e_kernel<1><<<hgrid, BLOCK, 0, s>>>(p);
+        radix_pick_kernel<1><<<c->n, BLOCK, 0, s>>>(p);
+        radix_hist_e_kernel<2><<<hgrid, BLOCK, 0, s>>>(p);
+        radix_pick_kernel<2><<<c->n, BLOCK, 0, s>>>(p);
+        tile_count_e_kernel<<<tgrid, BLOCK, 0, s>>>(p);
+        tile_scan_kernel<<<c->n, SCAN_BLOCK, 0, s>>>(p, 1u);
+        emit_e_kernel<<<tgrid, BLOCK, 0, s>>>(p);
+        c->launches += 9;
+        return cudaGetLastError();
+    }
+    // staged pairs per worker are a few times k: size the histogram grid for that
+    dim3 sgrid(part_blocks(c, 2 * c->k + 65536, BLOCK * 8), c->n);
+    dim3 wgrid((c->ntiles + WARPS - 1) / WARPS, c->n);
+    stage_hist_pick_kernel<0><<<sgrid, BLOCK, 0, s>>>(p);
+    stage_hist_pick_kernel<1><<<sgrid, BLOCK, 0, s>>>(p);
+    stage_hist_pick_kernel<2><<<sgrid, BLOCK, 0, s>>>(p);
+    tile_count_stage_kernel<<<wgrid, BLOCK, 0, s>>>(p);
+    tile_scan_kernel<<<c->n, SCAN_BLOCK, 0, s>>>(p, 0u);
+    emit_stage_kernel<<<wgrid, BLOCK, 0, s>>>(p);
+    c->launches += 6;
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    void *args[] = {&p};
+    err = cudaLaunchCooperativeKernel(reinterpret_cast<void *>(exact_fallback_kernel),
+                                      dim3(c->fallback_grid), dim3(BLOCK), args, 0, s);
+    c->launches += 1;
+    return err;
 }
 
 }  // namespace deco

@@ -73,7 +73,9 @@ struct deco_ctx {
     deco_pair *msg = nullptr;
     deco_pair *slots = nullptr;         // [ring][n * k_cap]
     deco_pair *stage = nullptr;         // [n][stage_cap]
-    uint32_t *hist = nullptr;           // [n][RADIX_LEVELS][RADIX_BINS]
+    uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
+    uint32_t *done = nullptr;           // [n][RADIX_LEVELS] CTA arrival counters
+    uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
     deco::SelectState *sel = nullptr;   // [n]
     uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
     uint32_t *tile_eq = nullptr;        // [n][ntiles]  entries equal to it per tile
@@ -81,8 +83,7 @@ struct deco_ctx {
     uint32_t *tile_start = nullptr;     // [n][ntiles + 1] message position of each tile
     uint32_t *tile_off = nullptr;       // [n][ntiles]  staging offset of each tile's candidates
     uint32_t *tile_cnt = nullptr;       // [n][ntiles]  staged candidates per tile
-    uint32_t *sample_keys = nullptr;    // [n][sample_cap]
-    uint32_t *dev_status = nullptr;     // [4]: status, detail words
+    uint32_t *dev_status = nullptr;     // [4]: status, two detail words, fallback flag
     void *grads_staging = nullptr;      // device copy of host gradients (deco_step_host)
     uint64_t device_bytes = 0;
     // host bookkeeping
@@ -91,14 +92,19 @@ struct deco_ctx {
     std::vector<deco::Slot> slot_info;
     uint64_t launches = 0;
     uint64_t k_of_msg = 0;              // k used by the last compress
+    // optional event timing: 8 events per recorded iteration
+    bool timing = false;
+    std::vector<cudaEvent_t> events;
+    size_t timed_iters = 0;
 };
 
 namespace deco {
 
 // --- kernel launchers (deco_compress.cu) -------------------------------------------------
-cudaError_t launch_begin_step(deco_ctx *c, cudaStream_t s);
+cudaError_t query_fallback_grid(deco_ctx *c);
+cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s);
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s);
-cudaError_t launch_exact_selection(deco_ctx *c, cudaStream_t s);
+cudaError_t launch_selection(deco_ctx *c, cudaStream_t s);
 // --- kernel launchers (deco_server.cu) ---------------------------------------------------
 cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s);
 cudaError_t launch_apply(deco_ctx *c, const deco_pair *slot, uint64_t positions, float neg_scale,

@@ -98,6 +98,29 @@ def test_degradation_to_dsgd_and_stepsize_at_server(mode):
                lr_at_server=True, select_mode=mode)
 
 
+def test_streaming_route_is_taken_and_falls_back_on_degenerate_inputs():
+    """With the default selection mode, ordinary inputs go through the sampled single-pass
+    route; inputs whose tie class is far larger than the staging area (all equal, all zero,
+    two-valued) must be handed to the multi-pass route inside the same call."""
+    d, n = 300_000, 3
+    run_parity(d, n, 0.01, 1, 0.1, lambda t: _values("normal", n, d, t, torch.float32),
+               steps=4, expect_exact=False)
+    for kind in ("all_equal", "all_zero"):
+        run_parity(d, n, 0.01, 1, 0.1, lambda t: _values(kind, n, d, t, torch.float32),
+                   steps=3, expect_exact=True)
+    # two-valued: the tie class overflows the staging area at step 0 only
+    st = run_parity(d, n, 0.01, 1, 0.1, lambda t: _values("two_valued", n, d, t, torch.float32),
+                    steps=3)
+    assert st["exact_pass_workers"] >= n
+    # mixed: worker 0 degenerate, the others ordinary -> per-worker decision
+    def mixed(t):
+        g = _values("normal", n, d, t, torch.float32)
+        g[0] = 0.5
+        return g
+    ctx_stats = run_parity(d, n, 0.01, 1, 0.1, mixed, steps=3)
+    assert 0 < ctx_stats["exact_pass_workers"] < 3 * n
+
+
 def test_call_order_and_capacity_errors():
     d, n = 10_000, 2
     ctx = B.deco_init(d, n, 0.01, 1, 0.1, tau_max=2, delta_max=0.05)
