@@ -245,6 +245,30 @@ deco_status deco_get_kernel_timing(deco_ctx *ctx, void *stream, double *ms_sum /
 /* Number of kernels and memset/memcpy nodes the library has enqueued so far. */
 uint64_t deco_launch_count(const deco_ctx *ctx);
 
+/*
+ * Top-k compression of one vector without any allocation.  (The paper has no counterpart:
+ * this entry point exists for callers that cannot allocate device memory at the moment they
+ * need C_delta — code running while a stream is being captured, plugins inside a host
+ * program that owns the memory pool, loops that cannot afford cudaMalloc's implicit
+ * synchronisation.)  Same selection rule as the context-based path: the k largest |a[j]|,
+ * equal magnitudes by increasing index, written as k pairs sorted by index.
+ *   a        DEVICE, [d] fp32, read-only, any alignment
+ *   msg_out  DEVICE, [k] pairs, 8-byte aligned
+ *   1 <= k <= d <= DECO_STATIC_MAX_D; longer vectors return DECO_ERR_CAPACITY (and print
+ *   the limit to stderr) — use a context for those.
+ * Works on the CURRENT device; a and msg_out must live there.  Calls no cudaMalloc, cudaFree
+ * or other allocating routine: the working memory (histograms, selection record, per-tile
+ * counters, 82 KB) is a fixed device array inside the library that every GPU loading the
+ * library holds until the process exits.  The first call on each device looks up that
+ * array's device address (cudaGetSymbolAddress) — make that first call before any stream
+ * capture begins.  All calls share the array and it keeps the previous call's contents; each
+ * call clears what it needs first, so calls in one stream are safe, but two calls that
+ * overlap on the GPU (different streams, different host threads) race on it.
+ */
+#define DECO_STATIC_MAX_D 16777216ull
+deco_status deco_topk_compress_static(const float *a, uint64_t d, uint64_t k,
+                                      deco_pair *msg_out, void *stream);
+
 const char *deco_status_string(deco_status s);
 
 #ifdef __cplusplus

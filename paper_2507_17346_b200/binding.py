@@ -88,6 +88,7 @@ SIGNATURES = {
     "deco_set_kernel_timing": (_i32, [_vp, _i32]),
     "deco_get_kernel_timing": (_i32, [_vp, _vp, _P(_f64), _P(_u64)]),
     "deco_launch_count": (_u64, [_vp]),
+    "deco_topk_compress_static": (_i32, [_vp, _u64, _u64, _vp, _vp]),
     "deco_status_string": (ctypes.c_char_p, [_i32]),
 }
 
@@ -265,6 +266,17 @@ def deco_get_kernel_timing(ctx, stream=None):
 
 def deco_launch_count(ctx):
     return load().deco_launch_count(ctx)
+
+
+DECO_STATIC_MAX_D = 16777216
+
+
+def deco_topk_compress_static(a, d, k, msg_out, stream=None):
+    """Top-k of one fp32 CUDA tensor `a` into `msg_out` ([k, 2] int32 view of the pairs), with
+    no allocation inside the library (fixed device scratch; d <= DECO_STATIC_MAX_D).  For
+    callers that cannot allocate: during stream capture, under a foreign memory pool."""
+    _check(load().deco_topk_compress_static(_ptr(a), d, k, _ptr(msg_out), _stream(stream)),
+           "deco_topk_compress_static")
 
 
 # ------------------------------------------------------------- device views (plumbing)
