@@ -111,6 +111,21 @@ class ClockSampler:
                 "samples_in_timed_region": len(inside)}
 
 
+def max_over_ranks(ms, dist, device):
+    """Slowest rank's time: every rank ends up with the same number (MAX all-reduce)."""
+    if dist is None:
+        return float(ms)
+    import torch
+    tt = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_value(bytes_per_replica_step, world, ms_per_step):
+    """Gradient GB/s of the whole job: every replica processes its own batch per step."""
+    return world * bytes_per_replica_step / (ms_per_step * 1e-3) / 1e9
+
+
 def workload_for(args):
     from paper_2507_17346_b200 import workloads as W
     wl = W.make_workload(args.workload)
@@ -257,13 +272,9 @@ def run_ours(args):
     B.deco_set_kernel_timing(ctx, False)
     stats = B.deco_get_stats(ctx, stream)
 
-    ms_max = ms_total
-    if dist is not None:
-        tt = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_max = float(tt.item())
+    ms_max = max_over_ranks(ms_total, dist, "cuda")
     ms_per_step = ms_max / steps
-    value = world * gbytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_value(gbytes, world, ms_per_step)
 
     # end to end through the host-buffer entry point: H2D gradients, step, D2H messages
     e2e = None
@@ -283,12 +294,8 @@ def run_ours(args):
             B.deco_step_host(ctx, host_g[t % 2], host_msg, None, stream)
         e1.record(stream)
         torch.cuda.synchronize()
-        e_ms = e0.elapsed_time(e1)
-        if dist is not None:
-            tt = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e_ms = float(tt.item())
-        e2e = {"value": world * gbytes / (e_ms / e_steps * 1e-3) / 1e9, "unit": UNIT,
+        e_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
+        e2e = {"value": whole_job_value(gbytes, world, e_ms / e_steps), "unit": UNIT,
                "h2d_bytes_per_step": gbytes, "d2h_bytes_per_step": wl.n * k * 8,
                "steps": e_steps, "ms_per_step": e_ms / e_steps}
     B.deco_destroy(ctx)

@@ -121,6 +121,30 @@ def test_streaming_route_is_taken_and_falls_back_on_degenerate_inputs():
     assert 0 < ctx_stats["exact_pass_workers"] < 3 * n
 
 
+def test_adaptive_policy_run():
+    """DeCo-SGD (Algorithm 2): every E iterations the host re-selects (tau, delta) with DeCo
+    (Algorithm 3) from a synthetic bandwidth/latency trace; the library's decision must equal
+    the oracle's, and the iterations stay in parity across the changes."""
+    from oracle import deco_policy as P
+    wl = W.make_workload("sweep_100m", 0.004)
+    d, n, steps, E = wl.d, wl.n, 60, 10
+    V_g, T_comp, tau_max, delta_max = 32.0 * 1e8, 0.05, 16, 0.2
+    lat, bw = W.network_trace(wl.seed, steps)
+    plan = {}
+    for t in range(E, steps, E):                      # decided after iteration t-1
+        a_bar, b = float(np.mean(bw[t - E:t])), float(lat[t - 1])
+        tau, delta = B.deco_policy_select(V_g, a_bar, b, T_comp, tau_max, False)
+        otau, odelta = P.deco_select(V_g, a_bar, b, T_comp)
+        if otau > tau_max:
+            otau, odelta = tau_max, P.delta_star(tau_max, V_g, a_bar, b, T_comp)
+        assert (tau, delta) == (otau, pytest.approx(odelta, rel=1e-12))
+        delta = min(delta_max, max(delta, 1.0 / d))
+        plan[t] = (delta, tau)
+    assert len({v for v in plan.values()}) >= 3          # the trace does move the decision
+    run_parity(d, n, 0.01, 2, 0.1, lambda t: W.gradients(wl, t, "cuda"), steps=steps,
+               policy_plan=plan, tau_max=tau_max, delta_max=delta_max, check_every=3)
+
+
 def test_call_order_and_capacity_errors():
     d, n = 10_000, 2
     ctx = B.deco_init(d, n, 0.01, 1, 0.1, tau_max=2, delta_max=0.05)

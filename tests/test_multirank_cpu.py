@@ -1,0 +1,54 @@
+"""The N > 1 logic of bench.py on CPU: two gloo ranks agree on the max-over-ranks time, the
+whole-job value counts every replica, and the reference arm prints one line from rank 0."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _rank_main(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    sys.path.insert(0, ROOT)
+    import bench
+    local_ms = 10.0 + 5.0 * rank                       # rank 1 is the slow one
+    dist.barrier()
+    slowest = bench.max_over_ranks(local_ms, dist, "cpu")
+    value = bench.whole_job_value(1e9, world, slowest / 5)
+    with open(out + ".%d" % rank, "w") as fh:
+        json.dump({"slowest": slowest, "value": value}, fh)
+    dist.destroy_process_group()
+
+
+def test_max_over_ranks_and_whole_job_value(tmp_path):
+    out = str(tmp_path / "r")
+    mp.spawn(_rank_main, args=(2, 29517, out), nprocs=2, join=True)
+    got = [json.load(open(out + ".%d" % r)) for r in range(2)]
+    assert got[0] == got[1]
+    assert got[0]["slowest"] == 15.0
+    # 2 replicas x 1 GB per step, 3 ms per step -> 666.7 GB/s
+    assert got[0]["value"] == pytest.approx(2 * 1e9 / 3e-3 / 1e9)
+
+
+def test_reference_arm_prints_one_line_from_rank_zero():
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+           "--master-addr", "127.0.0.1", "--master-port", "29519",
+           os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+           "--workload", "flat_1m", "--steps", "1", "--warmup", "0"]
+    res = subprocess.run(cmd, capture_output=True, text=True, cwd=ROOT, env=env, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
+    assert line["e2e"]["h2d_bytes_per_step"] == 0
