@@ -53,6 +53,9 @@ void free_all(deco_ctx *c)
     cudaFree(c->tile_start);
     cudaFree(c->tile_off);
     cudaFree(c->tile_cnt);
+    cudaFree(c->tile_rej);
+    cudaFree(c->boundary);
+    cudaFree(c->sample_keys);
     cudaFree(c->done);
     cudaFree(c->dev_status);
     cudaFree(c->grads_staging);
@@ -67,6 +70,8 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
         err = cudaMemsetAsync(c->params, 0, sizeof(float) * c->d, s);
     if (err == cudaSuccess) err = cudaMemsetAsync(c->sel, 0, sizeof(SelectState) * c->n, s);
     if (err == cudaSuccess) err = cudaMemsetAsync(c->dev_status, 0, sizeof(uint32_t) * 4, s);
+    if (err == cudaSuccess)
+        err = cudaMemsetAsync(c->done, 0, sizeof(uint32_t) * c->n * (RADIX_LEVELS + 1), s);
     if (err == cudaSuccess)
         err = cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n * (c->ntiles + 1), s);
     c->launches += 5;
@@ -180,7 +185,8 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * n * c->k_cap));
     need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
     need(dev_alloc(c, &c->hist, static_cast<uint64_t>(n) * 2 * RADIX_LEVELS * RADIX_BINS));
-    need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * RADIX_LEVELS));
+    need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * (RADIX_LEVELS + 1)));
+    need(dev_alloc(c, &c->sample_keys, static_cast<uint64_t>(n) * SAMPLE_KEYS));
     need(dev_alloc(c, &c->sel, n));
     need(dev_alloc(c, &c->tile_gt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_eq, static_cast<uint64_t>(n) * c->ntiles));
@@ -188,6 +194,8 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->tile_start, static_cast<uint64_t>(n) * (c->ntiles + 1)));
     need(dev_alloc(c, &c->tile_off, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_cnt, static_cast<uint64_t>(n) * c->ntiles));
+    need(dev_alloc(c, &c->tile_rej, static_cast<uint64_t>(n) * c->ntiles));
+    need(dev_alloc(c, &c->boundary, static_cast<uint64_t>(n) * BOUNDARY_CAP));
     need(dev_alloc(c, &c->dev_status, 4));
     if (st == DECO_OK && query_fallback_grid(c) != cudaSuccess) st = DECO_ERR_CUDA;
     if (st == DECO_OK) st = zero_state(c, nullptr);

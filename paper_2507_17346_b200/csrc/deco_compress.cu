@@ -6,11 +6,12 @@
 // Streaming route (DECO_SELECT_AUTO): a small sample of a fixes, per worker, a lower bound
 // `spec_key` that is below the k-th largest magnitude with overwhelming probability.  One pass
 // reads e and g, writes a into e and stages every entry whose key reaches the bound (a few
-// times k pairs, each tile's entries in index order).  The exact threshold is then found by
-// a three-level radix selection over the staged pairs only, and the message is an ordered
-// filter of them.  The count of staged pairs proves the bound was valid (>= k of them); if it
-// was not, or the staging area overflowed, that worker takes the second route in the same
-// call.
+// times k pairs, each tile's entries in index order); staged entries are written to e as +0
+// on the guess that they will be selected.  The exact threshold is then found by a two-level
+// radix selection over the staged pairs only (on key - spec_key), the message is an ordered
+// filter of them, and the few staged entries that are not selected get their value back.
+// The count of staged pairs proves the bound was valid (>= k of them); if it was not, or the
+// staging area overflowed, that worker takes the second route in the same call.
 //
 // Multi-pass route (DECO_SELECT_EXACT_PASSES, and the fallback of the first): three radix
 // histogram passes over e fix the threshold key, one pass counts per tile, one pass emits.
@@ -42,8 +43,10 @@ struct Sel {
     uint32_t k;
     SelectState *sel;
     uint32_t *hist;          // [n][2][RADIX_LEVELS][RADIX_BINS]: 0 = staged route, 1 = multi-pass
-    uint32_t *done;          // [n][RADIX_LEVELS] CTA arrival counters of the staged route
-    uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt;
+    uint32_t *done;          // [n][RADIX_LEVELS + 1] CTA arrival counters
+    uint32_t *sample_keys;   // [n][4 * SAMPLE_CHUNKS] keys of the sample
+    uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt, *tile_rej;
+    deco_pair *boundary;     // [n][BOUNDARY_CAP]
     deco_pair *msg;
     uint64_t k_cap;
     deco_pair *stage;
@@ -147,7 +150,7 @@ __device__ __forceinline__ float load_g(const void *grow, uint64_t j)
 }
 
 // ------------------------------------------------------------------------------------------
-// Radix helpers shared by both routes: 31-bit key = 12 + 12 + 7 bits.
+// Radix helpers.  Multi-pass route: 31-bit key = 12 + 12 + 7 bits, most significant first.
 // ------------------------------------------------------------------------------------------
 template <int LEVEL>
 __device__ __forceinline__ void radix_bin(uint32_t key, uint32_t prefix, uint32_t *h)
@@ -161,120 +164,165 @@ __device__ __forceinline__ void radix_bin(uint32_t key, uint32_t prefix, uint32_
     }
 }
 
-// One CTA (BLOCK threads).  Finds the bin b with  count(bins > b) < k_rem <= count(bins >= b)
-// in histogram h and appends it to the key prefix of s.  After the last level the prefix is
-// the threshold key.  suf: BLOCK + 1 words of shared memory.
-template <int LEVEL>
-__device__ __forceinline__ void pick_body(SelectState &s, const uint32_t *h, uint32_t *suf,
-                                          uint32_t *status, uint32_t i)
+// One CTA of BLOCK threads: the bin b with  count(bins > b) < want <= count(bins >= b)  of
+// histogram h (RADIX_BINS bins, read through L2) and the count above it.  s_scan: 33 words,
+// s_out: 2 words.  All threads get the result; bin 0xFFFFFFFF means the histogram holds fewer
+// than `want` entries.
+__device__ __forceinline__ void pick_bin(const uint32_t *h, uint32_t want, uint32_t *s_scan,
+                                         uint32_t *s_out, uint32_t &bin_out, uint32_t &above_out)
 {
-    constexpr int BITS = (LEVEL == 2) ? 7 : 12;
     constexpr int PER = RADIX_BINS / BLOCK;   // 16 bins per thread
-    const uint32_t k_rem = s.k_rem;
-    const int t = threadIdx.x;
+    // thread t owns the bins of the mirrored position, so the exclusive prefix over threads
+    // is the number of entries in higher bins
+    const int rt = BLOCK - 1 - static_cast<int>(threadIdx.x);
     uint32_t loc[PER], sum = 0;
 #pragma unroll
     for (int b = 0; b < PER; ++b) {
-        loc[b] = __ldcg(&h[t * PER + b]);
+        loc[b] = __ldcg(&h[rt * PER + b]);
         sum += loc[b];
     }
-    suf[t] = sum;
-    if (t == 0) suf[BLOCK] = 0;
-    __syncthreads();
-    for (int o = 1; o < BLOCK; o <<= 1) {      // inclusive suffix sums over threads
-        const uint32_t v = (t + o < BLOCK) ? suf[t + o] : 0u;
-        __syncthreads();
-        suf[t] += v;
-        __syncthreads();
+    if (threadIdx.x == 0) {
+        s_out[0] = 0xFFFFFFFFu;
+        s_out[1] = 0;
     }
-    const uint32_t s_here = suf[t], s_above = suf[t + 1];
-    if (t == 0 && s_here < k_rem) latch(status, DECO_ERR_DEVICE_CHECK, 0x100u + LEVEL, i);
-    if (s_here >= k_rem && s_above < k_rem) {
+    uint32_t total;
+    const uint32_t s_above = block_excl_scan(sum, s_scan, total);
+    if (s_above < want && s_above + sum >= want) {
         uint32_t acc = s_above;
-        int bin = t * PER;
+        int bin = rt * PER;
 #pragma unroll
         for (int b = PER - 1; b >= 0; --b) {
-            if (acc + loc[b] >= k_rem) {
-                bin = t * PER + b;
+            if (acc + loc[b] >= want) {
+                bin = rt * PER + b;
                 break;
             }
             acc += loc[b];
         }
-        s.n_greater += acc;
-        s.k_rem = k_rem - acc;
-        const uint32_t prefix = (s.prefix << BITS) | static_cast<uint32_t>(bin);
-        s.prefix = prefix;
-        if (LEVEL == 2) {
-            s.threshold = prefix;
-            s.ties_take = k_rem - acc;
+        s_out[0] = static_cast<uint32_t>(bin);
+        s_out[1] = acc;
+    }
+    __syncthreads();
+    bin_out = s_out[0];
+    above_out = s_out[1];
+    __syncthreads();
+}
+
+// Multi-pass route: one CTA appends the picked bin of level LEVEL to the key prefix of s.
+template <int LEVEL>
+__device__ __forceinline__ void pick_body(SelectState &s, const uint32_t *h, uint32_t *s_scan,
+                                          uint32_t *s_out, uint32_t *status, uint32_t i)
+{
+    constexpr int BITS = (LEVEL == 2) ? 7 : 12;
+    const uint32_t k_rem = s.k_rem;
+    uint32_t bin, above;
+    pick_bin(h, k_rem, s_scan, s_out, bin, above);
+    if (threadIdx.x == 0) {
+        if (bin == 0xFFFFFFFFu) {
+            latch(status, DECO_ERR_DEVICE_CHECK, 0x100u + LEVEL, i);
+        } else {
+            s.n_greater += above;
+            s.k_rem = k_rem - above;
+            const uint32_t prefix = (s.prefix << BITS) | bin;
+            s.prefix = prefix;
+            if (LEVEL == 2) {
+                s.threshold = prefix;
+                s.ties_take = k_rem - above;
+            }
         }
     }
     __syncthreads();
 }
 
+// true for exactly one CTA per counter: the last of gridDim.x to get here (nothing waits)
+__device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *s_flag)
+{
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *s_flag = (atomicAdd(counter, 1u) == gridDim.x - 1) ? 1u : 0u;
+    __syncthreads();
+    const bool last = *s_flag != 0;
+    if (last) __threadfence();
+    return last;
+}
+
 // ------------------------------------------------------------------------------------------
-// Start of an iteration: one CTA per worker re-arms the selection record, clears the
-// histograms and, on the streaming route, draws the sample that fixes spec_key.
+// Start of an iteration.  SAMPLE_CTAS CTAs per worker: together they clear the histograms and,
+// on the streaming route, draw the sample (each thread one group of 4 consecutive entries,
+// groups evenly spread over [0, d)) and leave its keys in global memory; CTA 0 re-arms the
+// selection record; the last CTA of a worker to arrive fixes spec_key from the sample.
 // ------------------------------------------------------------------------------------------
 constexpr int BEGIN_BLOCK = 1024;
-constexpr int SAMPLE_CHUNKS = 8192;                        // 4 consecutive entries each
-constexpr int SAMPLE_PER_THREAD = SAMPLE_CHUNKS / BEGIN_BLOCK;   // 8 chunks = 32 keys
+constexpr int SAMPLE_CTAS = 8;
+constexpr int SAMPLE_CHUNKS = SAMPLE_CTAS * BEGIN_BLOCK;   // 8192 groups of 4 entries
+constexpr int SAMPLE_KEYS_PER_THREAD = 4 * SAMPLE_CTAS;    // keys per thread in the search
 
 template <int GT>
 __global__ void __launch_bounds__(BEGIN_BLOCK)
 begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t exact_all)
 {
-    const uint32_t i = blockIdx.x;
+    const uint32_t i = blockIdx.y, part = blockIdx.x;
     const int t = threadIdx.x;
     SelectState &s = p.sel[i];
     uint32_t *hz = hist_of(p, i, 0, 0);
-    for (int q = t; q < 2 * RADIX_LEVELS * RADIX_BINS; q += BEGIN_BLOCK) hz[q] = 0;
-    if (t < RADIX_LEVELS) p.done[i * RADIX_LEVELS + t] = 0;
-    if (i == 0 && t == 0) p.status[3] = exact_all;
-    if (t == 0) {
-        s.prefix = 0;
-        s.k_rem = p.k;
-        s.n_greater = 0;
-        s.threshold = 0;
-        s.ties_take = 0;
-        s.exact = exact_all;
-        s.spec_key = SPEC_DISABLED;
-        s.n_staged = 0;
-        if (exact_all) s.exact_total += 1;
+    for (int q = part * BEGIN_BLOCK + t; q < 2 * RADIX_LEVELS * RADIX_BINS;
+         q += SAMPLE_CTAS * BEGIN_BLOCK)
+        hz[q] = 0;
+    if (part == 0) {
+        if (t < RADIX_LEVELS) p.done[i * (RADIX_LEVELS + 1) + t] = 0;
+        if (i == 0 && t == 0) p.status[3] = exact_all;
+        if (t == 0) {
+            s.prefix = 0;
+            s.k_rem = p.k;
+            s.n_greater = 0;
+            s.threshold = 0;
+            s.ties_take = 0;
+            s.exact = exact_all;
+            s.spec_key = SPEC_DISABLED;
+            s.n_staged = 0;
+            s.n_boundary = 0;
+            if (exact_all) s.exact_total += 1;
+        }
     }
     if (exact_all) return;
 
-    // ---- sample: SAMPLE_CHUNKS groups of 4 consecutive entries, evenly spread over [0, d)
-    __shared__ uint32_t h[RADIX_BINS];
     __shared__ uint32_t s_w[33];
-    __shared__ uint32_t s_pick[2];
+    __shared__ uint32_t s_flag;
     const float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     const char *grow = reinterpret_cast<const char *>(grads) +
                        static_cast<size_t>(i) * p.d * (GT ? 2 : 4);
     const uint64_t nchunks = (p.d + 3) >> 2;
     const uint32_t S = nchunks < SAMPLE_CHUNKS ? static_cast<uint32_t>(nchunks) : SAMPLE_CHUNKS;
-    uint32_t keys[SAMPLE_PER_THREAD * 4];
-    uint32_t valid = 0;
+    uint4 *skeys = reinterpret_cast<uint4 *>(p.sample_keys) + static_cast<size_t>(i) * SAMPLE_CHUNKS;
+    {
+        const uint32_t sidx = part * BEGIN_BLOCK + t;
+        uint32_t kk[4] = {0, 0, 0, 0};                       // 0 = "not a sample"
+        if (sidx < S) {
+            const uint64_t j = ((static_cast<uint64_t>(sidx) * nchunks) / S) << 2;
+            const float4 ev = *reinterpret_cast<const float4 *>(erow + j);
+            const float es[4] = {ev.x, ev.y, ev.z, ev.w};
 #pragma unroll
-    for (int q = 0; q < SAMPLE_PER_THREAD; ++q) {
-        const uint32_t sidx = q * BEGIN_BLOCK + t;
-        uint64_t j = 0;
-        const bool on = sidx < S;
-        if (on) j = ((static_cast<uint64_t>(sidx) * nchunks) / S) << 2;
-        float4 ev = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (on) ev = *reinterpret_cast<const float4 *>(erow + j);
-        const float es[4] = {ev.x, ev.y, ev.z, ev.w};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const bool in = on && (j + c < p.d);
-            uint32_t key = 0xFFFFFFFFu;                      // marks "not a sample"
-            if (in) key = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
-            keys[q * 4 + c] = key;
-            valid += in ? 1u : 0u;
+            for (int c = 0; c < 4; ++c)
+                if (j + c < p.d)
+                    kk[c] = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
         }
+        skeys[sidx] = make_uint4(kk[0], kk[1], kk[2], kk[3]);
     }
-    uint32_t m_total;
-    block_excl_scan(valid, s_w, m_total);
+    // the arrival counter resets itself: only the last CTA touches it afterwards
+    uint32_t *arrive = &p.done[i * (RADIX_LEVELS + 1) + RADIX_LEVELS];
+    if (!last_cta_to_arrive(arrive, &s_flag)) return;
+    if (t == 0) *arrive = 0;
+
+    uint32_t keys[SAMPLE_KEYS_PER_THREAD];
+#pragma unroll
+    for (int q = 0; q < SAMPLE_CTAS; ++q) {
+        const uint4 v = __ldcg(skeys + q * BEGIN_BLOCK + t);
+        keys[q * 4 + 0] = v.x;
+        keys[q * 4 + 1] = v.y;
+        keys[q * 4 + 2] = v.z;
+        keys[q * 4 + 3] = v.w;
+    }
+    // every sampled group is complete unless the sample is the whole vector
+    const uint32_t m_total = (S == nchunks) ? static_cast<uint32_t>(p.d) : 4u * S;
     // rank inside the sample: mean + 5 sigma + 2 of a binomial with p = k/d (exact when the
     // sample is the whole vector)
     uint32_t R;
@@ -289,49 +337,71 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         if (t == 0) s.spec_key = 0;            // stage everything: the count check decides
         return;
     }
-    uint32_t prefix = 0, rem = R;
+    // Largest 24-bit key prefix v with  #(sample keys >= v) >= R, found bit by bit (no
+    // histogram, so equal or clustered keys cost nothing extra).  The exponent bits are
+    // settled on the whole sample; the keys that survive (those in the threshold's octave and
+    // above, a few percent) go onto per-warp lists in shared memory and the mantissa bits are
+    // settled on those.  Zero keys never count: every candidate is positive.
+    constexpr int WARP_LIST = 128;
+    constexpr int NW = BEGIN_BLOCK / 32;
+    __shared__ uint32_t s_list[NW * WARP_LIST];
+    __shared__ uint32_t s_cnt[NW];
+    auto count_all = [&](uint32_t cand) {
+        uint32_t c = 0;
+#pragma unroll
+        for (int q = 0; q < SAMPLE_KEYS_PER_THREAD; ++q) c += (keys[q] >= cand) ? 1u : 0u;
+        for (int o = 16; o > 0; o >>= 1) c += __shfl_down_sync(FULL, c, o);
+        if ((t & 31) == 0) s_w[t >> 5] = c;
+        __syncthreads();
+        if (t < 32) {
+            uint32_t v = s_w[t];
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(FULL, v, o);
+            if (t == 0) s_w[32] = v;
+        }
+        __syncthreads();
+        const uint32_t tot = s_w[32];
+        __syncthreads();
+        return tot;
+    };
+    uint32_t bound = 0;
 #pragma unroll 1
-    for (int level = 0; level < 2; ++level) {
-        for (int q = t; q < RADIX_BINS; q += BEGIN_BLOCK) h[q] = 0;
-        __syncthreads();
-#pragma unroll
-        for (int q = 0; q < SAMPLE_PER_THREAD * 4; ++q) {
-            const uint32_t key = keys[q];
-            if (key == 0xFFFFFFFFu) continue;
-            if (level == 0) atomicAdd(&h[key >> 19], 1u);
-            else if ((key >> 19) == prefix) atomicAdd(&h[(key >> 7) & 0xFFFu], 1u);
-        }
-        __syncthreads();
-        // suffix pick with 4 bins per thread
-        uint32_t loc[4], sum = 0;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            loc[b] = h[t * 4 + b];
-            sum += loc[b];
-        }
-        uint32_t tot;
-        const uint32_t below = block_excl_scan(sum, s_w, tot);   // bins below this thread's
-        const uint32_t s_here = tot - below, s_above = tot - below - sum;
-        if (s_here >= rem && s_above < rem) {
-            uint32_t acc = s_above;
-            int bin = t * 4;
-#pragma unroll
-            for (int b = 3; b >= 0; --b) {
-                if (acc + loc[b] >= rem) {
-                    bin = t * 4 + b;
-                    break;
-                }
-                acc += loc[b];
-            }
-            s_pick[0] = static_cast<uint32_t>(bin);
-            s_pick[1] = rem - acc;
-        }
-        __syncthreads();
-        prefix = (prefix << 12) | s_pick[0];
-        rem = s_pick[1];
-        __syncthreads();
+    for (int bit = 30; bit >= 23; --bit) {
+        const uint32_t cand = bound | (1u << bit);
+        if (count_all(cand) >= R) bound = cand;
     }
-    if (t == 0) s.spec_key = prefix << 7;      // lower edge of the 24-bit bin
+    const int lane = t & 31, w = t >> 5;
+    uint32_t mine = 0;                                       // warp-uniform running count
+#pragma unroll
+    for (int q = 0; q < SAMPLE_KEYS_PER_THREAD; ++q) {
+        const bool keep = keys[q] >= bound && keys[q] != 0;
+        const uint32_t m = __ballot_sync(FULL, keep);
+        const uint32_t at = mine + __popc(m & ((1u << lane) - 1u));
+        if (keep && at < WARP_LIST) s_list[w * WARP_LIST + at] = keys[q];
+        mine += __popc(m);
+    }
+    if (lane == 0) s_cnt[w] = mine;
+    __syncthreads();
+    bool fits = true;
+#pragma unroll
+    for (int ww = 0; ww < NW; ++ww) fits = fits && (s_cnt[ww] <= WARP_LIST);
+    // everything >= bound is on the lists, so counts over the lists equal counts over the
+    // sample for any candidate >= bound; lane l of warp w looks at slots l, l+32, ...
+#pragma unroll 1
+    for (int bit = 22; bit >= 7; --bit) {
+        const uint32_t cand = bound | (1u << bit);
+        uint32_t tot = 0;
+        if (fits) {
+#pragma unroll
+            for (int r = 0; r < WARP_LIST / 32; ++r) {
+                const uint32_t slot = r * 32 + lane;
+                tot += __syncthreads_count(slot < mine && s_list[w * WARP_LIST + slot] >= cand);
+            }
+        } else {
+            tot = count_all(cand);
+        }
+        if (tot >= R) bound = cand;
+    }
+    if (t == 0) s.spec_key = bound;            // a multiple of 128: lower edge of a 24-bit bin
 }
 
 // ------------------------------------------------------------------------------------------
@@ -346,6 +416,7 @@ ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__res
                      uint64_t d, float alpha, SelectState *__restrict__ sel,
                      deco_pair *__restrict__ stage, uint64_t stage_cap,
                      uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
+                     uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
                      uint32_t ntiles)
 {
     constexpr int V = Geo<GT>::V, U = Geo<GT>::U;
@@ -408,146 +479,274 @@ ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__res
             }
         }
     }
+    // zero_mask: per round, the entries to write as +0 instead of their value
+    auto store_tile = [&](const uint32_t *zero_mask) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint64_t j = wbase + u * (32 * V) + lane * V;
+            float y[V];
+#pragma unroll
+            for (int c = 0; c < V; ++c)
+                y[c] = (zero_mask && (zero_mask[u] & (1u << c))) ? 0.0f : x[u][c];
+#pragma unroll
+            for (int q = 0; q < V / 4; ++q)
+                *reinterpret_cast<float4 *>(erow + j + 4 * q) =
+                    make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+        }
+    };
+    if (!SPEC) {
+        store_tile(nullptr);
+        return;
+    }
+
+    // Stage every entry whose key reaches the speculative bound, in index order, into a
+    // segment reserved with one atomic per tile.  Staged entries are written to e as +0 (the
+    // guess is that they are selected); the selection kernels write the value back for the
+    // few that are not.  The store is issued before any barrier; a tile whose segment turns
+    // out not to fit stores its values again.
+    __shared__ uint32_t s_w[WARPS];
+    __shared__ uint32_t s_off;
+    const uint32_t bound = sel[i].spec_key;
+    uint32_t m[U], cnt[U], pos[U], any = 0;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint64_t j = wbase + u * (32 * V) + lane * V;
+        m[u] = 0;
 #pragma unroll
-        for (int q = 0; q < V / 4; ++q)
-            *reinterpret_cast<float4 *>(erow + j + 4 * q) =
-                make_float4(x[u][4 * q], x[u][4 * q + 1], x[u][4 * q + 2], x[u][4 * q + 3]);
+        for (int c = 0; c < V; ++c)
+            if (mag_key(x[u][c]) >= bound && (full || j + c < d)) m[u] |= 1u << c;
+        cnt[u] = __popc(m[u]);
+        any |= m[u];
     }
-
-    if (SPEC) {
-        // Stage every entry whose key reaches the speculative bound, in index order, into a
-        // segment reserved with one atomic per tile.
-        __shared__ uint32_t s_w[WARPS];
-        __shared__ uint32_t s_off;
-        const uint32_t bound = sel[i].spec_key;
-        uint32_t m[U], cnt[U], pos[U], any = 0;
+    store_tile(m);
+    uint32_t total = 0;
+    if (__syncthreads_or(any != 0)) {
+        ordered_prefix<U>(cnt, pos, s_w, total);
+    }
+    if (threadIdx.x == 0) {
+        uint32_t off = 0;
+        if (total) off = atomicAdd(&sel[i].n_staged, total);
+        tile_off[static_cast<size_t>(i) * ntiles + tile] = off;
+        tile_cnt[static_cast<size_t>(i) * ntiles + tile] = total;
+        tile_rej[static_cast<size_t>(i) * ntiles + tile] = 0;
+        tile_eq[static_cast<size_t>(i) * ntiles + tile] = 0;
+        s_off = off;
+    }
+    if (total == 0) return;
+    __syncthreads();
+    const uint64_t off = s_off;
+    if (off + total > stage_cap) {                   // overflow: n_staged tells the selector,
+        store_tile(nullptr);                         // and this tile takes its values back
+        return;
+    }
+    deco_pair *out = stage + static_cast<size_t>(i) * stage_cap + off;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t j = wbase + u * (32 * V) + lane * V;
-            m[u] = 0;
+    for (int u = 0; u < U; ++u) {
+        const uint64_t j = wbase + u * (32 * V) + lane * V;
+        uint32_t q = pos[u];
 #pragma unroll
-            for (int c = 0; c < V; ++c)
-                if (mag_key(x[u][c]) >= bound && (full || j + c < d)) m[u] |= 1u << c;
-            cnt[u] = __popc(m[u]);
-            any |= m[u];
-        }
-        uint32_t total = 0;
-        if (__syncthreads_or(any != 0)) {
-            ordered_prefix<U>(cnt, pos, s_w, total);
-        }
-        if (threadIdx.x == 0) {
-            uint32_t off = 0;
-            if (total) off = atomicAdd(&sel[i].n_staged, total);
-            tile_off[static_cast<size_t>(i) * ntiles + tile] = off;
-            tile_cnt[static_cast<size_t>(i) * ntiles + tile] = total;
-            s_off = off;
-        }
-        if (total == 0) return;
-        __syncthreads();
-        const uint64_t off = s_off;
-        if (off + total > stage_cap) return;         // overflow: n_staged tells the selector
-        deco_pair *out = stage + static_cast<size_t>(i) * stage_cap + off;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t j = wbase + u * (32 * V) + lane * V;
-            uint32_t q = pos[u];
-#pragma unroll
-            for (int c = 0; c < V; ++c)
-                if (m[u] & (1u << c)) {
-                    deco_pair pr;
-                    pr.idx = static_cast<uint32_t>(j + c);
-                    pr.val = x[u][c];
-                    out[q++] = pr;
-                }
-        }
+        for (int c = 0; c < V; ++c)
+            if (m[u] & (1u << c)) {
+                deco_pair pr;
+                pr.idx = static_cast<uint32_t>(j + c);
+                pr.val = x[u][c];
+                out[q++] = pr;
+            }
     }
 }
 
 // ------------------------------------------------------------------------------------------
 // Streaming route: exact selection among the staged pairs.
 // ------------------------------------------------------------------------------------------
-// Histogram of one radix level over the staged pairs of each worker; the last CTA of a worker
-// to arrive (counted with an atomic after a fence, no waiting) does the pick.  At level 0 the
-// pick first checks that the staged set is valid: n_staged in [k, stage_cap].  If not, the
-// worker is handed to the multi-pass route.
-template <int LEVEL>
+// Staged keys are at or above spec_key, and the threshold sits just above it, so the two
+// radix levels work on  rel = key - spec_key : level A bins rel >> 12 (everything from
+// 4095 * 4096 up shares the top bin), level B bins the low 12 bits inside the chosen A bin.
+constexpr uint32_t REL_TOP = RADIX_BINS - 1;
+
+__device__ __forceinline__ uint32_t rel_bin_a(uint32_t key, uint32_t spec)
+{
+    const uint32_t b = (key - spec) >> 12;
+    return b < REL_TOP ? b : REL_TOP;
+}
+
+__device__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w, bool streaming);
+
+// Level A: histogram of the coarse bins of all staged keys (nothing else; the decision is
+// taken by the next kernel).
 __global__ void __launch_bounds__(BLOCK)
-stage_hist_pick_kernel(Sel p)
+stage_hist_a_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.y;
+    const SelectState &s = p.sel[i];
+    if (s.exact) return;
+    const uint32_t n_staged = s.n_staged, spec = s.spec_key;
+    if (n_staged < p.k || n_staged > p.stage_cap) return;
+    __shared__ uint32_t h[RADIX_BINS];
+    for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
+    __syncthreads();
+    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
+    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+         base += gridDim.x * (4 * BLOCK)) {
+        float v[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint32_t q = base + r * BLOCK + threadIdx.x;
+            v[r] = q < n_staged ? src[q].val : 0.0f;
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+            if (base + r * BLOCK + threadIdx.x < n_staged)
+                atomicAdd(&h[rel_bin_a(mag_key(v[r]), spec)], 1u);
+    }
+    __syncthreads();
+    uint32_t *out = hist_of(p, i, 0, 0);
+    for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
+        if (h[b]) atomicAdd(&out[b], h[b]);
+}
+
+// Every CTA first repeats the same small decision from the level-A histogram: is the staged
+// set usable (at least k entries, so it contains the k largest, and no overflow of the
+// staging area), and which coarse bin holds the k-th largest.  If the set is not usable, or
+// the threshold falls into the shared top bin, the worker is handed to the multi-pass route.
+//
+// Level B.  Every staged entry is looked at once more: those below the chosen A bin are
+// rejected for good and counted per tile; those inside it go into the level-B histogram and
+// onto the short boundary list.  The last CTA to arrive then fixes the threshold, settles the
+// boundary entries (below -> rejected, equal -> tie), and turns the per-tile counts into
+// message positions.  Rejected entries get their value back in e.
+__global__ void __launch_bounds__(BLOCK)
+stage_select_kernel(Sel p)
 {
     const uint32_t i = blockIdx.y;
     SelectState &s = p.sel[i];
     if (s.exact) return;
     __shared__ uint32_t h[RADIX_BINS];
-    __shared__ uint32_t suf[BLOCK + 1];
-    __shared__ uint32_t s_last;
-    const uint32_t n_staged = s.n_staged;
+    __shared__ uint32_t s_scan[33];
+    __shared__ uint32_t s_misc[3];
+    const uint32_t n_staged = s.n_staged, spec = s.spec_key;
     const bool valid = n_staged >= p.k && n_staged <= p.stage_cap;
-    if (valid) {
-        for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
-        __syncthreads();
-        const uint32_t prefix = s.prefix;
-        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
-        for (uint32_t q = blockIdx.x * BLOCK + threadIdx.x; q < n_staged; q += gridDim.x * BLOCK)
-            radix_bin<LEVEL>(mag_key(src[q].val), prefix, h);
-        __syncthreads();
-        uint32_t *out = hist_of(p, i, 0, LEVEL);
-        for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
-            if (h[b]) atomicAdd(&out[b], h[b]);
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0)
-        s_last = (atomicAdd(&p.done[i * RADIX_LEVELS + LEVEL], 1u) == gridDim.x - 1) ? 1u : 0u;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    if (!valid) {
-        if (threadIdx.x == 0) {
+    uint32_t a_sel = REL_TOP, above_a = 0;
+    if (valid) pick_bin(hist_of(p, i, 0, 0), p.k, s_scan, s_misc, a_sel, above_a);
+    if (!valid || a_sel >= REL_TOP) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
             s.exact = 1;
             s.exact_total += 1;
             p.status[3] = 1;
         }
         return;
     }
-    pick_body<LEVEL>(s, hist_of(p, i, 0, LEVEL), suf, p.status, i);
-}
-
-// One warp per tile: entries above / equal to the threshold among the tile's staged pairs.
-__global__ void __launch_bounds__(BLOCK)
-tile_count_stage_kernel(Sel p)
-{
-    const uint32_t i = blockIdx.y;
-    if (p.sel[i].exact) return;
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t tile = blockIdx.x * WARPS + w;
-    if (tile >= p.ntiles) return;
-    const uint32_t T = p.sel[i].threshold;
-    const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
-    const uint32_t cnt = p.tile_cnt[ti];
-    uint32_t gt = 0, eq = 0;
-    if (cnt) {
-        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + p.tile_off[ti];
-        for (uint32_t q = lane; q < cnt; q += 32) {
-            const uint32_t key = mag_key(src[q].val);
-            gt += key > T;
-            eq += key == T;
+    const uint32_t k_rem = p.k - above_a;
+    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
+    uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
+    uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
+    deco_pair *bnd = p.boundary + static_cast<size_t>(i) * BOUNDARY_CAP;
+    float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+    for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+         base += gridDim.x * (4 * BLOCK)) {                  // the loop is uniform per CTA
+        deco_pair prs[4];
+        uint32_t bm[4], on = 0, warp_total = 0;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint32_t q = base + r * BLOCK + threadIdx.x;
+            prs[r].idx = 0;
+            prs[r].val = 0.f;
+            if (q < n_staged) prs[r] = src[q];
         }
-        for (int o = 16; o > 0; o >>= 1) {
-            gt += __shfl_down_sync(FULL, gt, o);
-            eq += __shfl_down_sync(FULL, eq, o);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            uint32_t a = REL_TOP + 1;                         // "no entry"
+            if (base + r * BLOCK + threadIdx.x < n_staged) a = rel_bin_a(mag_key(prs[r].val), spec);
+            if (a < a_sel) atomicAdd(&rej[prs[r].idx / TILE], 1u);   // rejected for good
+            const bool f = (a == a_sel);
+            on |= f ? (1u << r) : 0u;
+            bm[r] = __ballot_sync(FULL, f);
+            warp_total += __popc(bm[r]);
+        }
+        if (warp_total) {                                    // one list reservation per warp
+            uint32_t at = 0;
+            if (lane == 0) at = atomicAdd(&s.n_boundary, warp_total);
+            at = __shfl_sync(FULL, at, 0);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                if (on & (1u << r)) {
+                    atomicAdd(&h[(mag_key(prs[r].val) - spec) & 0xFFFu], 1u);
+                    const uint32_t slot = at + __popc(bm[r] & ((1u << lane) - 1u));
+                    if (slot < BOUNDARY_CAP) bnd[slot] = prs[r];
+                }
+                at += __popc(bm[r]);
+            }
         }
     }
-    if (lane == 0) {
-        p.tile_gt[ti] = gt;
-        p.tile_eq[ti] = eq;
+    __syncthreads();
+    uint32_t *out = hist_of(p, i, 0, 1);
+    for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
+        if (h[b]) atomicAdd(&out[b], h[b]);
+    const bool last = last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 1], &s_misc[2]);
+
+    // Off the critical path (after the arrival): undo the guess for the rejected entries.
+    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+         base += gridDim.x * (4 * BLOCK)) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint32_t q = base + r * BLOCK + threadIdx.x;
+            if (q < n_staged) {
+                const deco_pair pr = src[q];
+                if (rel_bin_a(mag_key(pr.val), spec) < a_sel) erow[pr.idx] = pr.val;
+            }
+        }
     }
+    if (!last) return;
+
+    uint32_t bin, above;
+    pick_bin(hist_of(p, i, 0, 1), k_rem, s_scan, s_misc, bin, above);
+    if (bin == 0xFFFFFFFFu) {                       // counts do not add up: report, stay safe
+        if (threadIdx.x == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x120u, i);
+        return;
+    }
+    const uint32_t T = spec + (a_sel << 12) + bin;
+    if (threadIdx.x == 0) {
+        s.prefix = (a_sel << 12) | bin;
+        s.k_rem = k_rem - above;
+        s.threshold = T;
+        s.n_greater = above_a + above;
+        s.ties_take = k_rem - above;
+    }
+    const uint32_t nb = __ldcg(&s.n_boundary);
+    if (nb <= BOUNDARY_CAP) {
+        for (uint32_t q = threadIdx.x; q < nb; q += BLOCK) {
+            // written by other CTAs of this launch: read through L2
+            const uint2 raw = __ldcg(reinterpret_cast<const uint2 *>(bnd) + q);
+            const uint32_t key = raw.y & 0x7FFFFFFFu;
+            if (key < T) {
+                atomicAdd(&rej[raw.x / TILE], 1u);
+                erow[raw.x] = __uint_as_float(raw.y);
+            } else if (key == T) {
+                atomicAdd(&eqc[raw.x / TILE], 1u);
+            }
+        }
+    } else {                                        // list overflowed: walk all staged entries
+        for (uint32_t q = threadIdx.x; q < n_staged; q += BLOCK) {
+            const deco_pair pr = src[q];
+            const uint32_t key = mag_key(pr.val);
+            if (rel_bin_a(key, spec) != a_sel) continue;
+            if (key < T) {
+                atomicAdd(&rej[pr.idx / TILE], 1u);
+                erow[pr.idx] = pr.val;
+            } else if (key == T) {
+                atomicAdd(&eqc[pr.idx / TILE], 1u);
+            }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    scan_tiles_body(p, i, s_scan, true);
 }
 
-// One warp per tile: ordered filter of the tile's staged pairs into the message; the selected
-// entries become +0 in e.
+// One warp per tile: ordered filter of the tile's staged pairs into the message.  The selected
+// entries are already +0 in e; ties that are not taken get their value back.
 __global__ void __launch_bounds__(BLOCK)
 emit_stage_kernel(Sel p)
 {
@@ -561,40 +760,46 @@ emit_stage_kernel(Sel p)
     if (cnt == 0) return;
     const uint32_t start = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile];
     const uint32_t want = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile + 1] - start;
-    if (want == 0) return;
     const uint32_t T = p.sel[i].threshold;
     const uint32_t take = p.tile_take[ti];
     const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + p.tile_off[ti];
     deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
     float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     uint32_t written = 0, ties_seen = 0;
-    for (uint32_t base = 0; base < cnt; base += 32) {
-        const uint32_t q = base + lane;
-        deco_pair pr;
-        pr.idx = 0;
-        pr.val = 0.f;
-        bool gt = false, eq = false;
-        if (q < cnt) {
-            pr = src[q];
-            const uint32_t key = mag_key(pr.val);
-            gt = key > T;
-            eq = key == T;
+    for (uint32_t base = 0; base < cnt; base += 128) {       // four loads in flight per lane
+        deco_pair prs[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint32_t q = base + r * 32 + lane;
+            prs[r].idx = 0;
+            prs[r].val = 0.f;
+            if (q < cnt) prs[r] = src[q];
         }
-        const uint32_t eq_mask = __ballot_sync(FULL, eq);
-        const uint32_t rank = ties_seen + __popc(eq_mask & ((1u << lane) - 1u));
-        const bool pick = gt || (eq && rank < take);
-        const uint32_t pick_mask = __ballot_sync(FULL, pick);
-        if (pick) {
-            const uint32_t pos = start + written + __popc(pick_mask & ((1u << lane) - 1u));
-            if (pos < p.k && pr.idx < p.d) {
-                out[pos] = pr;
-                erow[pr.idx] = 0.0f;
-            } else {
-                latch(p.status, DECO_ERR_DEVICE_CHECK, 0x310u, tile);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const deco_pair pr = prs[r];
+            bool gt = false, eq = false;
+            if (base + r * 32 + lane < cnt) {
+                const uint32_t key = mag_key(pr.val);
+                gt = key > T;
+                eq = key == T;
             }
+            const uint32_t eq_mask = __ballot_sync(FULL, eq);
+            const uint32_t rank = ties_seen + __popc(eq_mask & ((1u << lane) - 1u));
+            const bool pick = gt || (eq && rank < take);
+            const uint32_t pick_mask = __ballot_sync(FULL, pick);
+            if (pick) {
+                const uint32_t pos = start + written + __popc(pick_mask & ((1u << lane) - 1u));
+                if (pos < p.k && pr.idx < p.d) {
+                    out[pos] = pr;                           // e already holds +0 there
+                } else {
+                    latch(p.status, DECO_ERR_DEVICE_CHECK, 0x310u, tile);
+                }
+            }
+            if (eq && !pick && pr.idx < p.d) erow[pr.idx] = pr.val;   // tie not taken: undo the guess
+            written += __popc(pick_mask);
+            ties_seen += __popc(eq_mask);
         }
-        written += __popc(pick_mask);
-        ties_seen += __popc(eq_mask);
     }
     if (lane == 0 && written != want) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x311u, tile);
 }
@@ -670,35 +875,79 @@ __device__ __forceinline__ void count_e_tile(const Sel &p, uint32_t i, uint32_t 
 }
 
 // One CTA per worker (any block size): ties are granted to tiles in index order until
-// ties_take are used up, then every tile gets its position in the message.
-__device__ __forceinline__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w /*[33]*/)
+// ties_take are used up, then every tile gets its position in the message.  On the streaming
+// route the entries above the threshold of a tile are its staged entries minus the rejected
+// ones and the ties; on the multi-pass route they were counted directly.
+__device__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w /*[33]*/, bool streaming)
 {
     const uint32_t nt = blockDim.x;
-    const uint32_t *gt = p.tile_gt + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t *gtp = p.tile_gt + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t *cnt = p.tile_cnt + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     const uint32_t *eq = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
+    auto gt = [&](uint32_t t) { return streaming ? cnt[t] - rej[t] - eq[t] : gtp[t]; };
     uint32_t *take = p.tile_take + static_cast<size_t>(i) * p.ntiles;
     uint32_t *start = p.tile_start + static_cast<size_t>(i) * (p.ntiles + 1);
     const uint32_t ties = p.sel[i].ties_take;
     const uint32_t per = (p.ntiles + nt - 1) / nt;
     const uint32_t lo = min(p.ntiles, threadIdx.x * per), hi = min(p.ntiles, lo + per);
-    uint32_t eq_sum = 0;
-    for (uint32_t t = lo; t < hi; ++t) eq_sum += eq[t];
-    uint32_t eq_total;
-    uint32_t eq_before = block_excl_scan(eq_sum, s_w, eq_total);
-    uint32_t sel_sum = 0;
-    for (uint32_t t = lo; t < hi; ++t) {
-        const uint32_t q = eq[t];
-        const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
-        const uint32_t tk = min(q, left);
-        take[t] = tk;
-        sel_sum += gt[t] + tk;
-        eq_before += q;
-    }
     uint32_t sel_total;
-    uint32_t pos = block_excl_scan(sel_sum, s_w, sel_total);
-    for (uint32_t t = lo; t < hi; ++t) {
-        start[t] = pos;
-        pos += gt[t] + take[t];
+    constexpr uint32_t REG = 8;
+    if (per <= REG) {
+        // short ranges: every load is issued once, up front
+        uint32_t g[REG], q[REG];
+#pragma unroll
+        for (uint32_t r = 0; r < REG; ++r) {
+            const uint32_t t = lo + r;
+            g[r] = q[r] = 0;
+            if (t < hi) {
+                q[r] = eq[t];
+                g[r] = gt(t);
+            }
+        }
+        uint32_t eq_sum = 0;
+#pragma unroll
+        for (uint32_t r = 0; r < REG; ++r) eq_sum += q[r];
+        uint32_t eq_total;
+        uint32_t eq_before = block_excl_scan(eq_sum, s_w, eq_total);
+        uint32_t sel_sum = 0;
+#pragma unroll
+        for (uint32_t r = 0; r < REG; ++r) {
+            const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
+            const uint32_t tk = min(q[r], left);
+            eq_before += q[r];
+            q[r] = tk;
+            sel_sum += g[r] + tk;
+        }
+        uint32_t pos = block_excl_scan(sel_sum, s_w, sel_total);
+#pragma unroll
+        for (uint32_t r = 0; r < REG; ++r) {
+            const uint32_t t = lo + r;
+            if (t < hi) {
+                take[t] = q[r];
+                start[t] = pos;
+            }
+            pos += g[r] + q[r];
+        }
+    } else {
+        uint32_t eq_sum = 0;
+        for (uint32_t t = lo; t < hi; ++t) eq_sum += eq[t];
+        uint32_t eq_total;
+        uint32_t eq_before = block_excl_scan(eq_sum, s_w, eq_total);
+        uint32_t sel_sum = 0;
+        for (uint32_t t = lo; t < hi; ++t) {
+            const uint32_t q = eq[t];
+            const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
+            const uint32_t tk = min(q, left);
+            take[t] = tk;
+            sel_sum += gt(t) + tk;
+            eq_before += q;
+        }
+        uint32_t pos = block_excl_scan(sel_sum, s_w, sel_total);
+        for (uint32_t t = lo; t < hi; ++t) {
+            start[t] = pos;
+            pos += gt(t) + take[t];
+        }
     }
     if (threadIdx.x == 0) {
         start[p.ntiles] = sel_total;
@@ -803,8 +1052,9 @@ __global__ void __launch_bounds__(BLOCK) radix_pick_kernel(Sel p)
 {
     const uint32_t i = blockIdx.x;
     if (!p.sel[i].exact) return;
-    __shared__ uint32_t suf[BLOCK + 1];
-    pick_body<LEVEL>(p.sel[i], hist_of(p, i, 1, LEVEL), suf, p.status, i);
+    __shared__ uint32_t s_scan[33];
+    __shared__ uint32_t s_out[2];
+    pick_body<LEVEL>(p.sel[i], hist_of(p, i, 1, LEVEL), s_scan, s_out, p.status, i);
 }
 
 __global__ void __launch_bounds__(BLOCK) tile_count_e_kernel(Sel p)
@@ -815,14 +1065,13 @@ __global__ void __launch_bounds__(BLOCK) tile_count_e_kernel(Sel p)
     count_e_tile(p, i, blockIdx.x, s_a, s_b);
 }
 
-// exact_only: 1 = scan the workers on the multi-pass route, 0 = those on the streaming route
 constexpr int SCAN_BLOCK = 1024;
-__global__ void __launch_bounds__(SCAN_BLOCK) tile_scan_kernel(Sel p, uint32_t exact_only)
+__global__ void __launch_bounds__(SCAN_BLOCK) tile_scan_kernel(Sel p)
 {
     const uint32_t i = blockIdx.x;
-    if ((p.sel[i].exact != 0) != (exact_only != 0)) return;
+    if (!p.sel[i].exact) return;
     __shared__ uint32_t s_w[33];
-    scan_tiles_body(p, i, s_w);
+    scan_tiles_body(p, i, s_w, false);
 }
 
 __global__ void __launch_bounds__(BLOCK) emit_e_kernel(Sel p)
@@ -841,9 +1090,27 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
     if (__ldcg(&p.status[3]) == 0) return;
     cg::grid_group grid = cg::this_grid();
     __shared__ uint32_t h[RADIX_BINS];
-    __shared__ uint32_t suf[BLOCK + 1];
-    __shared__ uint32_t s_a[33], s_b[WARPS];
+    __shared__ uint32_t s_a[33], s_b[WARPS], s_out[2];
     const uint32_t cta = blockIdx.x, ncta = gridDim.x;
+    // The streaming pass wrote +0 over the staged entries of every tile whose segment fitted;
+    // the passes below need the values back.
+    for (uint32_t i = 0; i < p.n; ++i) {
+        if (!p.sel[i].exact) continue;
+        float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+        for (uint32_t tile = cta; tile < p.ntiles; tile += ncta) {
+            const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
+            const uint32_t cnt = p.tile_cnt[ti];
+            const uint64_t off = p.tile_off[ti];
+            if (cnt == 0 || off + cnt > p.stage_cap) continue;
+            const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
+            for (uint32_t q = threadIdx.x; q < cnt; q += BLOCK) {
+                const deco_pair pr = src[q];
+                if (pr.idx < p.d) erow[pr.idx] = pr.val;
+            }
+        }
+    }
+    __threadfence();
+    grid.sync();
     for (int level = 0; level < RADIX_LEVELS; ++level) {
         for (uint32_t i = 0; i < p.n; ++i) {
             if (!p.sel[i].exact) continue;
@@ -855,9 +1122,9 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
         grid.sync();
         for (uint32_t i = cta; i < p.n; i += ncta) {
             if (!p.sel[i].exact) continue;
-            if (level == 0) pick_body<0>(p.sel[i], hist_of(p, i, 1, 0), suf, p.status, i);
-            else if (level == 1) pick_body<1>(p.sel[i], hist_of(p, i, 1, 1), suf, p.status, i);
-            else pick_body<2>(p.sel[i], hist_of(p, i, 1, 2), suf, p.status, i);
+            if (level == 0) pick_body<0>(p.sel[i], hist_of(p, i, 1, 0), s_a, s_out, p.status, i);
+            else if (level == 1) pick_body<1>(p.sel[i], hist_of(p, i, 1, 1), s_a, s_out, p.status, i);
+            else pick_body<2>(p.sel[i], hist_of(p, i, 1, 2), s_a, s_out, p.status, i);
         }
         __threadfence();
         grid.sync();
@@ -870,7 +1137,7 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
     grid.sync();
     for (uint32_t i = cta; i < p.n; i += ncta) {
         if (!p.sel[i].exact) continue;
-        scan_tiles_body(p, i, s_a);
+        scan_tiles_body(p, i, s_a, false);
     }
     __threadfence();
     grid.sync();
@@ -895,12 +1162,15 @@ Sel make_sel(const deco_ctx *c)
     p.sel = c->sel;
     p.hist = c->hist;
     p.done = c->done;
+    p.sample_keys = c->sample_keys;
     p.tile_gt = c->tile_gt;
     p.tile_eq = c->tile_eq;
     p.tile_take = c->tile_take;
     p.tile_start = c->tile_start;
     p.tile_off = c->tile_off;
     p.tile_cnt = c->tile_cnt;
+    p.tile_rej = c->tile_rej;
+    p.boundary = c->boundary;
     p.msg = c->msg;
     p.k_cap = c->k_cap;
     p.stage = c->stage;
@@ -928,10 +1198,11 @@ cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s)
 {
     const float alpha = c->lr_at_server ? 1.0f : c->lr;
     const uint32_t exact_all = streaming_route(c) ? 0u : 1u;
+    const dim3 grid(SAMPLE_CTAS, c->n);
     if (c->grad_dtype == DECO_BF16)
-        begin_step_kernel<1><<<c->n, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
+        begin_step_kernel<1><<<grid, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
     else
-        begin_step_kernel<0><<<c->n, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
+        begin_step_kernel<0><<<grid, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
     c->launches += 1;
     return cudaGetLastError();
 }
@@ -943,11 +1214,11 @@ static void launch_acc(deco_ctx *c, const void *grads, float alpha, cudaStream_t
     if (streaming_route(c))
         ef_accumulate_kernel<GT, ALIGNED, true><<<grid, BLOCK, 0, s>>>(
             c->e, c->e_stride, grads, c->d, alpha, c->sel, c->stage, c->stage_cap, c->tile_off,
-            c->tile_cnt, c->ntiles);
+            c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
     else
         ef_accumulate_kernel<GT, ALIGNED, false><<<grid, BLOCK, 0, s>>>(
             c->e, c->e_stride, grads, c->d, alpha, c->sel, c->stage, c->stage_cap, c->tile_off,
-            c->tile_cnt, c->ntiles);
+            c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
 }
 
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s)
@@ -993,21 +1264,18 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
         radix_hist_e_kernel<2><<<hgrid, BLOCK, 0, s>>>(p);
         radix_pick_kernel<2><<<c->n, BLOCK, 0, s>>>(p);
         tile_count_e_kernel<<<tgrid, BLOCK, 0, s>>>(p);
-        tile_scan_kernel<<<c->n, SCAN_BLOCK, 0, s>>>(p, 1u);
+        tile_scan_kernel<<<c->n, SCAN_BLOCK, 0, s>>>(p);
         emit_e_kernel<<<tgrid, BLOCK, 0, s>>>(p);
         c->launches += 9;
         return cudaGetLastError();
     }
-    // staged pairs per worker are a few times k: size the histogram grid for that
-    dim3 sgrid(part_blocks(c, 2 * c->k + 65536, BLOCK * 8), c->n);
+    // staged pairs per worker are a few times k: size the grids for that
+    dim3 sgrid(part_blocks(c, 2 * c->k + 65536, BLOCK * 4), c->n);
     dim3 wgrid((c->ntiles + WARPS - 1) / WARPS, c->n);
-    stage_hist_pick_kernel<0><<<sgrid, BLOCK, 0, s>>>(p);
-    stage_hist_pick_kernel<1><<<sgrid, BLOCK, 0, s>>>(p);
-    stage_hist_pick_kernel<2><<<sgrid, BLOCK, 0, s>>>(p);
-    tile_count_stage_kernel<<<wgrid, BLOCK, 0, s>>>(p);
-    tile_scan_kernel<<<c->n, SCAN_BLOCK, 0, s>>>(p, 0u);
+    stage_hist_a_kernel<<<sgrid, BLOCK, 0, s>>>(p);
+    stage_select_kernel<<<sgrid, BLOCK, 0, s>>>(p);
     emit_stage_kernel<<<wgrid, BLOCK, 0, s>>>(p);
-    c->launches += 6;
+    c->launches += 3;
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     void *args[] = {&p};

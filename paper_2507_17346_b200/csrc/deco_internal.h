@@ -35,11 +35,19 @@ struct SelectState {
     uint32_t spec_key;      // speculative lower bound used by the streaming pass (or DISABLED)
     uint32_t n_staged;      // candidates staged by the streaming pass
     uint32_t exact_total;   // cumulative count of steps that took the multi-pass path
-    uint32_t pad[7];
+    uint32_t n_boundary;    // staged entries that fell into the threshold's coarse bin
+    uint32_t pad[6];
 };
 static_assert(sizeof(SelectState) == 64, "one line per worker");
 
 constexpr uint32_t SPEC_DISABLED = 0x80000000u;   // above every 31-bit key
+
+// Staged entries whose coarse bin is the threshold's are also appended to a short list so
+// that one CTA can settle them; if the list overflows that CTA walks all staged entries.
+constexpr uint32_t BOUNDARY_CAP = 8192;
+
+// Keys of the per-iteration sample kept per worker (8192 groups of 4 entries).
+constexpr uint32_t SAMPLE_KEYS = 32768;
 
 struct Slot {
     uint64_t step = 0;
@@ -74,7 +82,8 @@ struct deco_ctx {
     deco_pair *slots = nullptr;         // [ring][n * k_cap]
     deco_pair *stage = nullptr;         // [n][stage_cap]
     uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
-    uint32_t *done = nullptr;           // [n][RADIX_LEVELS] CTA arrival counters
+    uint32_t *done = nullptr;           // [n][RADIX_LEVELS + 1] CTA arrival counters
+    uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
     uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
     deco::SelectState *sel = nullptr;   // [n]
     uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
@@ -83,6 +92,8 @@ struct deco_ctx {
     uint32_t *tile_start = nullptr;     // [n][ntiles + 1] message position of each tile
     uint32_t *tile_off = nullptr;       // [n][ntiles]  staging offset of each tile's candidates
     uint32_t *tile_cnt = nullptr;       // [n][ntiles]  staged candidates per tile
+    uint32_t *tile_rej = nullptr;       // [n][ntiles]  staged candidates below the threshold
+    deco_pair *boundary = nullptr;      // [n][BOUNDARY_CAP] staged entries of the threshold's bin
     uint32_t *dev_status = nullptr;     // [4]: status, two detail words, fallback flag
     void *grads_staging = nullptr;      // device copy of host gradients (deco_step_host)
     uint64_t device_bytes = 0;

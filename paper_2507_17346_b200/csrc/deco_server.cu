@@ -17,6 +17,7 @@ namespace deco {
 namespace {
 
 constexpr uint32_t FULL = 0xFFFFFFFFu;
+constexpr uint32_t PREFETCH_WORKERS = 16;   // workers whose entries one thread holds at once
 
 __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t a, uint32_t b)
 {
@@ -42,12 +43,13 @@ aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
 
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         uint64_t out_off = 0;
-        uint32_t cap = 0;
+        uint32_t cap = 0, longest = 0;
         for (uint32_t i = 0; i < n; ++i) {
             const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
             const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
             out_off += a;
             cap += b - a;
+            longest = max(longest, b - a);
         }
         if (cap == 0) continue;
         if (out_off + cap > positions) {
@@ -55,22 +57,63 @@ aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
             continue;
         }
         const uint32_t first = tile * static_cast<uint32_t>(TILE);
-        for (uint32_t i = 0; i < n; ++i) {                     // worker order 0..n-1
-            const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-            const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
-            if (b == a) continue;
-            const deco_pair *src = msg + static_cast<size_t>(i) * k_cap;
-            for (uint32_t p = a + threadIdx.x; p < b; p += BLOCK) {
-                const deco_pair pr = src[p];
-                const uint32_t loc = pr.idx - first;
-                if (loc >= static_cast<uint32_t>(TILE)) {
-                    latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pr.idx);
-                    continue;
+        if (n <= PREFETCH_WORKERS && longest <= static_cast<uint32_t>(BLOCK)) {
+            // Sparse case: at most one entry per thread and worker.  All loads are issued
+            // before the first barrier, then the workers are added in order from registers.
+            deco_pair pre[PREFETCH_WORKERS];
+#pragma unroll
+            for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
+                pre[i].idx = DECO_NO_INDEX;
+                pre[i].val = 0.0f;
+                if (i < n) {
+                    const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
+                    const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+                    if (a + threadIdx.x < b) pre[i] = msg[static_cast<size_t>(i) * k_cap + a + threadIdx.x];
                 }
-                acc[loc] = acc[loc] + pr.val;                  // indices are unique per worker
-                atomicOr(&mask[loc >> 5], 1u << (loc & 31));
             }
-            __syncthreads();
+#pragma unroll
+            for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
+                if (i >= n) break;
+                if (pre[i].idx != DECO_NO_INDEX) {
+                    const uint32_t loc = pre[i].idx - first;
+                    if (loc >= static_cast<uint32_t>(TILE)) {
+                        latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pre[i].idx);
+                    } else {
+                        acc[loc] = acc[loc] + pre[i].val;      // indices are unique per worker
+                        atomicOr(&mask[loc >> 5], 1u << (loc & 31));
+                    }
+                }
+                __syncthreads();
+            }
+        } else {
+            for (uint32_t i = 0; i < n; ++i) {                 // worker order 0..n-1
+                const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
+                const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+                if (b == a) continue;
+                const deco_pair *src = msg + static_cast<size_t>(i) * k_cap;
+                for (uint32_t p0 = a; p0 < b; p0 += 4 * BLOCK) {   // four loads in flight
+                    deco_pair prs[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const uint32_t p = p0 + r * BLOCK + threadIdx.x;
+                        prs[r].idx = DECO_NO_INDEX;
+                        prs[r].val = 0.0f;
+                        if (p < b) prs[r] = src[p];
+                    }
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        if (prs[r].idx == DECO_NO_INDEX) continue;
+                        const uint32_t loc = prs[r].idx - first;
+                        if (loc >= static_cast<uint32_t>(TILE)) {
+                            latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, prs[r].idx);
+                            continue;
+                        }
+                        acc[loc] = acc[loc] + prs[r].val;      // indices are unique per worker
+                        atomicOr(&mask[loc >> 5], 1u << (loc & 31));
+                    }
+                }
+                __syncthreads();
+            }
         }
         uint32_t word = mask[threadIdx.x];
         const uint32_t c = __popc(word);
