@@ -45,6 +45,7 @@ struct Sel {
     uint32_t *hist;          // [n][2][RADIX_LEVELS][RADIX_BINS]: 0 = staged route, 1 = multi-pass
     uint32_t *done;          // [n][RADIX_LEVELS + 1] CTA arrival counters
     uint32_t *sample_keys;   // [n][4 * SAMPLE_CHUNKS] keys of the sample
+    uint32_t *sample_hist;   // [n][256] sample keys per exponent; cleared by its reader
     uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt, *tile_rej;
     deco_pair *boundary;     // [n][BOUNDARY_CAP]
     deco_pair *msg;
@@ -306,6 +307,19 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
                     kk[c] = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
         }
         skeys[sidx] = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+        // exponent histogram of this CTA's nonzero keys: lanes with the same exponent elect
+        // one of them to add the group's size
+        __shared__ uint32_t s_exp[256];
+        if (t < 256) s_exp[t] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t e8 = kk[c] ? (kk[c] >> 23) : 256u;
+            const uint32_t grp = __match_any_sync(FULL, e8);
+            if (e8 < 256u && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_exp[e8], __popc(grp));
+        }
+        __syncthreads();
+        if (t < 256 && s_exp[t]) atomicAdd(&p.sample_hist[i * 256 + t], s_exp[t]);
     }
     // the arrival counter resets itself: only the last CTA touches it afterwards
     uint32_t *arrive = &p.done[i * (RADIX_LEVELS + 1) + RADIX_LEVELS];
@@ -335,11 +349,11 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     }
     if (R > m_total) {                         // the sample cannot bound the threshold
         if (t == 0) s.spec_key = 0;            // stage everything: the count check decides
+        if (t < 256) p.sample_hist[i * 256 + t] = 0;
         return;
     }
-    // Largest 24-bit key prefix v with  #(sample keys >= v) >= R, found bit by bit (no
-    // histogram, so equal or clustered keys cost nothing extra).  The exponent bits are
-    // settled on the whole sample; the keys that survive (those in the threshold's octave and
+    // Largest 24-bit key prefix v with  #(sample keys >= v) >= R.  The exponent bits come
+    // from the exponent histogram the sampling CTAs filled; the keys that survive (those in the threshold's octave and
     // above, a few percent) go onto per-warp lists in shared memory and the mantissa bits are
     // settled on those.  Zero keys never count: every candidate is positive.
     constexpr int WARP_LIST = 128;
@@ -363,11 +377,23 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         __syncthreads();
         return tot;
     };
+    // exponent (octave) of the R-th largest sample key from the 256-bin histogram; thread t
+    // looks at exponent 255 - t so that the prefix over threads counts the higher octaves
     uint32_t bound = 0;
-#pragma unroll 1
-    for (int bit = 30; bit >= 23; --bit) {
-        const uint32_t cand = bound | (1u << bit);
-        if (count_all(cand) >= R) bound = cand;
+    {
+        uint32_t mine_e = 0;
+        if (t < 256) {
+            mine_e = __ldcg(&p.sample_hist[i * 256 + (255 - t)]);
+            p.sample_hist[i * 256 + (255 - t)] = 0;             // ready for the next iteration
+        }
+        uint32_t tot;
+        const uint32_t higher = block_excl_scan(mine_e, s_w, tot);
+        if (t == 0) s_flag = 0;
+        __syncthreads();
+        if (t < 256 && higher < R && higher + mine_e >= R) s_flag = static_cast<uint32_t>(255 - t) << 23;
+        __syncthreads();
+        bound = s_flag;
+        __syncthreads();
     }
     const int lane = t & 31, w = t >> 5;
     uint32_t mine = 0;                                       // warp-uniform running count
@@ -686,19 +712,25 @@ stage_select_kernel(Sel p)
         if (h[b]) atomicAdd(&out[b], h[b]);
     const bool last = last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 1], &s_misc[2]);
 
-    // Off the critical path (after the arrival): undo the guess for the rejected entries.
-    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
-         base += gridDim.x * (4 * BLOCK)) {
+    // Off the critical path: undo the guess for the rejected entries.  The last CTA does its
+    // share at the very end, after the serial work the next kernel is waiting for.
+    auto write_back_rejected = [&]() {
+        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+             base += gridDim.x * (4 * BLOCK)) {
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const uint32_t q = base + r * BLOCK + threadIdx.x;
-            if (q < n_staged) {
-                const deco_pair pr = src[q];
-                if (rel_bin_a(mag_key(pr.val), spec) < a_sel) erow[pr.idx] = pr.val;
+            for (int r = 0; r < 4; ++r) {
+                const uint32_t q = base + r * BLOCK + threadIdx.x;
+                if (q < n_staged) {
+                    const deco_pair pr = src[q];
+                    if (rel_bin_a(mag_key(pr.val), spec) < a_sel) erow[pr.idx] = pr.val;
+                }
             }
         }
+    };
+    if (!last) {
+        write_back_rejected();
+        return;
     }
-    if (!last) return;
 
     uint32_t bin, above;
     pick_bin(hist_of(p, i, 0, 1), k_rem, s_scan, s_misc, bin, above);
@@ -743,6 +775,7 @@ stage_select_kernel(Sel p)
     __threadfence();
     __syncthreads();
     scan_tiles_body(p, i, s_scan, true);
+    write_back_rejected();
 }
 
 // One warp per tile: ordered filter of the tile's staged pairs into the message.  The selected
@@ -1163,6 +1196,7 @@ Sel make_sel(const deco_ctx *c)
     p.hist = c->hist;
     p.done = c->done;
     p.sample_keys = c->sample_keys;
+    p.sample_hist = c->sample_hist;
     p.tile_gt = c->tile_gt;
     p.tile_eq = c->tile_eq;
     p.tile_take = c->tile_take;

@@ -84,6 +84,7 @@ struct deco_ctx {
     uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
     uint32_t *done = nullptr;           // [n][RADIX_LEVELS + 1] CTA arrival counters
     uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
+    uint32_t *sample_hist = nullptr;    // [n][256] sample keys per exponent (self-clearing)
     uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
     deco::SelectState *sel = nullptr;   // [n]
     uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
