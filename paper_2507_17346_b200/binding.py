@@ -9,7 +9,8 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdeco.so")
+# DECO_LIB names another build of the library (for instance a debug build); default: in-tree.
+LIB_PATH = os.environ.get("DECO_LIB") or os.path.join(_HERE, "libdeco.so")
 
 DECO_OK = 0
 DECO_ERR_INVALID_ARG = 1

@@ -45,7 +45,7 @@ struct Sel {
     uint32_t *hist;          // [n][2][RADIX_LEVELS][RADIX_BINS]: 0 = staged route, 1 = multi-pass
     uint32_t *done;          // [n][RADIX_LEVELS + 1] CTA arrival counters
     uint32_t *sample_keys;   // [n][4 * SAMPLE_CHUNKS] keys of the sample
-    uint32_t *sample_hist;   // [n][256] sample keys per exponent; cleared by its reader
+    uint32_t *sample_hist;   // [n][1024] sample keys per top-10-bit bin; cleared by its reader
     uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt, *tile_rej;
     deco_pair *boundary;     // [n][BOUNDARY_CAP]
     deco_pair *msg;
@@ -256,6 +256,9 @@ constexpr int BEGIN_BLOCK = 1024;
 constexpr int SAMPLE_CTAS = 8;
 constexpr int SAMPLE_CHUNKS = SAMPLE_CTAS * BEGIN_BLOCK;   // 8192 groups of 4 entries
 constexpr int SAMPLE_KEYS_PER_THREAD = 4 * SAMPLE_CTAS;    // keys per thread in the search
+constexpr int SAMPLE_HIST_SHIFT = 21;                      // 31-bit key -> its top 10 bits
+constexpr uint32_t SAMPLE_HIST_BINS = 1u << (31 - SAMPLE_HIST_SHIFT);
+static_assert(SAMPLE_HIST_BINS == BEGIN_BLOCK, "one histogram bin per thread");
 
 template <int GT>
 __global__ void __launch_bounds__(BEGIN_BLOCK)
@@ -281,6 +284,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
             s.spec_key = SPEC_DISABLED;
             s.n_staged = 0;
             s.n_boundary = 0;
+            s.rel_shift = 12;
             if (exact_all) s.exact_total += 1;
         }
     }
@@ -307,19 +311,20 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
                     kk[c] = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
         }
         skeys[sidx] = make_uint4(kk[0], kk[1], kk[2], kk[3]);
-        // exponent histogram of this CTA's nonzero keys: lanes with the same exponent elect
-        // one of them to add the group's size
-        __shared__ uint32_t s_exp[256];
-        if (t < 256) s_exp[t] = 0;
+        // histogram of the top SAMPLE_HIST_BITS key bits (exponent and two mantissa bits) of
+        // this CTA's nonzero keys: lanes with the same bin elect one of them to add the
+        // group's size
+        __shared__ uint32_t s_exp[SAMPLE_HIST_BINS];
+        s_exp[t] = 0;
         __syncthreads();
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const uint32_t e8 = kk[c] ? (kk[c] >> 23) : 256u;
-            const uint32_t grp = __match_any_sync(FULL, e8);
-            if (e8 < 256u && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_exp[e8], __popc(grp));
+            const uint32_t hb = kk[c] ? (kk[c] >> SAMPLE_HIST_SHIFT) : SAMPLE_HIST_BINS;
+            const uint32_t grp = __match_any_sync(FULL, hb);
+            if (hb < SAMPLE_HIST_BINS && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_exp[hb], __popc(grp));
         }
         __syncthreads();
-        if (t < 256 && s_exp[t]) atomicAdd(&p.sample_hist[i * 256 + t], s_exp[t]);
+        if (s_exp[t]) atomicAdd(&p.sample_hist[i * SAMPLE_HIST_BINS + t], s_exp[t]);
     }
     // the arrival counter resets itself: only the last CTA touches it afterwards
     uint32_t *arrive = &p.done[i * (RADIX_LEVELS + 1) + RADIX_LEVELS];
@@ -340,20 +345,25 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     // rank inside the sample: mean + 5 sigma + 2 of a binomial with p = k/d (exact when the
     // sample is the whole vector)
     uint32_t R;
+    uint32_t rel_shift = 10;
     if (m_total >= p.d) {
         R = p.k;
     } else {
         const double mean = static_cast<double>(p.k) * m_total / static_cast<double>(p.d);
         const double r = mean + 5.0 * sqrt(mean) + 2.0;
         R = r >= static_cast<double>(m_total) ? m_total + 1u : static_cast<uint32_t>(r) + 1u;
+        // how far the sampled rank sits above k/d decides how far above the bound the
+        // threshold may lie (in value: that ratio to the power 1/tail-index)
+        const double rho = static_cast<double>(R) / (mean > 1e-9 ? mean : 1e-9);
+        rel_shift = rho <= 2.0 ? 10u : (rho <= 8.0 ? 11u : 12u);
     }
     if (R > m_total) {                         // the sample cannot bound the threshold
         if (t == 0) s.spec_key = 0;            // stage everything: the count check decides
-        if (t < 256) p.sample_hist[i * 256 + t] = 0;
+        p.sample_hist[i * SAMPLE_HIST_BINS + t] = 0;
         return;
     }
-    // Largest 24-bit key prefix v with  #(sample keys >= v) >= R.  The exponent bits come
-    // from the exponent histogram the sampling CTAs filled; the keys that survive (those in the threshold's octave and
+    // Largest 24-bit key prefix v with  #(sample keys >= v) >= R.  The top bits come from
+    // the histogram the sampling CTAs filled; the keys that survive (those in the threshold's octave and
     // above, a few percent) go onto per-warp lists in shared memory and the mantissa bits are
     // settled on those.  Zero keys never count: every candidate is positive.
     constexpr int WARP_LIST = 128;
@@ -377,20 +387,18 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         __syncthreads();
         return tot;
     };
-    // exponent (octave) of the R-th largest sample key from the 256-bin histogram; thread t
-    // looks at exponent 255 - t so that the prefix over threads counts the higher octaves
+    // top bits of the R-th largest sample key from the histogram; thread t looks at the
+    // mirrored bin so that the prefix over threads counts the higher bins
     uint32_t bound = 0;
     {
-        uint32_t mine_e = 0;
-        if (t < 256) {
-            mine_e = __ldcg(&p.sample_hist[i * 256 + (255 - t)]);
-            p.sample_hist[i * 256 + (255 - t)] = 0;             // ready for the next iteration
-        }
+        const uint32_t hb = SAMPLE_HIST_BINS - 1 - t;
+        const uint32_t mine_e = __ldcg(&p.sample_hist[i * SAMPLE_HIST_BINS + hb]);
+        p.sample_hist[i * SAMPLE_HIST_BINS + hb] = 0;           // ready for the next iteration
         uint32_t tot;
         const uint32_t higher = block_excl_scan(mine_e, s_w, tot);
         if (t == 0) s_flag = 0;
         __syncthreads();
-        if (t < 256 && higher < R && higher + mine_e >= R) s_flag = static_cast<uint32_t>(255 - t) << 23;
+        if (higher < R && higher + mine_e >= R) s_flag = hb << SAMPLE_HIST_SHIFT;
         __syncthreads();
         bound = s_flag;
         __syncthreads();
@@ -407,18 +415,19 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     }
     if (lane == 0) s_cnt[w] = mine;
     __syncthreads();
-    bool fits = true;
+    uint32_t longest = 0;
 #pragma unroll
-    for (int ww = 0; ww < NW; ++ww) fits = fits && (s_cnt[ww] <= WARP_LIST);
+    for (int ww = 0; ww < NW; ++ww) longest = max(longest, s_cnt[ww]);
+    const bool fits = longest <= WARP_LIST;
+    const int rounds = (longest + 31) / 32;                  // same for every thread
     // everything >= bound is on the lists, so counts over the lists equal counts over the
     // sample for any candidate >= bound; lane l of warp w looks at slots l, l+32, ...
 #pragma unroll 1
-    for (int bit = 22; bit >= 7; --bit) {
+    for (int bit = SAMPLE_HIST_SHIFT - 1; bit >= 7; --bit) {
         const uint32_t cand = bound | (1u << bit);
         uint32_t tot = 0;
         if (fits) {
-#pragma unroll
-            for (int r = 0; r < WARP_LIST / 32; ++r) {
+            for (int r = 0; r < rounds; ++r) {
                 const uint32_t slot = r * 32 + lane;
                 tot += __syncthreads_count(slot < mine && s_list[w * WARP_LIST + slot] >= cand);
             }
@@ -427,7 +436,10 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         }
         if (tot >= R) bound = cand;
     }
-    if (t == 0) s.spec_key = bound;            // a multiple of 128: lower edge of a 24-bit bin
+    if (t == 0) {
+        s.spec_key = bound;                    // a multiple of 128: lower edge of a 24-bit bin
+        s.rel_shift = rel_shift;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -585,56 +597,76 @@ ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__res
 // Streaming route: exact selection among the staged pairs.
 // ------------------------------------------------------------------------------------------
 // Staged keys are at or above spec_key, and the threshold sits just above it, so the two
-// radix levels work on  rel = key - spec_key : level A bins rel >> 12 (everything from
-// 4095 * 4096 up shares the top bin), level B bins the low 12 bits inside the chosen A bin.
+// radix levels work on  rel = key - spec_key : level A bins rel >> shift (everything from
+// 4095 << shift up, i.e. half an octave to two octaves above the bound, shares the top bin),
+// level B bins the low `shift` bits inside the chosen A bin.
 constexpr uint32_t REL_TOP = RADIX_BINS - 1;
 
-__device__ __forceinline__ uint32_t rel_bin_a(uint32_t key, uint32_t spec)
+// The width of a level-A bin is 2^shift key units with shift = sel[i].rel_shift in 10..12,
+// chosen with the bound: the further the sampled rank had to be pushed above k/d (small k),
+// the further above the bound the threshold may lie, and the wider the bins.
+__device__ __forceinline__ uint32_t rel_bin_a(uint32_t key, uint32_t spec, uint32_t shift)
 {
-    const uint32_t b = (key - spec) >> 12;
+    const uint32_t b = (key - spec) >> shift;
     return b < REL_TOP ? b : REL_TOP;
 }
 
 __device__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w, bool streaming);
 
-// Level A: histogram of the coarse bins of all staged keys (nothing else; the decision is
-// taken by the next kernel).
+// Level A: histogram of the coarse bins of all staged keys.  The last CTA of a worker to
+// arrive takes the decision: is the staged set usable (at least k entries, so it contains the
+// k largest, and no overflow of the staging area), and which coarse bin holds the k-th
+// largest.  If the set is not usable, or the threshold falls into the shared top bin, the
+// worker is handed to the multi-pass route.
 __global__ void __launch_bounds__(BLOCK)
 stage_hist_a_kernel(Sel p)
 {
     const uint32_t i = blockIdx.y;
-    const SelectState &s = p.sel[i];
+    SelectState &s = p.sel[i];
     if (s.exact) return;
-    const uint32_t n_staged = s.n_staged, spec = s.spec_key;
-    if (n_staged < p.k || n_staged > p.stage_cap) return;
+    const uint32_t n_staged = s.n_staged, spec = s.spec_key, shift = s.rel_shift;
+    const bool valid = n_staged >= p.k && n_staged <= p.stage_cap;
     __shared__ uint32_t h[RADIX_BINS];
-    for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
-    __syncthreads();
-    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
-    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
-         base += gridDim.x * (4 * BLOCK)) {
-        float v[4];
+    __shared__ uint32_t s_scan[33];
+    __shared__ uint32_t s_misc[3];
+    if (valid) {
+        for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
+        __syncthreads();
+        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
+        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+             base += gridDim.x * (4 * BLOCK)) {
+            float v[4];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const uint32_t q = base + r * BLOCK + threadIdx.x;
-            v[r] = q < n_staged ? src[q].val : 0.0f;
+            for (int r = 0; r < 4; ++r) {
+                const uint32_t q = base + r * BLOCK + threadIdx.x;
+                v[r] = q < n_staged ? src[q].val : 0.0f;
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                if (base + r * BLOCK + threadIdx.x < n_staged)
+                    atomicAdd(&h[rel_bin_a(mag_key(v[r]), spec, shift)], 1u);
         }
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-            if (base + r * BLOCK + threadIdx.x < n_staged)
-                atomicAdd(&h[rel_bin_a(mag_key(v[r]), spec)], 1u);
+        __syncthreads();
+        uint32_t *out = hist_of(p, i, 0, 0);
+        for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
+            if (h[b]) atomicAdd(&out[b], h[b]);
     }
-    __syncthreads();
-    uint32_t *out = hist_of(p, i, 0, 0);
-    for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
-        if (h[b]) atomicAdd(&out[b], h[b]);
+    if (!last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 0], &s_misc[2])) return;
+    uint32_t a_sel = REL_TOP, above_a = 0;
+    if (valid) pick_bin(hist_of(p, i, 0, 0), p.k, s_scan, s_misc, a_sel, above_a);
+    if (threadIdx.x == 0) {
+        if (!valid || a_sel >= REL_TOP) {
+            s.exact = 1;
+            s.exact_total += 1;
+            p.status[3] = 1;
+        } else {
+            s.prefix = a_sel;
+            s.n_greater = above_a;
+            s.k_rem = p.k - above_a;
+        }
+    }
 }
 
-// Every CTA first repeats the same small decision from the level-A histogram: is the staged
-// set usable (at least k entries, so it contains the k largest, and no overflow of the
-// staging area), and which coarse bin holds the k-th largest.  If the set is not usable, or
-// the threshold falls into the shared top bin, the worker is handed to the multi-pass route.
-//
 // Level B.  Every staged entry is looked at once more: those below the chosen A bin are
 // rejected for good and counted per tile; those inside it go into the level-B histogram and
 // onto the short boundary list.  The last CTA to arrive then fixes the threshold, settles the
@@ -649,19 +681,9 @@ stage_select_kernel(Sel p)
     __shared__ uint32_t h[RADIX_BINS];
     __shared__ uint32_t s_scan[33];
     __shared__ uint32_t s_misc[3];
-    const uint32_t n_staged = s.n_staged, spec = s.spec_key;
-    const bool valid = n_staged >= p.k && n_staged <= p.stage_cap;
-    uint32_t a_sel = REL_TOP, above_a = 0;
-    if (valid) pick_bin(hist_of(p, i, 0, 0), p.k, s_scan, s_misc, a_sel, above_a);
-    if (!valid || a_sel >= REL_TOP) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) {
-            s.exact = 1;
-            s.exact_total += 1;
-            p.status[3] = 1;
-        }
-        return;
-    }
-    const uint32_t k_rem = p.k - above_a;
+    const uint32_t n_staged = s.n_staged, spec = s.spec_key, shift = s.rel_shift;
+    const uint32_t a_sel = s.prefix, above_a = s.n_greater, k_rem = s.k_rem;   // from level A
+    const uint32_t low_mask = (1u << shift) - 1u;
     const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
     uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
@@ -684,7 +706,7 @@ stage_select_kernel(Sel p)
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             uint32_t a = REL_TOP + 1;                         // "no entry"
-            if (base + r * BLOCK + threadIdx.x < n_staged) a = rel_bin_a(mag_key(prs[r].val), spec);
+            if (base + r * BLOCK + threadIdx.x < n_staged) a = rel_bin_a(mag_key(prs[r].val), spec, shift);
             if (a < a_sel) atomicAdd(&rej[prs[r].idx / TILE], 1u);   // rejected for good
             const bool f = (a == a_sel);
             on |= f ? (1u << r) : 0u;
@@ -698,7 +720,7 @@ stage_select_kernel(Sel p)
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 if (on & (1u << r)) {
-                    atomicAdd(&h[(mag_key(prs[r].val) - spec) & 0xFFFu], 1u);
+                    atomicAdd(&h[(mag_key(prs[r].val) - spec) & low_mask], 1u);
                     const uint32_t slot = at + __popc(bm[r] & ((1u << lane) - 1u));
                     if (slot < BOUNDARY_CAP) bnd[slot] = prs[r];
                 }
@@ -722,7 +744,7 @@ stage_select_kernel(Sel p)
                 const uint32_t q = base + r * BLOCK + threadIdx.x;
                 if (q < n_staged) {
                     const deco_pair pr = src[q];
-                    if (rel_bin_a(mag_key(pr.val), spec) < a_sel) erow[pr.idx] = pr.val;
+                    if (rel_bin_a(mag_key(pr.val), spec, shift) < a_sel) erow[pr.idx] = pr.val;
                 }
             }
         }
@@ -738,9 +760,9 @@ stage_select_kernel(Sel p)
         if (threadIdx.x == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x120u, i);
         return;
     }
-    const uint32_t T = spec + (a_sel << 12) + bin;
+    const uint32_t T = spec + (a_sel << shift) + bin;
     if (threadIdx.x == 0) {
-        s.prefix = (a_sel << 12) | bin;
+        s.prefix = (a_sel << shift) | bin;
         s.k_rem = k_rem - above;
         s.threshold = T;
         s.n_greater = above_a + above;
@@ -748,22 +770,32 @@ stage_select_kernel(Sel p)
     }
     const uint32_t nb = __ldcg(&s.n_boundary);
     if (nb <= BOUNDARY_CAP) {
-        for (uint32_t q = threadIdx.x; q < nb; q += BLOCK) {
-            // written by other CTAs of this launch: read through L2
-            const uint2 raw = __ldcg(reinterpret_cast<const uint2 *>(bnd) + q);
-            const uint32_t key = raw.y & 0x7FFFFFFFu;
-            if (key < T) {
-                atomicAdd(&rej[raw.x / TILE], 1u);
-                erow[raw.x] = __uint_as_float(raw.y);
-            } else if (key == T) {
-                atomicAdd(&eqc[raw.x / TILE], 1u);
+        for (uint32_t q0 = 0; q0 < nb; q0 += 4 * BLOCK) {
+            // written by other CTAs of this launch: read through L2; four loads in flight
+            uint2 raw[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const uint32_t q = q0 + r * BLOCK + threadIdx.x;
+                raw[r] = make_uint2(0u, 0xFFFFFFFFu);
+                if (q < nb) raw[r] = __ldcg(reinterpret_cast<const uint2 *>(bnd) + q);
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                if (q0 + r * BLOCK + threadIdx.x >= nb) continue;
+                const uint32_t key = raw[r].y & 0x7FFFFFFFu;
+                if (key < T) {
+                    atomicAdd(&rej[raw[r].x / TILE], 1u);
+                    erow[raw[r].x] = __uint_as_float(raw[r].y);
+                } else if (key == T) {
+                    atomicAdd(&eqc[raw[r].x / TILE], 1u);
+                }
             }
         }
     } else {                                        // list overflowed: walk all staged entries
         for (uint32_t q = threadIdx.x; q < n_staged; q += BLOCK) {
             const deco_pair pr = src[q];
             const uint32_t key = mag_key(pr.val);
-            if (rel_bin_a(key, spec) != a_sel) continue;
+            if (rel_bin_a(key, spec, shift) != a_sel) continue;
             if (key < T) {
                 atomicAdd(&rej[pr.idx / TILE], 1u);
                 erow[pr.idx] = pr.val;

@@ -36,7 +36,8 @@ struct SelectState {
     uint32_t n_staged;      // candidates staged by the streaming pass
     uint32_t exact_total;   // cumulative count of steps that took the multi-pass path
     uint32_t n_boundary;    // staged entries that fell into the threshold's coarse bin
-    uint32_t pad[6];
+    uint32_t rel_shift;     // log2 width of a coarse bin of the staged-key histogram (10..12)
+    uint32_t pad[5];
 };
 static_assert(sizeof(SelectState) == 64, "one line per worker");
 
@@ -84,7 +85,7 @@ struct deco_ctx {
     uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
     uint32_t *done = nullptr;           // [n][RADIX_LEVELS + 1] CTA arrival counters
     uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
-    uint32_t *sample_hist = nullptr;    // [n][256] sample keys per exponent (self-clearing)
+    uint32_t *sample_hist = nullptr;    // [n][1024] sample keys per top-10-bit bin (self-clearing)
     uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
     deco::SelectState *sel = nullptr;   // [n]
     uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
