@@ -54,7 +54,11 @@ void free_all(deco_ctx *c)
     cudaFree(c->tile_off);
     cudaFree(c->tile_cnt);
     cudaFree(c->tile_rej);
-    cudaFree(c->boundary);
+    cudaFree(c->chunk_cnt);
+    cudaFree(c->chunk_rej);
+    cudaFree(c->chunk_eq);
+    cudaFree(c->chunk_eqb);
+    cudaFree(c->chunk_start);
     cudaFree(c->sample_keys);
     cudaFree(c->sample_hist);
     cudaFree(c->done);
@@ -164,6 +168,7 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     c->k_cap = deco_k_from_delta(c->delta_max, d);
     c->ntiles = static_cast<uint32_t>((d + TILE - 1) / TILE);
     c->e_stride = static_cast<uint64_t>(c->ntiles) * TILE;
+    c->nchunks = (c->ntiles + CHUNK_TILES - 1) / CHUNK_TILES;
     c->ring = c->tau_max + 1;
     // staged candidates per worker: six times the message capacity plus slack, at most d
     c->stage_cap = 6 * c->k_cap + 65536;
@@ -199,7 +204,11 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->tile_off, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_cnt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_rej, static_cast<uint64_t>(n) * c->ntiles));
-    need(dev_alloc(c, &c->boundary, static_cast<uint64_t>(n) * BOUNDARY_CAP));
+    need(dev_alloc(c, &c->chunk_cnt, static_cast<uint64_t>(n) * c->nchunks));
+    need(dev_alloc(c, &c->chunk_rej, static_cast<uint64_t>(n) * c->nchunks));
+    need(dev_alloc(c, &c->chunk_eq, static_cast<uint64_t>(n) * c->nchunks));
+    need(dev_alloc(c, &c->chunk_eqb, static_cast<uint64_t>(n) * c->nchunks));
+    need(dev_alloc(c, &c->chunk_start, static_cast<uint64_t>(n) * (c->nchunks + 1)));
     need(dev_alloc(c, &c->dev_status, 4));
     if (st == DECO_OK && query_fallback_grid(c) != cudaSuccess) st = DECO_ERR_CUDA;
     if (st == DECO_OK) st = zero_state(c, nullptr);

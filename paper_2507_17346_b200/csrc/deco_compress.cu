@@ -8,8 +8,9 @@
 // reads e and g, writes a into e and stages every entry whose key reaches the bound (a few
 // times k pairs, each tile's entries in index order); staged entries are written to e as +0
 // on the guess that they will be selected.  The exact threshold is then found by a two-level
-// radix selection over the staged pairs only (on key - spec_key), the message is an ordered
-// filter of them, and the few staged entries that are not selected get their value back.
+// radix selection over the staged pairs only (on key - spec_key), a classification pass counts
+// the rejected entries and the ties per tile and per chunk of tiles, the message is an ordered
+// filter of the staged pairs, and the few that are not selected get their value back.
 // The count of staged pairs proves the bound was valid (>= k of them); if it was not, or the
 // staging area overflowed, that worker takes the second route in the same call.
 //
@@ -47,7 +48,10 @@ struct Sel {
     uint32_t *sample_keys;   // [n][4 * SAMPLE_CHUNKS] keys of the sample
     uint32_t *sample_hist;   // [n][1024] sample keys per top-10-bit bin; cleared by its reader
     uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt, *tile_rej;
-    deco_pair *boundary;     // [n][BOUNDARY_CAP]
+    uint32_t nchunks;        // chunks of CHUNK_TILES tiles
+    uint32_t *chunk_cnt, *chunk_rej, *chunk_eq;   // [n][nchunks] staged / rejected / ties
+    uint32_t *chunk_eqb;     // [n][nchunks] ties in earlier chunks
+    uint32_t *chunk_start;   // [n][nchunks + 1] message position of each chunk
     deco_pair *msg;
     uint64_t k_cap;
     deco_pair *stage;
@@ -283,7 +287,6 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
             s.exact = exact_all;
             s.spec_key = SPEC_DISABLED;
             s.n_staged = 0;
-            s.n_boundary = 0;
             s.rel_shift = 12;
             if (exact_all) s.exact_total += 1;
         }
@@ -667,13 +670,10 @@ stage_hist_a_kernel(Sel p)
     }
 }
 
-// Level B.  Every staged entry is looked at once more: those below the chosen A bin are
-// rejected for good and counted per tile; those inside it go into the level-B histogram and
-// onto the short boundary list.  The last CTA to arrive then fixes the threshold, settles the
-// boundary entries (below -> rejected, equal -> tie), and turns the per-tile counts into
-// message positions.  Rejected entries get their value back in e.
+// Level B: histogram of the low bits of the staged keys that fell into the chosen A bin; the
+// last CTA of a worker to arrive fixes the threshold key and the number of ties to take.
 __global__ void __launch_bounds__(BLOCK)
-stage_select_kernel(Sel p)
+stage_hist_b_kernel(Sel p)
 {
     const uint32_t i = blockIdx.y;
     SelectState &s = p.sel[i];
@@ -685,57 +685,90 @@ stage_select_kernel(Sel p)
     const uint32_t a_sel = s.prefix, above_a = s.n_greater, k_rem = s.k_rem;   // from level A
     const uint32_t low_mask = (1u << shift) - 1u;
     const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
-    uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
-    uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
-    deco_pair *bnd = p.boundary + static_cast<size_t>(i) * BOUNDARY_CAP;
-    float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
     __syncthreads();
-    const int lane = threadIdx.x & 31;
     for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
-         base += gridDim.x * (4 * BLOCK)) {                  // the loop is uniform per CTA
-        deco_pair prs[4];
-        uint32_t bm[4], on = 0, warp_total = 0;
+         base += gridDim.x * (4 * BLOCK)) {
+        float v[4];
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const uint32_t q = base + r * BLOCK + threadIdx.x;
-            prs[r].idx = 0;
-            prs[r].val = 0.f;
-            if (q < n_staged) prs[r] = src[q];
+            v[r] = q < n_staged ? src[q].val : 0.0f;
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            uint32_t a = REL_TOP + 1;                         // "no entry"
-            if (base + r * BLOCK + threadIdx.x < n_staged) a = rel_bin_a(mag_key(prs[r].val), spec, shift);
-            if (a < a_sel) atomicAdd(&rej[prs[r].idx / TILE], 1u);   // rejected for good
-            const bool f = (a == a_sel);
-            on |= f ? (1u << r) : 0u;
-            bm[r] = __ballot_sync(FULL, f);
-            warp_total += __popc(bm[r]);
-        }
-        if (warp_total) {                                    // one list reservation per warp
-            uint32_t at = 0;
-            if (lane == 0) at = atomicAdd(&s.n_boundary, warp_total);
-            at = __shfl_sync(FULL, at, 0);
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                if (on & (1u << r)) {
-                    atomicAdd(&h[(mag_key(prs[r].val) - spec) & low_mask], 1u);
-                    const uint32_t slot = at + __popc(bm[r] & ((1u << lane) - 1u));
-                    if (slot < BOUNDARY_CAP) bnd[slot] = prs[r];
-                }
-                at += __popc(bm[r]);
-            }
+            if (base + r * BLOCK + threadIdx.x >= n_staged) continue;
+            const uint32_t key = mag_key(v[r]);
+            if (rel_bin_a(key, spec, shift) == a_sel) atomicAdd(&h[(key - spec) & low_mask], 1u);
         }
     }
     __syncthreads();
     uint32_t *out = hist_of(p, i, 0, 1);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
         if (h[b]) atomicAdd(&out[b], h[b]);
-    const bool last = last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 1], &s_misc[2]);
+    if (!last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 1], &s_misc[2])) return;
+    uint32_t bin, above;
+    pick_bin(hist_of(p, i, 0, 1), k_rem, s_scan, s_misc, bin, above);
+    if (threadIdx.x == 0) {
+        if (bin == 0xFFFFFFFFu) {                   // counts do not add up: report, stay safe
+            latch(p.status, DECO_ERR_DEVICE_CHECK, 0x120u, i);
+            s.threshold = 0x7FFFFFFFu;
+            s.ties_take = 0;
+        } else {
+            s.prefix = (a_sel << shift) | bin;
+            s.k_rem = k_rem - above;
+            s.threshold = spec + (a_sel << shift) + bin;
+            s.n_greater = above_a + above;
+            s.ties_take = k_rem - above;
+        }
+    }
+}
 
-    // Off the critical path: undo the guess for the rejected entries.  The last CTA does its
-    // share at the very end, after the serial work the next kernel is waiting for.
+// Classification.  With the threshold known every staged entry below it is rejected: counted
+// for its tile and its chunk (CHUNK_TILES consecutive tiles) and given its value back in e;
+// entries equal to it are counted as ties.  The last CTA of a worker to arrive then walks the
+// chunks once: ties are granted in index order until ties_take are used up and every chunk
+// gets its position in the message.  (The per-tile positions follow from these inside the
+// emit kernel, so nothing here is serial in the number of tiles.)
+__global__ void __launch_bounds__(BLOCK)
+stage_classify_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.y;
+    const SelectState &s = p.sel[i];
+    if (s.exact) return;
+    __shared__ uint32_t s_scan[33];
+    __shared__ uint32_t s_flag;
+    const uint32_t n_staged = s.n_staged, T = s.threshold;
+    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
+    uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
+    uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
+    float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+    const int lane = threadIdx.x & 31;
+    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+         base += gridDim.x * (4 * BLOCK)) {
+        deco_pair prs[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint32_t q = base + r * BLOCK + threadIdx.x;
+            prs[r].idx = 0;
+            prs[r].val = __uint_as_float(0x7FFFFFFFu);       // above any threshold: no action
+            if (q < n_staged) prs[r] = src[q];
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            // neighbours in the staging area mostly belong to the same tile: lanes with the
+            // same (tile, class) elect one of them to add the group's size
+            const uint32_t key = mag_key(prs[r].val);
+            const uint32_t tile = prs[r].idx / TILE;
+            const bool in = base + r * BLOCK + threadIdx.x < n_staged;
+            const uint32_t cls = !in ? 0u : (key < T ? 1u : (key == T ? 2u : 0u));
+            const uint32_t grp = __match_any_sync(FULL, cls ? (tile * 2 + cls - 1) : 0xFFFFFFFFu);
+            if (cls && lane == __ffs(grp) - 1)
+                atomicAdd(cls == 1 ? &rej[tile] : &eqc[tile], static_cast<uint32_t>(__popc(grp)));
+        }
+    }
+    const bool last = last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 2], &s_flag);
+    // after the arrival, off the critical path: undo the +0 guess for the rejected entries
     auto write_back_rejected = [&]() {
         for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
              base += gridDim.x * (4 * BLOCK)) {
@@ -744,7 +777,7 @@ stage_select_kernel(Sel p)
                 const uint32_t q = base + r * BLOCK + threadIdx.x;
                 if (q < n_staged) {
                     const deco_pair pr = src[q];
-                    if (rel_bin_a(mag_key(pr.val), spec, shift) < a_sel) erow[pr.idx] = pr.val;
+                    if (mag_key(pr.val) < T) erow[pr.idx] = pr.val;
                 }
             }
         }
@@ -753,81 +786,101 @@ stage_select_kernel(Sel p)
         write_back_rejected();
         return;
     }
-
-    uint32_t bin, above;
-    pick_bin(hist_of(p, i, 0, 1), k_rem, s_scan, s_misc, bin, above);
-    if (bin == 0xFFFFFFFFu) {                       // counts do not add up: report, stay safe
-        if (threadIdx.x == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x120u, i);
-        return;
+    // chunk walk (one CTA): per thread a contiguous range of chunks; the sums of a chunk
+    // come from its CHUNK_TILES tiles (one cache line per array)
+    uint32_t *ccnt = p.chunk_cnt + static_cast<size_t>(i) * p.nchunks;
+    uint32_t *crej = p.chunk_rej + static_cast<size_t>(i) * p.nchunks;
+    uint32_t *ceq = p.chunk_eq + static_cast<size_t>(i) * p.nchunks;
+    uint32_t *cstart = p.chunk_start + static_cast<size_t>(i) * (p.nchunks + 1);
+    uint32_t *ceqb = p.chunk_eqb + static_cast<size_t>(i) * p.nchunks;
+    const uint32_t *tcnt = p.tile_cnt + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t ties = s.ties_take;
+    const uint32_t per = (p.nchunks + BLOCK - 1) / BLOCK;
+    const uint32_t lo = min(p.nchunks, threadIdx.x * per), hi = min(p.nchunks, lo + per);
+    uint32_t eq_sum = 0;
+    for (uint32_t c = lo; c < hi; ++c) {
+        uint32_t a = 0, b = 0, q = 0;
+        const uint32_t t0 = c * CHUNK_TILES, t1 = min(p.ntiles, t0 + CHUNK_TILES);
+        for (uint32_t t = t0; t < t1; ++t) {
+            a += tcnt[t];
+            b += __ldcg(&rej[t]);
+            q += __ldcg(&eqc[t]);
+        }
+        ccnt[c] = a;
+        crej[c] = b;
+        ceq[c] = q;
+        eq_sum += q;
     }
-    const uint32_t T = spec + (a_sel << shift) + bin;
+    uint32_t eq_total;
+    uint32_t eq_before = block_excl_scan(eq_sum, s_scan, eq_total);
+    uint32_t sel_sum = 0;
+    for (uint32_t c = lo; c < hi; ++c) {
+        const uint32_t q = ceq[c];
+        const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
+        ceqb[c] = eq_before;
+        sel_sum += ccnt[c] - crej[c] - q + min(q, left);
+        eq_before += q;
+    }
+    uint32_t sel_total;
+    uint32_t pos = block_excl_scan(sel_sum, s_scan, sel_total);
+    for (uint32_t c = lo; c < hi; ++c) {
+        const uint32_t q = ceq[c];
+        const uint32_t eb = ceqb[c];
+        const uint32_t left = ties > eb ? ties - eb : 0u;
+        cstart[c] = pos;
+        pos += ccnt[c] - crej[c] - q + min(q, left);
+    }
     if (threadIdx.x == 0) {
-        s.prefix = (a_sel << shift) | bin;
-        s.k_rem = k_rem - above;
-        s.threshold = T;
-        s.n_greater = above_a + above;
-        s.ties_take = k_rem - above;
+        cstart[p.nchunks] = sel_total;
+        if (sel_total != p.k) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x200u, i);
     }
-    const uint32_t nb = __ldcg(&s.n_boundary);
-    if (nb <= BOUNDARY_CAP) {
-        for (uint32_t q0 = 0; q0 < nb; q0 += 4 * BLOCK) {
-            // written by other CTAs of this launch: read through L2; four loads in flight
-            uint2 raw[4];
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const uint32_t q = q0 + r * BLOCK + threadIdx.x;
-                raw[r] = make_uint2(0u, 0xFFFFFFFFu);
-                if (q < nb) raw[r] = __ldcg(reinterpret_cast<const uint2 *>(bnd) + q);
-            }
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                if (q0 + r * BLOCK + threadIdx.x >= nb) continue;
-                const uint32_t key = raw[r].y & 0x7FFFFFFFu;
-                if (key < T) {
-                    atomicAdd(&rej[raw[r].x / TILE], 1u);
-                    erow[raw[r].x] = __uint_as_float(raw[r].y);
-                } else if (key == T) {
-                    atomicAdd(&eqc[raw[r].x / TILE], 1u);
-                }
-            }
-        }
-    } else {                                        // list overflowed: walk all staged entries
-        for (uint32_t q = threadIdx.x; q < n_staged; q += BLOCK) {
-            const deco_pair pr = src[q];
-            const uint32_t key = mag_key(pr.val);
-            if (rel_bin_a(key, spec, shift) != a_sel) continue;
-            if (key < T) {
-                atomicAdd(&rej[pr.idx / TILE], 1u);
-                erow[pr.idx] = pr.val;
-            } else if (key == T) {
-                atomicAdd(&eqc[pr.idx / TILE], 1u);
-            }
-        }
-    }
-    __threadfence();
-    __syncthreads();
-    scan_tiles_body(p, i, s_scan, true);
     write_back_rejected();
 }
 
-// One warp per tile: ordered filter of the tile's staged pairs into the message.  The selected
-// entries are already +0 in e; ties that are not taken get their value back.
-__global__ void __launch_bounds__(BLOCK)
-emit_stage_kernel(Sel p)
+// What a warp learns about the CHUNK_TILES tiles of one chunk from three coalesced loads and
+// two warp scans: lane l holds tile chunk*32 + l.
+struct TileInfo {
+    uint32_t cnt;     // staged entries of the tile
+    uint32_t take;    // ties of the tile that are taken
+    uint32_t sel;     // entries of the tile that go into the message
+    uint32_t start;   // message position of the tile's first entry
+};
+
+__device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint32_t chunk)
 {
-    const uint32_t i = blockIdx.y;
-    if (p.sel[i].exact) return;
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t tile = blockIdx.x * WARPS + w;
-    if (tile >= p.ntiles) return;
+    const int lane = threadIdx.x & 31;
+    const uint32_t tile = chunk * CHUNK_TILES + lane;
     const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
-    const uint32_t cnt = p.tile_cnt[ti];
-    if (cnt == 0) return;
-    const uint32_t start = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile];
-    const uint32_t want = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile + 1] - start;
-    const uint32_t T = p.sel[i].threshold;
-    const uint32_t take = p.tile_take[ti];
-    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + p.tile_off[ti];
+    uint32_t cnt = 0, rej = 0, eq = 0;
+    if (tile < p.ntiles) {
+        cnt = p.tile_cnt[ti];
+        rej = p.tile_rej[ti];
+        eq = p.tile_eq[ti];
+    }
+    const uint32_t ties = p.sel[i].ties_take;
+    const uint32_t eqb0 = p.chunk_eqb[static_cast<size_t>(i) * p.nchunks + chunk];
+    const uint32_t start0 = p.chunk_start[static_cast<size_t>(i) * (p.nchunks + 1) + chunk];
+    const uint32_t eq_before = eqb0 + warp_incl_scan(eq) - eq;
+    const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
+    TileInfo t;
+    t.cnt = cnt;
+    t.take = min(eq, left);
+    t.sel = cnt - rej - eq + t.take;
+    t.start = start0 + warp_incl_scan(t.sel) - t.sel;
+    // the directory the aggregation reads: message position of every tile
+    if (tile < p.ntiles) p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile] = t.start;
+    if (tile == p.ntiles - 1) p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + p.ntiles] = t.start + t.sel;
+    return t;
+}
+
+// The whole warp filters one tile's staged segment, in order, into the message.  The selected
+// entries are already +0 in e; ties that are not taken get their value back.
+__device__ __forceinline__ void emit_segment_warp(const Sel &p, uint32_t i, uint32_t tile,
+                                                  uint32_t off, uint32_t cnt, uint32_t start,
+                                                  uint32_t want, uint32_t take, uint32_t T)
+{
+    const int lane = threadIdx.x & 31;
+    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
     deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
     float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     uint32_t written = 0, ties_seen = 0;
@@ -867,6 +920,74 @@ emit_stage_kernel(Sel p)
         }
     }
     if (lane == 0 && written != want) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x311u, tile);
+}
+
+// Emit, many staged entries per tile: one warp per tile.
+__global__ void __launch_bounds__(BLOCK)
+emit_stage_tile_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.y;
+    if (p.sel[i].exact) return;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t tile = blockIdx.x * WARPS + w;
+    if (tile >= p.ntiles) return;
+    const uint32_t my = tile % CHUNK_TILES;
+    const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
+    if (my != 0 && p.tile_cnt[ti] == 0) return;               // lane-0 warps write the directory
+    const TileInfo t = chunk_header(p, i, tile / CHUNK_TILES);
+    const uint32_t cnt = __shfl_sync(FULL, t.cnt, my);
+    if (cnt == 0) return;
+    const uint32_t start = __shfl_sync(FULL, t.start, my), want = __shfl_sync(FULL, t.sel, my);
+    const uint32_t take = __shfl_sync(FULL, t.take, my);
+    (void)lane;
+    emit_segment_warp(p, i, tile, p.tile_off[ti], cnt, start, want, take, p.sel[i].threshold);
+}
+
+// Emit, few staged entries per tile: one warp per chunk, each lane walks its own tile's few
+// entries; a tile with many entries is done by the whole warp.
+__global__ void __launch_bounds__(BLOCK)
+emit_stage_chunk_kernel(Sel p)
+{
+    constexpr uint32_t LANE_MAX = 16;
+    const uint32_t i = blockIdx.y;
+    if (p.sel[i].exact) return;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t chunk = blockIdx.x * WARPS + w;
+    if (chunk >= p.nchunks) return;
+    const TileInfo t = chunk_header(p, i, chunk);
+    const uint32_t tile = chunk * CHUNK_TILES + lane;
+    const uint32_t T = p.sel[i].threshold;
+    uint32_t off = 0;
+    if (t.cnt) off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
+    if (t.cnt && t.cnt <= LANE_MAX) {
+        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
+        deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
+        float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+        uint32_t written = 0, ties_seen = 0;
+        for (uint32_t q = 0; q < t.cnt; ++q) {
+            const deco_pair pr = src[q];
+            const uint32_t key = mag_key(pr.val);
+            const bool eq = key == T;
+            const bool pick = key > T || (eq && ties_seen < t.take);
+            ties_seen += eq ? 1u : 0u;
+            if (pick) {
+                const uint32_t pos = t.start + written++;
+                if (pos < p.k && pr.idx < p.d) out[pos] = pr;
+                else latch(p.status, DECO_ERR_DEVICE_CHECK, 0x312u, tile);
+            } else if (eq && pr.idx < p.d) {
+                erow[pr.idx] = pr.val;                       // tie not taken: undo the guess
+            }
+        }
+        if (written != t.sel) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x313u, tile);
+    }
+    uint32_t big = __ballot_sync(FULL, t.cnt > LANE_MAX);
+    while (big) {
+        const int b = __ffs(big) - 1;
+        big &= big - 1;
+        emit_segment_warp(p, i, chunk * CHUNK_TILES + b, __shfl_sync(FULL, off, b),
+                          __shfl_sync(FULL, t.cnt, b), __shfl_sync(FULL, t.start, b),
+                          __shfl_sync(FULL, t.sel, b), __shfl_sync(FULL, t.take, b), T);
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1236,7 +1357,12 @@ Sel make_sel(const deco_ctx *c)
     p.tile_off = c->tile_off;
     p.tile_cnt = c->tile_cnt;
     p.tile_rej = c->tile_rej;
-    p.boundary = c->boundary;
+    p.nchunks = c->nchunks;
+    p.chunk_cnt = c->chunk_cnt;
+    p.chunk_rej = c->chunk_rej;
+    p.chunk_eq = c->chunk_eq;
+    p.chunk_eqb = c->chunk_eqb;
+    p.chunk_start = c->chunk_start;
     p.msg = c->msg;
     p.k_cap = c->k_cap;
     p.stage = c->stage;
@@ -1337,11 +1463,19 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     }
     // staged pairs per worker are a few times k: size the grids for that
     dim3 sgrid(part_blocks(c, 2 * c->k + 65536, BLOCK * 4), c->n);
-    dim3 wgrid((c->ntiles + WARPS - 1) / WARPS, c->n);
     stage_hist_a_kernel<<<sgrid, BLOCK, 0, s>>>(p);
-    stage_select_kernel<<<sgrid, BLOCK, 0, s>>>(p);
-    emit_stage_kernel<<<wgrid, BLOCK, 0, s>>>(p);
-    c->launches += 3;
+    stage_hist_b_kernel<<<sgrid, BLOCK, 0, s>>>(p);
+    stage_classify_kernel<<<sgrid, BLOCK, 0, s>>>(p);
+    // about 1.3 k staged entries spread over ntiles tiles: a warp per tile when a tile holds
+    // many, a warp per chunk of tiles when it holds few
+    if (13 * c->k >= 240ull * c->ntiles) {
+        dim3 wgrid((c->ntiles + WARPS - 1) / WARPS, c->n);
+        emit_stage_tile_kernel<<<wgrid, BLOCK, 0, s>>>(p);
+    } else {
+        dim3 wgrid((c->nchunks + WARPS - 1) / WARPS, c->n);
+        emit_stage_chunk_kernel<<<wgrid, BLOCK, 0, s>>>(p);
+    }
+    c->launches += 4;
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     void *args[] = {&p};

@@ -35,7 +35,7 @@ struct SelectState {
     uint32_t spec_key;      // speculative lower bound used by the streaming pass (or DISABLED)
     uint32_t n_staged;      // candidates staged by the streaming pass
     uint32_t exact_total;   // cumulative count of steps that took the multi-pass path
-    uint32_t n_boundary;    // staged entries that fell into the threshold's coarse bin
+    uint32_t unused0;
     uint32_t rel_shift;     // log2 width of a coarse bin of the staged-key histogram (10..12)
     uint32_t pad[5];
 };
@@ -43,9 +43,9 @@ static_assert(sizeof(SelectState) == 64, "one line per worker");
 
 constexpr uint32_t SPEC_DISABLED = 0x80000000u;   // above every 31-bit key
 
-// Staged entries whose coarse bin is the threshold's are also appended to a short list so
-// that one CTA can settle them; if the list overflows that CTA walks all staged entries.
-constexpr uint32_t BOUNDARY_CAP = 8192;
+// Tiles are grouped into chunks of one warp's width; message positions are first fixed per
+// chunk (one CTA walks the chunks) and then per tile inside each chunk (one warp scan).
+constexpr uint32_t CHUNK_TILES = 32;
 
 // Keys of the per-iteration sample kept per worker (8192 groups of 4 entries).
 constexpr uint32_t SAMPLE_KEYS = 32768;
@@ -95,7 +95,12 @@ struct deco_ctx {
     uint32_t *tile_off = nullptr;       // [n][ntiles]  staging offset of each tile's candidates
     uint32_t *tile_cnt = nullptr;       // [n][ntiles]  staged candidates per tile
     uint32_t *tile_rej = nullptr;       // [n][ntiles]  staged candidates below the threshold
-    deco_pair *boundary = nullptr;      // [n][BOUNDARY_CAP] staged entries of the threshold's bin
+    uint32_t nchunks = 0;               // ceil(ntiles / CHUNK_TILES)
+    uint32_t *chunk_cnt = nullptr;      // [n][nchunks] staged candidates per chunk
+    uint32_t *chunk_rej = nullptr;      // [n][nchunks] rejected candidates per chunk
+    uint32_t *chunk_eq = nullptr;       // [n][nchunks] ties per chunk
+    uint32_t *chunk_eqb = nullptr;      // [n][nchunks] ties in earlier chunks
+    uint32_t *chunk_start = nullptr;    // [n][nchunks + 1] message position of each chunk
     uint32_t *dev_status = nullptr;     // [4]: status, two detail words, fallback flag
     void *grads_staging = nullptr;      // device copy of host gradients (deco_step_host)
     uint64_t device_bytes = 0;
