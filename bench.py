@@ -140,6 +140,12 @@ def grad_bytes(wl):
     return wl.n * wl.d * (4 if wl.grad_dtype == "f32" else 2)
 
 
+# DRAM read + write bytes of one ef_accumulate_kernel launch from the ncu capture summarised in
+# profiles/ef_accumulate_kernel_resnet18.md (taken on this kernel version); other workloads
+# were not captured.
+NCU_TRAFFIC_BYTES = {"resnet18": 1076.4e6}
+
+
 def algorithmic_bytes_accumulate(wl):
     """Streaming pass: read e (4), read g (4 or 2), write e (4) per entry and worker."""
     return wl.n * wl.d * (8 + (4 if wl.grad_dtype == "f32" else 2))
@@ -311,7 +317,8 @@ def run_ours(args):
     achieved = algorithmic_bytes_accumulate(wl) / (acc_ms * 1e-3) / 1e9 if acc_ms > 0 else None
     roofline = {"bound": "hbm", "kernel": "ef_accumulate_kernel", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "frac": (achieved / peak) if achieved else None,
+                "traffic": NCU_TRAFFIC_BYTES.get(wl.name) if (args.delta is None) else None,
                 "algorithmic_bytes_per_launch": algorithmic_bytes_accumulate(wl),
                 "avg_launch_ms": acc_ms, "launches_timed": iters}
     step_alg_bytes = algorithmic_bytes_accumulate(wl)
