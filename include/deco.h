@@ -187,6 +187,23 @@ deco_status deco_policy_select(double V_g_bits, double a_bar_bps, double b_s, do
                                uint32_t tau_cap, int32_t non_iid,
                                uint32_t *tau_out, double *delta_out);
 
+/*
+ * Look-up table of the implementation section ("Efficient Implementation of DeCo"): the
+ * bandwidth range [a_min, a_max] profiled during warm-up is cut into `points` linearly spaced
+ * sample bandwidths (the paper uses about 20) and DeCo is run once per sample for the measured
+ * latency b.  deco_lut_lookup returns the entry of the sample nearest to a_bar (the lower one
+ * on a tie) when a_min <= a_bar <= a_max, and falls back to deco_policy_select outside the
+ * range.  Both are pure host arithmetic; `lut` is a HOST array of `points` entries owned by
+ * the caller.  points >= 1, a_min <= a_max.
+ */
+typedef struct { double a_bps; double delta; uint32_t tau; uint32_t reserved; } deco_lut_entry;
+deco_status deco_lut_build(double V_g_bits, double a_min_bps, double a_max_bps, double b_s,
+                           double T_comp_s, uint32_t points, uint32_t tau_cap, int32_t non_iid,
+                           deco_lut_entry *lut);
+deco_status deco_lut_lookup(const deco_lut_entry *lut, uint32_t points, double a_bar_bps,
+                            double V_g_bits, double b_s, double T_comp_s, uint32_t tau_cap,
+                            int32_t non_iid, uint32_t *tau_out, double *delta_out);
+
 /* Theorem 3: T_avg ~ max{(T_comp + b + delta V_g/a_bar)/(tau+1), delta V_g/a_bar, T_comp}.
  * Returns a negative value for invalid arguments. */
 double deco_t_avg(double delta, uint32_t tau, double V_g_bits, double a_bar_bps, double b_s,

@@ -43,6 +43,11 @@ class deco_options(ctypes.Structure):
                 ("reserved", ctypes.c_uint32 * 8)]
 
 
+class deco_lut_entry(ctypes.Structure):
+    _fields_ = [("a_bps", ctypes.c_double), ("delta", ctypes.c_double),
+                ("tau", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+
 class deco_stats(ctypes.Structure):
     _fields_ = [("step", ctypes.c_uint64),
                 ("k", ctypes.c_uint64),
@@ -79,6 +84,10 @@ SIGNATURES = {
     "deco_set_policy": (_i32, [_vp, _f64, _u32]),
     "deco_set_lr": (_i32, [_vp, _f32]),
     "deco_policy_select": (_i32, [_f64, _f64, _f64, _f64, _u32, _i32, _P(_u32), _P(_f64)]),
+    "deco_lut_build": (_i32, [_f64, _f64, _f64, _f64, _f64, _u32, _u32, _i32,
+                              _P(deco_lut_entry)]),
+    "deco_lut_lookup": (_i32, [_P(deco_lut_entry), _u32, _f64, _f64, _f64, _f64, _u32, _i32,
+                               _P(_u32), _P(_f64)]),
     "deco_t_avg": (_f64, [_f64, _u32, _f64, _f64, _f64, _f64]),
     "deco_k_from_delta": (_u64, [_f64, _u64]),
     "deco_get_k": (_i32, [_vp, _P(_u64)]),
@@ -202,6 +211,24 @@ def deco_policy_select(V_g_bits, a_bar_bps, b_s, T_comp_s, tau_cap=0, non_iid=Fa
     _check(load().deco_policy_select(V_g_bits, a_bar_bps, b_s, T_comp_s, tau_cap,
                                      int(bool(non_iid)), ctypes.byref(tau),
                                      ctypes.byref(delta)), "deco_policy_select")
+    return tau.value, delta.value
+
+
+def deco_lut_build(V_g_bits, a_min_bps, a_max_bps, b_s, T_comp_s, points=20, tau_cap=0,
+                   non_iid=False):
+    """-> ctypes array of `points` deco_lut_entry (bandwidth sample, delta, tau)."""
+    lut = (deco_lut_entry * points)()
+    _check(load().deco_lut_build(V_g_bits, a_min_bps, a_max_bps, b_s, T_comp_s, points, tau_cap,
+                                 int(bool(non_iid)), lut), "deco_lut_build")
+    return lut
+
+
+def deco_lut_lookup(lut, a_bar_bps, V_g_bits, b_s, T_comp_s, tau_cap=0, non_iid=False):
+    """Nearest sample inside the profiled range, online DeCo outside -> (tau, delta)."""
+    tau, delta = _u32(), _f64()
+    _check(load().deco_lut_lookup(lut, len(lut), a_bar_bps, V_g_bits, b_s, T_comp_s, tau_cap,
+                                  int(bool(non_iid)), ctypes.byref(tau), ctypes.byref(delta)),
+           "deco_lut_lookup")
     return tau.value, delta.value
 
 

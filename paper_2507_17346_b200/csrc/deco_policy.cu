@@ -95,3 +95,45 @@ extern "C" uint64_t deco_k_from_delta(double delta, uint64_t d)
     if (k > d) k = d;
     return k;
 }
+
+extern "C" deco_status deco_lut_build(double Vg, double a_min, double a_max, double b, double Tc,
+                                      uint32_t points, uint32_t tau_cap, int32_t non_iid,
+                                      deco_lut_entry *lut)
+{
+    if (!lut || points == 0 || !(a_min > 0.0) || !(a_max >= a_min)) return DECO_ERR_INVALID_ARG;
+    for (uint32_t q = 0; q < points; ++q) {
+        const double a = points < 2 ? a_min
+                                    : a_min + (a_max - a_min) * static_cast<double>(q) /
+                                                  static_cast<double>(points - 1);
+        uint32_t tau = 0;
+        double delta = 0.0;
+        const deco_status st = deco_policy_select(Vg, a, b, Tc, tau_cap, non_iid, &tau, &delta);
+        if (st != DECO_OK) return st;
+        lut[q].a_bps = a;
+        lut[q].delta = delta;
+        lut[q].tau = tau;
+        lut[q].reserved = 0;
+    }
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_lut_lookup(const deco_lut_entry *lut, uint32_t points, double a_bar,
+                                       double Vg, double b, double Tc, uint32_t tau_cap,
+                                       int32_t non_iid, uint32_t *tau_out, double *delta_out)
+{
+    if (!lut || points == 0 || !tau_out || !delta_out || !(a_bar > 0.0)) return DECO_ERR_INVALID_ARG;
+    if (a_bar < lut[0].a_bps || a_bar > lut[points - 1].a_bps)     // outside the profiled range
+        return deco_policy_select(Vg, a_bar, b, Tc, tau_cap, non_iid, tau_out, delta_out);
+    uint32_t best = 0;
+    double best_dist = std::fabs(lut[0].a_bps - a_bar);
+    for (uint32_t q = 1; q < points; ++q) {
+        const double dist = std::fabs(lut[q].a_bps - a_bar);
+        if (dist < best_dist) {            // strict: the lower sample wins a tie
+            best = q;
+            best_dist = dist;
+        }
+    }
+    *tau_out = lut[best].tau;
+    *delta_out = lut[best].delta;
+    return DECO_OK;
+}

@@ -42,6 +42,7 @@ def test_every_declared_symbol_is_exported_and_bound(B):
 
 def test_struct_layouts_match_the_header(B):
     assert ctypes.sizeof(B.deco_pair) == 8
+    assert ctypes.sizeof(B.deco_lut_entry) == 24
     assert ctypes.sizeof(B.deco_options) == 4 + 4 + 8 + 4 + 4 + 8 + 4 + 4 + 32
     assert ctypes.sizeof(B.deco_stats) == 8 + 8 + 8 + 4 + 4 + 8 + 8 + 8
 
@@ -78,6 +79,26 @@ def test_policy_select_matches_oracle(B):
     assert tau == 4 and delta == P.delta_star(4, 3.2e9, 0.1e9, 0.2, 0.05)
     with pytest.raises(B.DecoError):
         B.deco_policy_select(0.0, 1e9, 0.1, 0.05)
+
+
+def test_lut_matches_oracle(B):
+    import random
+    Vg, b, Tc = 3.2e9, 0.1, 0.05
+    lut = B.deco_lut_build(Vg, 0.5e9, 2.0e9, b, Tc, points=20)
+    want = P.build_lut(Vg, 0.5e9, 2.0e9, b, Tc, points=20)
+    assert len(lut) == 20
+    for got, (a, tau, delta) in zip(lut, want):
+        assert got.a_bps == pytest.approx(a, rel=1e-15) and got.tau == tau
+        assert got.delta == pytest.approx(delta, rel=1e-12)
+    rnd = random.Random(3)
+    for _ in range(500):
+        a = 10 ** rnd.uniform(8.3, 9.6)              # inside and outside [0.5, 2] Gbps
+        assert B.deco_lut_lookup(lut, a, Vg, b, Tc) == \
+            pytest.approx(P.lut_lookup(want, a, Vg, b, Tc), rel=1e-12)
+    one = B.deco_lut_build(Vg, 1e9, 1e9, b, Tc, points=1)
+    assert (one[0].tau, one[0].delta) == P.deco_select(Vg, 1e9, b, Tc)
+    with pytest.raises(B.DecoError):
+        B.deco_lut_build(Vg, 2e9, 1e9, b, Tc, points=5)
 
 
 def test_init_without_a_device_fails_loudly(B):
