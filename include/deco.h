@@ -148,7 +148,10 @@ deco_status deco_aggregate_stale(deco_ctx *ctx, void *stream);
  */
 deco_status deco_apply_update(deco_ctx *ctx, void *stream);
 
-/* The three calls above in order, for callers that do not interleave other work. */
+/* The three calls above for callers that do not interleave other work.  With tau >= 1 the
+ * update of the aggregates that are due runs on an internal stream concurrently with the
+ * worker side (it depends on neither); that stream is forked from and joined back into
+ * `stream` inside the call, so the caller sees plain stream order. */
 deco_status deco_step(deco_ctx *ctx, const void *grads /* DEVICE */, void *stream);
 
 /*

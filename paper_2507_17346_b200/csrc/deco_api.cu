@@ -66,6 +66,9 @@ void free_all(deco_ctx *c)
     cudaFree(c->grads_staging);
     for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
     c->events.clear();
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side_stream) cudaStreamDestroy(c->side_stream);
 }
 
 deco_status zero_state(deco_ctx *c, cudaStream_t s)
@@ -211,6 +214,11 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->chunk_start, static_cast<uint64_t>(n) * (c->nchunks + 1)));
     need(dev_alloc(c, &c->dev_status, 4));
     if (st == DECO_OK && query_fallback_grid(c) != cudaSuccess) st = DECO_ERR_CUDA;
+    if (st == DECO_OK &&
+        (cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+         cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
+        st = DECO_ERR_CUDA;
     if (st == DECO_OK) st = zero_state(c, nullptr);
     if (st == DECO_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = DECO_ERR_CUDA;
     if (st != DECO_OK) {
@@ -280,32 +288,48 @@ extern "C" deco_status deco_aggregate_stale(deco_ctx *c, void *stream)
     return DECO_OK;
 }
 
+namespace {
+
+// Launch the update for every cached aggregate that is due at iteration t (step <= t - tau),
+// oldest first, on stream s.
+deco_status apply_due(deco_ctx *c, cudaStream_t s)
+{
+    const float beta = c->lr_at_server ? c->lr : 1.0f;
+    const float neg_scale = -(beta / static_cast<float>(c->n));
+    if (c->t < c->tau) return DECO_OK;
+    const uint64_t due = c->t - c->tau;
+    // step ids still cached lie in (t - ring, t]
+    const uint64_t lo = c->t + 1 >= c->ring ? c->t + 1 - c->ring : 0;
+    for (uint64_t step = lo; step <= due; ++step) {
+        Slot &sl = c->slot_info[step % c->ring];
+        if (!sl.valid || sl.step != step) continue;
+        const deco_pair *slot = c->slots + (step % c->ring) * c->n * c->k_cap;
+        if (launch_apply(c, slot, sl.positions, neg_scale, s) != cudaSuccess) return DECO_ERR_CUDA;
+        sl.valid = false;
+    }
+    return DECO_OK;
+}
+
+void finish_iteration(deco_ctx *c)
+{
+    if (c->timing && c->timed_iters < MAX_TIMED_ITERS) c->timed_iters += 1;
+    c->t += 1;
+    c->phase = 0;
+}
+
+}  // namespace
+
 extern "C" deco_status deco_apply_update(deco_ctx *c, void *stream)
 {
     if (!c) return DECO_ERR_INVALID_ARG;
     if (c->phase != 2) return DECO_ERR_STATE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
-    const float beta = c->lr_at_server ? c->lr : 1.0f;
-    const float neg_scale = -(beta / static_cast<float>(c->n));
     mark(c, 5, as_stream(stream));
-    if (c->t >= c->tau) {
-        const uint64_t due = c->t - c->tau;
-        // oldest first: step ids still cached lie in (t - ring, t]
-        const uint64_t lo = c->t + 1 >= c->ring ? c->t + 1 - c->ring : 0;
-        for (uint64_t s = lo; s <= due; ++s) {
-            Slot &sl = c->slot_info[s % c->ring];
-            if (!sl.valid || sl.step != s) continue;
-            const deco_pair *slot = c->slots + (s % c->ring) * c->n * c->k_cap;
-            if (launch_apply(c, slot, sl.positions, neg_scale, as_stream(stream)) != cudaSuccess)
-                return DECO_ERR_CUDA;
-            sl.valid = false;
-        }
-    }
+    const deco_status st = apply_due(c, as_stream(stream));
+    if (st != DECO_OK) return st;
     mark(c, 6, as_stream(stream));
-    if (c->timing && c->timed_iters < MAX_TIMED_ITERS) c->timed_iters += 1;
-    c->t += 1;
-    c->phase = 0;
+    finish_iteration(c);
     return DECO_OK;
 }
 
@@ -343,10 +367,35 @@ extern "C" deco_status deco_get_kernel_timing(deco_ctx *c, void *stream, double 
 
 extern "C" deco_status deco_step(deco_ctx *c, const void *grads, void *stream)
 {
-    deco_status st = deco_ef_compress(c, grads, stream);
+    if (!c || !grads) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    if (c->tau == 0 || !c->side_stream) {
+        // the update of this iteration needs this iteration's aggregate: strictly in order
+        deco_status st = deco_ef_compress(c, grads, stream);
+        if (st == DECO_OK) st = deco_aggregate_stale(c, stream);
+        if (st == DECO_OK) st = deco_apply_update(c, stream);
+        return st;
+    }
+    // tau >= 1: the aggregates due now were cached in earlier iterations and touch neither e
+    // nor the messages, so their update runs on an internal stream next to the streaming
+    // pass.  It is forked from and joined back into the caller's stream inside this call:
+    // everything is complete, in stream order, when the caller's stream passes the call.
+    if (reinterpret_cast<uintptr_t>(grads) & 15u) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    cudaStream_t s = as_stream(stream);
+    if (cudaEventRecord(c->ev_fork, s) != cudaSuccess) return DECO_ERR_CUDA;
+    if (cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0) != cudaSuccess) return DECO_ERR_CUDA;
+    mark(c, 5, c->side_stream);
+    deco_status st = apply_due(c, c->side_stream);
+    mark(c, 6, c->side_stream);
+    if (cudaEventRecord(c->ev_join, c->side_stream) != cudaSuccess) return DECO_ERR_CUDA;
+    if (st == DECO_OK) st = deco_ef_compress(c, grads, stream);
     if (st == DECO_OK) st = deco_aggregate_stale(c, stream);
-    if (st == DECO_OK) st = deco_apply_update(c, stream);
-    return st;
+    if (cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) return DECO_ERR_CUDA;
+    if (st != DECO_OK) return st;
+    finish_iteration(c);
+    return DECO_OK;
 }
 
 extern "C" deco_status deco_step_host(deco_ctx *c, const void *grads_host, deco_pair *msg_out,

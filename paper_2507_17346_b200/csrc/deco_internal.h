@@ -110,6 +110,9 @@ struct deco_ctx {
     std::vector<deco::Slot> slot_info;
     uint64_t launches = 0;
     uint64_t k_of_msg = 0;              // k used by the last compress
+    // internal stream of deco_step: the stale update runs next to the streaming pass
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // optional event timing: 8 events per recorded iteration
     bool timing = false;
     std::vector<cudaEvent_t> events;
