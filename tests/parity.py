@@ -106,7 +106,8 @@ def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mo
                 terms = np.zeros(d)
                 for s, v in ref["msgs"]:
                     terms[s] += np.abs(v.astype(np.float64))
-                assert close(aval, ref["S64"][touched], terms[touched] / n, rtol)
+                assert close(aval, ref["S64"][touched], terms[touched], rtol), \
+                    "step %d: aggregate vs float64" % t
                 assert np.array_equal(bits(aval), bits(ref["S"][touched])), \
                     "step %d: aggregate not the worker-order fp32 sum" % t
             B.deco_apply_update(ctx)

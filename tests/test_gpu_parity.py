@@ -145,6 +145,18 @@ def test_adaptive_policy_run():
                policy_plan=plan, tau_max=tau_max, delta_max=delta_max, check_every=3)
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_many_workers_and_odd_length(mode):
+    """More workers than the aggregation keeps in registers at once, rows that are not
+    16-byte aligned, a vector that ends in the middle of a tile."""
+    d, n = 50_001, 20
+    for dtype, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        run_parity(d, n, 0.02, 2, 0.1, lambda t: _values("normal", n, d, t, dtype), steps=5,
+                   grad_dtype=name, select_mode=mode)
+    run_parity(d, n, 0.5, 1, 0.1, lambda t: _values("coarse", n, d, t, torch.float32), steps=3,
+               select_mode=mode)
+
+
 def test_call_order_and_capacity_errors():
     d, n = 10_000, 2
     ctx = B.deco_init(d, n, 0.01, 1, 0.1, tau_max=2, delta_max=0.05)
