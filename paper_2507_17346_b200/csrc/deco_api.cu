@@ -79,7 +79,7 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
     if (err == cudaSuccess) err = cudaMemsetAsync(c->sel, 0, sizeof(SelectState) * c->n, s);
     if (err == cudaSuccess) err = cudaMemsetAsync(c->dev_status, 0, sizeof(uint32_t) * 4, s);
     if (err == cudaSuccess)
-        err = cudaMemsetAsync(c->done, 0, sizeof(uint32_t) * c->n * (RADIX_LEVELS + 1), s);
+        err = cudaMemsetAsync(c->done, 0, sizeof(uint32_t) * c->n * DONE_SLOTS, s);
     if (err == cudaSuccess)
         err = cudaMemsetAsync(c->sample_hist, 0, sizeof(uint32_t) * c->n * 1024, s);
     if (err == cudaSuccess)
@@ -196,7 +196,7 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * n * c->k_cap));
     need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
     need(dev_alloc(c, &c->hist, static_cast<uint64_t>(n) * 2 * RADIX_LEVELS * RADIX_BINS));
-    need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * (RADIX_LEVELS + 1)));
+    need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * DONE_SLOTS));
     need(dev_alloc(c, &c->sample_keys, static_cast<uint64_t>(n) * SAMPLE_KEYS));
     need(dev_alloc(c, &c->sample_hist, static_cast<uint64_t>(n) * 1024));
     need(dev_alloc(c, &c->sel, n));

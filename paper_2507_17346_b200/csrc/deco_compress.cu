@@ -44,7 +44,7 @@ struct Sel {
     uint32_t k;
     SelectState *sel;
     uint32_t *hist;          // [n][2][RADIX_LEVELS][RADIX_BINS]: 0 = staged route, 1 = multi-pass
-    uint32_t *done;          // [n][RADIX_LEVELS + 1] CTA arrival counters
+    uint32_t *done;          // [n][DONE_SLOTS] CTA arrival counters
     uint32_t *sample_keys;   // [n][4 * SAMPLE_CHUNKS] keys of the sample
     uint32_t *sample_hist;   // [n][1024] sample keys per top-10-bit bin; cleared by its reader
     uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt, *tile_rej;
@@ -276,7 +276,8 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
          q += SAMPLE_CTAS * BEGIN_BLOCK)
         hz[q] = 0;
     if (part == 0) {
-        if (t < RADIX_LEVELS) p.done[i * (RADIX_LEVELS + 1) + t] = 0;
+        if (t < 3) p.done[i * DONE_SLOTS + t] = 0;          // levels A, B, classification
+        if (t == 4) p.done[i * DONE_SLOTS + 4] = 0;         // chunk sums
         if (i == 0 && t == 0) p.status[3] = exact_all;
         if (t == 0) {
             s.prefix = 0;
@@ -330,7 +331,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         if (s_exp[t]) atomicAdd(&p.sample_hist[i * SAMPLE_HIST_BINS + t], s_exp[t]);
     }
     // the arrival counter resets itself: only the last CTA touches it afterwards
-    uint32_t *arrive = &p.done[i * (RADIX_LEVELS + 1) + RADIX_LEVELS];
+    uint32_t *arrive = &p.done[i * DONE_SLOTS + 3];
     if (!last_cta_to_arrive(arrive, &s_flag)) return;
     if (t == 0) *arrive = 0;
 
@@ -654,7 +655,7 @@ stage_hist_a_kernel(Sel p)
         for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
             if (h[b]) atomicAdd(&out[b], h[b]);
     }
-    if (!last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 0], &s_misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 0], &s_misc[2])) return;
     uint32_t a_sel = REL_TOP, above_a = 0;
     if (valid) pick_bin(hist_of(p, i, 0, 0), p.k, s_scan, s_misc, a_sel, above_a);
     if (threadIdx.x == 0) {
@@ -706,7 +707,7 @@ stage_hist_b_kernel(Sel p)
     uint32_t *out = hist_of(p, i, 0, 1);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
         if (h[b]) atomicAdd(&out[b], h[b]);
-    if (!last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 1], &s_misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 1], &s_misc[2])) return;
     uint32_t bin, above;
     pick_bin(hist_of(p, i, 0, 1), k_rem, s_scan, s_misc, bin, above);
     if (threadIdx.x == 0) {
@@ -724,14 +725,111 @@ stage_hist_b_kernel(Sel p)
     }
 }
 
+// One CTA: ties are granted to chunks in index order until ties_take are used up, then every
+// chunk gets its position in the message.  Per thread a contiguous range of chunks.  With
+// sums_ready the per-chunk sums were left in chunk_cnt/rej/eq by chunk_sums_kernel; otherwise
+// (few chunks) they are taken here from the CHUNK_TILES tile counters of each chunk.
+__device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, bool sums_ready)
+{
+    uint32_t *ccnt = p.chunk_cnt + static_cast<size_t>(i) * p.nchunks;
+    uint32_t *crej = p.chunk_rej + static_cast<size_t>(i) * p.nchunks;
+    uint32_t *ceq = p.chunk_eq + static_cast<size_t>(i) * p.nchunks;
+    uint32_t *cstart = p.chunk_start + static_cast<size_t>(i) * (p.nchunks + 1);
+    uint32_t *ceqb = p.chunk_eqb + static_cast<size_t>(i) * p.nchunks;
+    const uint32_t *tcnt = p.tile_cnt + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
+    const uint32_t ties = p.sel[i].ties_take;
+    const uint32_t per = (p.nchunks + blockDim.x - 1) / blockDim.x;
+    const uint32_t lo = min(p.nchunks, threadIdx.x * per), hi = min(p.nchunks, lo + per);
+    uint32_t eq_sum = 0;
+    for (uint32_t c = lo; c < hi; ++c) {
+        uint32_t q;
+        if (sums_ready) {
+            q = __ldcg(&ceq[c]);
+        } else {
+            uint32_t a = 0, b = 0;
+            q = 0;
+            const uint32_t t0 = c * CHUNK_TILES, t1 = min(p.ntiles, t0 + CHUNK_TILES);
+            for (uint32_t t = t0; t < t1; ++t) {
+                a += tcnt[t];
+                b += __ldcg(&rej[t]);
+                q += __ldcg(&eqc[t]);
+            }
+            ccnt[c] = a;
+            crej[c] = b;
+            ceq[c] = q;
+        }
+        eq_sum += q;
+    }
+    uint32_t eq_total;
+    uint32_t eq_before = block_excl_scan(eq_sum, s_scan, eq_total);
+    uint32_t sel_sum = 0;
+    for (uint32_t c = lo; c < hi; ++c) {
+        const uint32_t q = __ldcg(&ceq[c]);
+        const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
+        ceqb[c] = eq_before;
+        sel_sum += __ldcg(&ccnt[c]) - __ldcg(&crej[c]) - q + min(q, left);
+        eq_before += q;
+    }
+    uint32_t sel_total;
+    uint32_t pos = block_excl_scan(sel_sum, s_scan, sel_total);
+    for (uint32_t c = lo; c < hi; ++c) {
+        const uint32_t q = __ldcg(&ceq[c]);
+        const uint32_t eb = ceqb[c];
+        const uint32_t left = ties > eb ? ties - eb : 0u;
+        cstart[c] = pos;
+        pos += __ldcg(&ccnt[c]) - __ldcg(&crej[c]) - q + min(q, left);
+    }
+    if (threadIdx.x == 0) {
+        cstart[p.nchunks] = sel_total;
+        if (sel_total != p.k) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x200u, i);
+    }
+    __syncthreads();
+}
+
+// Many chunks: their sums are taken in parallel, one warp per chunk (three coalesced loads
+// and a warp reduction), and the last CTA of a worker to arrive walks the chunks.
+__global__ void __launch_bounds__(BLOCK)
+chunk_sums_kernel(Sel p)
+{
+    const uint32_t i = blockIdx.y;
+    if (p.sel[i].exact) return;
+    __shared__ uint32_t s_scan[33];
+    __shared__ uint32_t s_flag;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t chunk = blockIdx.x * WARPS + w;
+    if (chunk < p.nchunks) {
+        const uint32_t tile = chunk * CHUNK_TILES + lane;
+        const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
+        uint32_t a = 0, b = 0, q = 0;
+        if (tile < p.ntiles) {
+            a = p.tile_cnt[ti];
+            b = p.tile_rej[ti];
+            q = p.tile_eq[ti];
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            a += __shfl_down_sync(FULL, a, o);
+            b += __shfl_down_sync(FULL, b, o);
+            q += __shfl_down_sync(FULL, q, o);
+        }
+        if (lane == 0) {
+            p.chunk_cnt[static_cast<size_t>(i) * p.nchunks + chunk] = a;
+            p.chunk_rej[static_cast<size_t>(i) * p.nchunks + chunk] = b;
+            p.chunk_eq[static_cast<size_t>(i) * p.nchunks + chunk] = q;
+        }
+    }
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 4], &s_flag)) return;
+    chunk_walk(p, i, s_scan, true);
+}
+
 // Classification.  With the threshold known every staged entry below it is rejected: counted
 // for its tile and its chunk (CHUNK_TILES consecutive tiles) and given its value back in e;
-// entries equal to it are counted as ties.  The last CTA of a worker to arrive then walks the
-// chunks once: ties are granted in index order until ties_take are used up and every chunk
-// gets its position in the message.  (The per-tile positions follow from these inside the
+// entries equal to it are counted as ties.  With few chunks (walk_here) the last CTA of a worker
+// to arrive then walks the chunks once; with many, chunk_sums_kernel follows.  (The per-tile positions follow from these inside the
 // emit kernel, so nothing here is serial in the number of tiles.)
 __global__ void __launch_bounds__(BLOCK)
-stage_classify_kernel(Sel p)
+stage_classify_kernel(Sel p, uint32_t walk_here)
 {
     const uint32_t i = blockIdx.y;
     const SelectState &s = p.sel[i];
@@ -767,7 +865,7 @@ stage_classify_kernel(Sel p)
                 atomicAdd(cls == 1 ? &rej[tile] : &eqc[tile], static_cast<uint32_t>(__popc(grp)));
         }
     }
-    const bool last = last_cta_to_arrive(&p.done[i * (RADIX_LEVELS + 1) + 2], &s_flag);
+    const bool last = last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &s_flag);
     // after the arrival, off the critical path: undo the +0 guess for the rejected entries
     auto write_back_rejected = [&]() {
         for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
@@ -786,54 +884,7 @@ stage_classify_kernel(Sel p)
         write_back_rejected();
         return;
     }
-    // chunk walk (one CTA): per thread a contiguous range of chunks; the sums of a chunk
-    // come from its CHUNK_TILES tiles (one cache line per array)
-    uint32_t *ccnt = p.chunk_cnt + static_cast<size_t>(i) * p.nchunks;
-    uint32_t *crej = p.chunk_rej + static_cast<size_t>(i) * p.nchunks;
-    uint32_t *ceq = p.chunk_eq + static_cast<size_t>(i) * p.nchunks;
-    uint32_t *cstart = p.chunk_start + static_cast<size_t>(i) * (p.nchunks + 1);
-    uint32_t *ceqb = p.chunk_eqb + static_cast<size_t>(i) * p.nchunks;
-    const uint32_t *tcnt = p.tile_cnt + static_cast<size_t>(i) * p.ntiles;
-    const uint32_t ties = s.ties_take;
-    const uint32_t per = (p.nchunks + BLOCK - 1) / BLOCK;
-    const uint32_t lo = min(p.nchunks, threadIdx.x * per), hi = min(p.nchunks, lo + per);
-    uint32_t eq_sum = 0;
-    for (uint32_t c = lo; c < hi; ++c) {
-        uint32_t a = 0, b = 0, q = 0;
-        const uint32_t t0 = c * CHUNK_TILES, t1 = min(p.ntiles, t0 + CHUNK_TILES);
-        for (uint32_t t = t0; t < t1; ++t) {
-            a += tcnt[t];
-            b += __ldcg(&rej[t]);
-            q += __ldcg(&eqc[t]);
-        }
-        ccnt[c] = a;
-        crej[c] = b;
-        ceq[c] = q;
-        eq_sum += q;
-    }
-    uint32_t eq_total;
-    uint32_t eq_before = block_excl_scan(eq_sum, s_scan, eq_total);
-    uint32_t sel_sum = 0;
-    for (uint32_t c = lo; c < hi; ++c) {
-        const uint32_t q = ceq[c];
-        const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
-        ceqb[c] = eq_before;
-        sel_sum += ccnt[c] - crej[c] - q + min(q, left);
-        eq_before += q;
-    }
-    uint32_t sel_total;
-    uint32_t pos = block_excl_scan(sel_sum, s_scan, sel_total);
-    for (uint32_t c = lo; c < hi; ++c) {
-        const uint32_t q = ceq[c];
-        const uint32_t eb = ceqb[c];
-        const uint32_t left = ties > eb ? ties - eb : 0u;
-        cstart[c] = pos;
-        pos += ccnt[c] - crej[c] - q + min(q, left);
-    }
-    if (threadIdx.x == 0) {
-        cstart[p.nchunks] = sel_total;
-        if (sel_total != p.k) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x200u, i);
-    }
+    if (walk_here) chunk_walk(p, i, s_scan, false);
     write_back_rejected();
 }
 
@@ -1465,7 +1516,13 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     dim3 sgrid(part_blocks(c, 2 * c->k + 65536, BLOCK * 4), c->n);
     stage_hist_a_kernel<<<sgrid, BLOCK, 0, s>>>(p);
     stage_hist_b_kernel<<<sgrid, BLOCK, 0, s>>>(p);
-    stage_classify_kernel<<<sgrid, BLOCK, 0, s>>>(p);
+    // the chunk walk is done by one CTA: with many chunks their sums are taken in parallel first
+    const bool walk_here = c->nchunks <= 256;
+    stage_classify_kernel<<<sgrid, BLOCK, 0, s>>>(p, walk_here ? 1u : 0u);
+    if (!walk_here) {
+        chunk_sums_kernel<<<dim3((c->nchunks + WARPS - 1) / WARPS, c->n), BLOCK, 0, s>>>(p);
+        c->launches += 1;
+    }
     // about 1.3 k staged entries spread over ntiles tiles: a warp per tile when a tile holds
     // many, a warp per chunk of tiles when it holds few
     if (13 * c->k >= 240ull * c->ntiles) {

@@ -24,6 +24,10 @@ constexpr int WARP_ELEMS = TILE / WARPS;   // 1024
 constexpr int RADIX_BINS = 4096;
 constexpr int RADIX_LEVELS = 3;
 
+// Arrival counters per worker: level A, level B, classification, sampling (resets itself),
+// chunk sums.
+constexpr int DONE_SLOTS = 5;
+
 // Per-worker selection record (device).  One 64-byte line per worker.
 struct SelectState {
     uint32_t prefix;        // key bits resolved so far (right-aligned)
@@ -83,7 +87,7 @@ struct deco_ctx {
     deco_pair *slots = nullptr;         // [ring][n * k_cap]
     deco_pair *stage = nullptr;         // [n][stage_cap]
     uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
-    uint32_t *done = nullptr;           // [n][RADIX_LEVELS + 1] CTA arrival counters
+    uint32_t *done = nullptr;           // [n][DONE_SLOTS] CTA arrival counters
     uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
     uint32_t *sample_hist = nullptr;    // [n][1024] sample keys per top-10-bit bin (self-clearing)
     uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
