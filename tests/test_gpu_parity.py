@@ -72,7 +72,7 @@ def test_resnet18_full_size():
     wl = W.make_workload("resnet18")
     assert wl.d == 11_689_512 and len(wl.tensors) == 62
     run_parity(wl.d, wl.n, wl.delta, wl.tau, wl.lr, lambda t: W.gradients(wl, t, "cuda"),
-               steps=6, grad_dtype=wl.grad_dtype)
+               steps=10, grad_dtype=wl.grad_dtype, check_every=2)
 
 
 @pytest.mark.parametrize("mode", MODES)
