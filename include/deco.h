@@ -246,6 +246,22 @@ deco_status deco_get_aggregate(deco_ctx *ctx, uint64_t step, const deco_pair **e
 deco_status deco_get_select_info(deco_ctx *ctx, void *stream, uint32_t *threshold_key,
                                  uint32_t *n_greater, uint32_t *exact_passes);
 
+/*
+ * Checkpoint / resume (no counterpart in the paper's algorithms; the state is exactly what
+ * Algorithm 1 carries between iterations): the iteration counter, gamma, (delta, tau), the
+ * error terms e, the parameters x and every cached aggregate with its step id.
+ *   deco_state_bytes   size of the blob for the current state
+ *   deco_export_state  waits for `stream`, then writes the blob to buf (HOST, `bytes` long)
+ *   deco_import_state  loads a blob into a context created with the same d, n, capacities
+ *                      and options (else DECO_ERR_INVALID_ARG); waits for `stream` before it
+ *                      returns.  Continuing from an imported state gives the same bits as
+ *                      continuing the run that exported it.
+ * All three may only be called between iterations.
+ */
+deco_status deco_state_bytes(const deco_ctx *ctx, uint64_t *bytes);
+deco_status deco_export_state(deco_ctx *ctx, void *buf, uint64_t bytes, void *stream);
+deco_status deco_import_state(deco_ctx *ctx, const void *buf, uint64_t bytes, void *stream);
+
 /* Waits for `stream`, then fills *out (HOST); returns DECO_ERR_DEVICE_CHECK if a kernel
  * latched an anomaly since the context was created or reset. */
 deco_status deco_get_stats(deco_ctx *ctx, void *stream, deco_stats *out);

@@ -97,6 +97,9 @@ SIGNATURES = {
     "deco_get_stats": (_i32, [_vp, _vp, _P(deco_stats)]),
     "deco_set_kernel_timing": (_i32, [_vp, _i32]),
     "deco_get_kernel_timing": (_i32, [_vp, _vp, _P(_f64), _P(_u64)]),
+    "deco_state_bytes": (_i32, [_vp, _P(_u64)]),
+    "deco_export_state": (_i32, [_vp, _vp, _u64, _vp]),
+    "deco_import_state": (_i32, [_vp, _vp, _u64, _vp]),
     "deco_launch_count": (_u64, [_vp]),
     "deco_topk_compress_static": (_i32, [_vp, _u64, _u64, _vp, _vp]),
     "deco_status_string": (ctypes.c_char_p, [_i32]),
@@ -290,6 +293,24 @@ def deco_get_kernel_timing(ctx, stream=None):
     _check(load().deco_get_kernel_timing(ctx, _stream(stream), ms, ctypes.byref(it)),
            "deco_get_kernel_timing")
     return dict(zip(("accumulate", "select", "aggregate", "apply"), list(ms))), it.value
+
+
+def deco_state_bytes(ctx):
+    n = _u64()
+    _check(load().deco_state_bytes(ctx, ctypes.byref(n)), "deco_state_bytes")
+    return n.value
+
+
+def deco_export_state(ctx, stream=None):
+    """-> bytes object holding the checkpoint of the context."""
+    n = deco_state_bytes(ctx)
+    buf = ctypes.create_string_buffer(n)
+    _check(load().deco_export_state(ctx, buf, n, _stream(stream)), "deco_export_state")
+    return buf.raw
+
+
+def deco_import_state(ctx, blob, stream=None):
+    _check(load().deco_import_state(ctx, blob, len(blob), _stream(stream)), "deco_import_state")
 
 
 def deco_launch_count(ctx):

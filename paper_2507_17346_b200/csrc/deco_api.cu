@@ -546,3 +546,139 @@ extern "C" deco_status deco_get_stats(deco_ctx *c, void *stream, deco_stats *out
 }
 
 extern "C" uint64_t deco_launch_count(const deco_ctx *c) { return c ? c->launches : 0; }
+
+// ------------------------------------------------------------------ checkpoint / resume
+namespace {
+
+struct StateHeader {
+    uint64_t magic, version;
+    uint64_t d, n, k_cap, ring, t, k;
+    double delta;
+    uint32_t tau, grad_dtype, lr_at_server, pad;
+    float lr;
+    uint32_t pad2;
+};
+constexpr uint64_t STATE_MAGIC = 0x4F434544534F4345ull;   // "ECOSDECO"
+
+struct SlotRecord {
+    uint64_t step, positions, valid;
+};
+
+uint64_t state_size(const deco_ctx *c)
+{
+    uint64_t bytes = sizeof(StateHeader) + sizeof(SlotRecord) * c->ring;
+    bytes += sizeof(float) * c->n * c->d + sizeof(float) * c->d;
+    for (const Slot &sl : c->slot_info)
+        if (sl.valid) bytes += sizeof(deco_pair) * sl.positions;
+    return bytes;
+}
+
+}  // namespace
+
+extern "C" deco_status deco_state_bytes(const deco_ctx *c, uint64_t *bytes)
+{
+    if (!c || !bytes) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    *bytes = state_size(c);
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_export_state(deco_ctx *c, void *buf, uint64_t bytes, void *stream)
+{
+    if (!c || !buf) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    if (bytes < state_size(c)) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    cudaStream_t s = as_stream(stream);
+    char *out = static_cast<char *>(buf);
+    StateHeader h;
+    std::memset(&h, 0, sizeof h);
+    h.magic = STATE_MAGIC;
+    h.version = 1;
+    h.d = c->d; h.n = c->n; h.k_cap = c->k_cap; h.ring = c->ring; h.t = c->t; h.k = c->k;
+    h.delta = c->delta; h.tau = c->tau; h.grad_dtype = c->grad_dtype;
+    h.lr_at_server = c->lr_at_server; h.lr = c->lr;
+    std::memcpy(out, &h, sizeof h);
+    out += sizeof h;
+    for (const Slot &sl : c->slot_info) {
+        SlotRecord r = {sl.step, sl.positions, sl.valid ? 1ull : 0ull};
+        std::memcpy(out, &r, sizeof r);
+        out += sizeof r;
+    }
+    // e without its padding, then the parameters, then the cached aggregates
+    if (cudaMemcpy2DAsync(out, sizeof(float) * c->d, c->e, sizeof(float) * c->e_stride,
+                          sizeof(float) * c->d, c->n, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    out += sizeof(float) * c->n * c->d;
+    if (cudaMemcpyAsync(out, c->params, sizeof(float) * c->d, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    out += sizeof(float) * c->d;
+    for (uint32_t q = 0; q < c->ring; ++q) {
+        const Slot &sl = c->slot_info[q];
+        if (!sl.valid) continue;
+        if (cudaMemcpyAsync(out, c->slots + static_cast<uint64_t>(q) * c->n * c->k_cap,
+                            sizeof(deco_pair) * sl.positions, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        out += sizeof(deco_pair) * sl.positions;
+    }
+    c->launches += 2 + c->ring;
+    return cudaStreamSynchronize(s) == cudaSuccess ? DECO_OK : DECO_ERR_CUDA;
+}
+
+extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t bytes, void *stream)
+{
+    if (!c || !buf || bytes < sizeof(StateHeader)) return DECO_ERR_INVALID_ARG;
+    if (c->phase != 0) return DECO_ERR_STATE;
+    const char *in = static_cast<const char *>(buf);
+    StateHeader h;
+    std::memcpy(&h, in, sizeof h);
+    in += sizeof h;
+    if (h.magic != STATE_MAGIC || h.version != 1 || h.d != c->d || h.n != c->n ||
+        h.k_cap != c->k_cap || h.ring != c->ring || h.grad_dtype != static_cast<uint32_t>(c->grad_dtype) ||
+        h.lr_at_server != static_cast<uint32_t>(c->lr_at_server) || h.tau > c->tau_max || h.k > c->k_cap)
+        return DECO_ERR_INVALID_ARG;
+    if (bytes < sizeof(StateHeader) + sizeof(SlotRecord) * c->ring) return DECO_ERR_INVALID_ARG;
+    std::vector<Slot> slots(c->ring);
+    uint64_t need = sizeof(StateHeader) + sizeof(SlotRecord) * c->ring +
+                    sizeof(float) * c->n * c->d + sizeof(float) * c->d;
+    for (uint32_t q = 0; q < c->ring; ++q) {
+        SlotRecord r;
+        std::memcpy(&r, in, sizeof r);
+        in += sizeof r;
+        if (r.valid && (r.positions > static_cast<uint64_t>(c->n) * c->k_cap || r.step % c->ring != q))
+            return DECO_ERR_INVALID_ARG;
+        slots[q].step = r.step;
+        slots[q].positions = r.positions;
+        slots[q].valid = r.valid != 0;
+        if (slots[q].valid) need += sizeof(deco_pair) * r.positions;
+    }
+    if (bytes < need) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    cudaStream_t s = as_stream(stream);
+    deco_status st = zero_state(c, s);                       // padding of e, status, counters
+    if (st != DECO_OK) return st;
+    if (cudaMemcpy2DAsync(c->e, sizeof(float) * c->e_stride, in, sizeof(float) * c->d,
+                          sizeof(float) * c->d, c->n, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    in += sizeof(float) * c->n * c->d;
+    if (cudaMemcpyAsync(c->params, in, sizeof(float) * c->d, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    in += sizeof(float) * c->d;
+    for (uint32_t q = 0; q < c->ring; ++q) {
+        if (!slots[q].valid) continue;
+        if (cudaMemcpyAsync(c->slots + static_cast<uint64_t>(q) * c->n * c->k_cap, in,
+                            sizeof(deco_pair) * slots[q].positions, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        in += sizeof(deco_pair) * slots[q].positions;
+    }
+    c->slot_info = slots;
+    c->t = h.t;
+    c->k = h.k;
+    c->delta = h.delta;
+    c->tau = h.tau;
+    c->lr = h.lr;
+    c->launches += 2 + c->ring;
+    return cudaStreamSynchronize(s) == cudaSuccess ? DECO_OK : DECO_ERR_CUDA;
+}

@@ -211,6 +211,45 @@ def test_two_runs_give_the_same_bits():
         assert torch.equal(a, b)
 
 
+def test_checkpoint_and_resume_give_the_same_bits():
+    wl = W.make_workload("gpt2_small", 0.08)
+    kw = dict(grad_dtype=B.DECO_BF16, tau_max=4, delta_max=0.01)
+    a = B.deco_init(wl.d, wl.n, wl.delta, 3, wl.lr, **kw)
+    b = B.deco_init(wl.d, wl.n, wl.delta, 3, wl.lr, **kw)
+    try:
+        for t in range(5):
+            if t == 3:
+                B.deco_set_policy(a, 0.004, 2)
+            B.deco_step(a, W.gradients(wl, t, "cuda"))
+        blob = B.deco_export_state(a)
+        assert len(blob) == B.deco_state_bytes(a)
+        B.deco_import_state(b, blob)
+        assert B.deco_get_stats(b)["step"] == 5 and B.deco_get_k(b) == B.deco_get_k(a)
+        assert B.deco_get_stats(b)["cached_aggregates"] == B.deco_get_stats(a)["cached_aggregates"]
+        for t in range(5, 10):
+            g = W.gradients(wl, t, "cuda")
+            B.deco_step(a, g)
+            B.deco_step(b, g)
+        torch.cuda.synchronize()
+        ba, bb = B.deco_get_buffers(a), B.deco_get_buffers(b)
+        k = B.deco_get_k(a)
+        for name, shape in (("e", (wl.n, ba["e_stride"])), ("params", (wl.d,))):
+            assert torch.equal(B.view_i32(ba[name], shape), B.view_i32(bb[name], shape)), name
+        assert torch.equal(B.view_i32(ba["msg"], (wl.n, ba["k_cap"], 2))[:, :k],
+                           B.view_i32(bb["msg"], (wl.n, bb["k_cap"], 2))[:, :k])
+        # a blob from another shape is refused
+        c = B.deco_init(wl.d + 8, wl.n, wl.delta, 3, wl.lr, **kw)
+        try:
+            with pytest.raises(B.DecoError) as e:
+                B.deco_import_state(c, blob)
+            assert e.value.status == B.DECO_ERR_INVALID_ARG
+        finally:
+            B.deco_destroy(c)
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
+
+
 def test_host_buffer_step_matches_device_step():
     wl = W.make_workload("resnet18", 0.25)
     k = B.deco_k_from_delta(wl.delta, wl.d)
