@@ -39,6 +39,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--delta", type=float, default=None)
     ap.add_argument("--tau", type=int, default=None)
+    ap.add_argument("--compressor", default="topk", choices=["topk", "randk"])
     return ap.parse_args()
 
 
@@ -246,7 +247,9 @@ def run_ours(args):
     mode = B.DECO_SELECT_AUTO if args.select_mode == "auto" else B.DECO_SELECT_EXACT_PASSES
     ctx = B.deco_init(wl.d, wl.n, wl.delta, wl.tau, wl.lr,
                       grad_dtype=B.DECO_F32 if wl.grad_dtype == "f32" else B.DECO_BF16,
-                      device=local, select_mode=mode)
+                      device=local, select_mode=mode,
+                      compressor=B.DECO_COMPRESSOR_RANDK if args.compressor == "randk"
+                      else B.DECO_COMPRESSOR_TOPK, seed=wl.seed)
     stream = torch.cuda.current_stream()
 
     for t in range(warmup):
@@ -318,7 +321,8 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "ef_accumulate_kernel", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
-                "traffic": NCU_TRAFFIC_BYTES.get(wl.name) if (args.delta is None) else None,
+                "traffic": NCU_TRAFFIC_BYTES.get(wl.name)
+                if (args.delta is None and args.compressor == "topk") else None,
                 "algorithmic_bytes_per_launch": algorithmic_bytes_accumulate(wl),
                 "avg_launch_ms": acc_ms, "launches_timed": iters}
     step_alg_bytes = algorithmic_bytes_accumulate(wl)
@@ -328,6 +332,7 @@ def run_ours(args):
             "config": {"workload": wl.name, "d": wl.d, "n": wl.n, "delta": wl.delta,
                        "tau": wl.tau, "lr": wl.lr, "grad_dtype": wl.grad_dtype,
                        "k": stats["k"], "select_mode": args.select_mode,
+                       "compressor": args.compressor,
                        "l2": "inputs larger than L2 (e and g of one step exceed 126 MB)"
                        if 2 * gbytes > 126e6 else "working set fits in L2",
                        "gradient_pool": pool_n, "replicas": world},

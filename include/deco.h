@@ -74,6 +74,16 @@ typedef enum {
     DECO_SELECT_EXACT_PASSES = 1 /* always the multi-pass radix selection (no sampling) */
 } deco_select_mode;
 
+/*
+ * The sparsifier C_delta.  Top-k is the paper's default; Random-k ("random k% of entries",
+ * the appendix on other compressors) keeps k entries chosen uniformly at random, independently
+ * per worker and iteration: entry j gets the priority  Philox4x32-10(key = seed,
+ * counter = (j / 4, t_lo, worker, t_hi ^ 0x52414E44))[j % 4] >> 9  and the k largest
+ * priorities are kept, equal ones by increasing index.  Error feedback, messages, aggregation
+ * and update are the same for both.
+ */
+typedef enum { DECO_COMPRESSOR_TOPK = 0, DECO_COMPRESSOR_RANDK = 1 } deco_compressor;
+
 /* Options of deco_init.  A zero-filled struct selects every default. */
 typedef struct {
     int32_t  grad_dtype;     /* deco_dtype of the gradients handed to deco_ef_compress; default F32 */
@@ -85,7 +95,10 @@ typedef struct {
                                 allocates a zero-filled vector and frees it in deco_destroy */
     int32_t  device;         /* CUDA device ordinal */
     int32_t  select_mode;    /* deco_select_mode */
-    uint32_t reserved[8];    /* must be zero */
+    int32_t  compressor;     /* deco_compressor; default Top-k */
+    uint32_t seed_lo;        /* Random-k: 64-bit seed of the priority stream, low word */
+    uint32_t seed_hi;        /*           high word */
+    uint32_t reserved[5];    /* must be zero */
 } deco_options;
 
 typedef struct {

@@ -84,9 +84,11 @@ def topk_select(a, k):
     return sel
 
 
-def compress(a, k):
-    """C_delta(a) as (indices ascending, values) and the residual a - C_delta(a)."""
-    sel = topk_select(a, k)
+def compress(a, k, sel=None):
+    """C_delta(a) as (indices ascending, values) and the residual a - C_delta(a).  `sel`
+    overrides the Top-k choice (Random-k passes its own index set)."""
+    if sel is None:
+        sel = topk_select(a, k)
     vals = a[sel].copy()
     resid = a.copy()
     resid[sel] = np.float32(0.0)
@@ -115,10 +117,13 @@ class DDEFSGD:
     lr_in_compress=True is the paper's form (a = e + gamma*g, update scale 1/n);
     False moves the stepsize to the server (a = e + g, update scale gamma/n)."""
 
-    def __init__(self, d, n, delta, tau, lr, x0=None, lr_in_compress=True):
+    def __init__(self, d, n, delta, tau, lr, x0=None, lr_in_compress=True, compressor="topk",
+                 seed=0):
         self.d, self.n = int(d), int(n)
         self.lr = np.float32(lr)
         self.lr_in_compress = bool(lr_in_compress)
+        assert compressor in ("topk", "randk")
+        self.compressor, self.seed = compressor, int(seed)
         self.delta, self.tau = float(delta), int(tau)
         self.k = k_from_delta(delta, d)
         self.x = (np.zeros(d, np.float32) if x0 is None
@@ -147,7 +152,11 @@ class DDEFSGD:
         msgs = []
         for i in range(n):                                # worker side
             a = accumulate(alpha, g[i], self.e[i])
-            sel, vals, resid = compress(a, self.k)
+            chosen = None
+            if self.compressor == "randk":
+                from . import random_k
+                chosen = random_k.randk_select(d, self.k, self.seed, self.t, i)
+            sel, vals, resid = compress(a, self.k, chosen)
             self.e[i] = resid
             msgs.append((sel, vals))
         S, S64 = aggregate(msgs, d)                       # server receives step t

@@ -26,6 +26,8 @@ DECO_BF16 = 1
 DECO_NO_INDEX = 0xFFFFFFFF
 DECO_SELECT_AUTO = 0
 DECO_SELECT_EXACT_PASSES = 1
+DECO_COMPRESSOR_TOPK = 0
+DECO_COMPRESSOR_RANDK = 1
 
 
 class deco_pair(ctypes.Structure):
@@ -40,7 +42,10 @@ class deco_options(ctypes.Structure):
                 ("params", ctypes.c_void_p),
                 ("device", ctypes.c_int32),
                 ("select_mode", ctypes.c_int32),
-                ("reserved", ctypes.c_uint32 * 8)]
+                ("compressor", ctypes.c_int32),
+                ("seed_lo", ctypes.c_uint32),
+                ("seed_hi", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32 * 5)]
 
 
 class deco_lut_entry(ctypes.Structure):
@@ -155,7 +160,8 @@ def _stream(stream):
 # ------------------------------------------------------------------ entry points
 
 def deco_init(d, n, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0, delta_max=0.0,
-              lr_at_server=False, params=None, device=0, select_mode=DECO_SELECT_AUTO):
+              lr_at_server=False, params=None, device=0, select_mode=DECO_SELECT_AUTO,
+              compressor=DECO_COMPRESSOR_TOPK, seed=0):
     """-> opaque context handle (int).  `params`: optional fp32 CUDA tensor of length d."""
     opt = deco_options()
     opt.grad_dtype = grad_dtype
@@ -165,6 +171,9 @@ def deco_init(d, n, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0, delta_max=0.
     opt.params = _ptr(params)
     opt.device = device
     opt.select_mode = select_mode
+    opt.compressor = compressor
+    opt.seed_lo = seed & 0xFFFFFFFF
+    opt.seed_hi = (seed >> 32) & 0xFFFFFFFF
     ctx = _vp()
     _check(load().deco_init(ctypes.byref(ctx), d, n, delta, tau, lr, ctypes.byref(opt)),
            "deco_init")

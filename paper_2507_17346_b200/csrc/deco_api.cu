@@ -139,6 +139,8 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     if (o.grad_dtype != DECO_F32 && o.grad_dtype != DECO_BF16) return DECO_ERR_INVALID_ARG;
     if (o.select_mode != DECO_SELECT_AUTO && o.select_mode != DECO_SELECT_EXACT_PASSES)
         return DECO_ERR_INVALID_ARG;
+    if (o.compressor != DECO_COMPRESSOR_TOPK && o.compressor != DECO_COMPRESSOR_RANDK)
+        return DECO_ERR_INVALID_ARG;
     if (o.delta_max != 0.0 && (!(o.delta_max <= 1.0) || o.delta_max < delta))
         return DECO_ERR_INVALID_ARG;
     if (o.tau_max != 0 && o.tau_max < tau) return DECO_ERR_INVALID_ARG;
@@ -166,6 +168,8 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     c->grad_dtype = o.grad_dtype;
     c->lr_at_server = o.lr_at_server;
     c->select_mode = o.select_mode;
+    c->compressor = o.compressor;
+    c->seed = (static_cast<uint64_t>(o.seed_hi) << 32) | o.seed_lo;
     c->device = o.device;
     c->k = deco_k_from_delta(delta, d);
     c->k_cap = deco_k_from_delta(c->delta_max, d);
@@ -554,9 +558,10 @@ struct StateHeader {
     uint64_t magic, version;
     uint64_t d, n, k_cap, ring, t, k;
     double delta;
-    uint32_t tau, grad_dtype, lr_at_server, pad;
+    uint32_t tau, grad_dtype, lr_at_server, compressor;
     float lr;
     uint32_t pad2;
+    uint64_t seed;
 };
 constexpr uint64_t STATE_MAGIC = 0x4F434544534F4345ull;   // "ECOSDECO"
 
@@ -599,6 +604,7 @@ extern "C" deco_status deco_export_state(deco_ctx *c, void *buf, uint64_t bytes,
     h.d = c->d; h.n = c->n; h.k_cap = c->k_cap; h.ring = c->ring; h.t = c->t; h.k = c->k;
     h.delta = c->delta; h.tau = c->tau; h.grad_dtype = c->grad_dtype;
     h.lr_at_server = c->lr_at_server; h.lr = c->lr;
+    h.compressor = c->compressor; h.seed = c->seed;
     std::memcpy(out, &h, sizeof h);
     out += sizeof h;
     for (const Slot &sl : c->slot_info) {
@@ -636,7 +642,8 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
     in += sizeof h;
     if (h.magic != STATE_MAGIC || h.version != 1 || h.d != c->d || h.n != c->n ||
         h.k_cap != c->k_cap || h.ring != c->ring || h.grad_dtype != static_cast<uint32_t>(c->grad_dtype) ||
-        h.lr_at_server != static_cast<uint32_t>(c->lr_at_server) || h.tau > c->tau_max || h.k > c->k_cap)
+        h.lr_at_server != static_cast<uint32_t>(c->lr_at_server) || h.tau > c->tau_max || h.k > c->k_cap ||
+        h.compressor != static_cast<uint32_t>(c->compressor) || h.seed != c->seed)
         return DECO_ERR_INVALID_ARG;
     if (bytes < sizeof(StateHeader) + sizeof(SlotRecord) * c->ring) return DECO_ERR_INVALID_ARG;
     std::vector<Slot> slots(c->ring);

@@ -34,6 +34,48 @@ namespace {
 
 constexpr uint32_t FULL = 0xFFFFFFFFu;
 
+__device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+// Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy
+// as 1, 2, 3", SC'11), written from the published definition: per round the two counter words
+// 0 and 2 are multiplied by fixed constants, the high halves are xored with the other two
+// words and the key, and the key is bumped by the Weyl constants between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c;
+}
+
+// Random-k: the priority of entry j of worker i at iteration t is a 23-bit word of the
+// Philox stream keyed by the context's seed with counter (j / 4, t_lo, i, t_hi ^ "RAND");
+// the k largest priorities (equal ones by increasing index) are the selected entries.
+struct RandParams {
+    uint32_t on;                 // 0: Top-k on |a|, 1: Random-k
+    uint32_t seed_lo, seed_hi, step_lo, step_hi;
+};
+
+__device__ __forceinline__ uint4 rand_keys4(const RandParams &rk, uint32_t worker, uint64_t j4)
+{
+    // priorities of the four entries 4*j4 .. 4*j4 + 3
+    uint4 o = philox4x32_10(make_uint4(static_cast<uint32_t>(j4), rk.step_lo, worker,
+                                       rk.step_hi ^ 0x52414E44u), rk.seed_lo, rk.seed_hi);
+    return make_uint4(o.x >> 9, o.y >> 9, o.z >> 9, o.w >> 9);
+}
+
+__device__ __forceinline__ uint32_t rand_key(const RandParams &rk, uint32_t worker, uint32_t j)
+{
+    const uint4 o = rand_keys4(rk, worker, j >> 2);
+    const uint32_t w = j & 3u;
+    return w == 0 ? o.x : (w == 1 ? o.y : (w == 2 ? o.z : o.w));
+}
+
 // Everything the selection kernels need, passed by value.
 struct Sel {
     float *e;
@@ -57,9 +99,17 @@ struct Sel {
     deco_pair *stage;
     uint64_t stage_cap;
     uint32_t *status;        // [0] latched status, [1..2] detail, [3] "some worker needs the multi-pass route"
+    RandParams rk;
+    uint32_t sample_shift;   // sample histogram bin = key >> sample_shift (top 10 key bits)
+    uint32_t bound_low_bit;  // lowest key bit the bound is refined to
 };
 
-__device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+// selection key of a staged pair
+__device__ __forceinline__ uint32_t key_of(const Sel &p, uint32_t i, const deco_pair &pr)
+{
+    return p.rk.on ? rand_key(p.rk, i, pr.idx) : mag_key(pr.val);
+}
+
 
 __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t a, uint32_t b)
 {
@@ -307,12 +357,20 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         uint32_t kk[4] = {0, 0, 0, 0};                       // 0 = "not a sample"
         if (sidx < S) {
             const uint64_t j = ((static_cast<uint64_t>(sidx) * nchunks) / S) << 2;
-            const float4 ev = *reinterpret_cast<const float4 *>(erow + j);
-            const float es[4] = {ev.x, ev.y, ev.z, ev.w};
+            if (p.rk.on) {
+                const uint4 r4 = rand_keys4(p.rk, i, j >> 2);
+                const uint32_t rs[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (j + c < p.d)
-                    kk[c] = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
+                for (int c = 0; c < 4; ++c)
+                    if (j + c < p.d) kk[c] = rs[c];
+            } else {
+                const float4 ev = *reinterpret_cast<const float4 *>(erow + j);
+                const float es[4] = {ev.x, ev.y, ev.z, ev.w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (j + c < p.d)
+                        kk[c] = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
+            }
         }
         skeys[sidx] = make_uint4(kk[0], kk[1], kk[2], kk[3]);
         // histogram of the top SAMPLE_HIST_BITS key bits (exponent and two mantissa bits) of
@@ -323,7 +381,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         __syncthreads();
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const uint32_t hb = kk[c] ? (kk[c] >> SAMPLE_HIST_SHIFT) : SAMPLE_HIST_BINS;
+            const uint32_t hb = kk[c] ? min(kk[c] >> p.sample_shift, SAMPLE_HIST_BINS - 1) : SAMPLE_HIST_BINS;
             const uint32_t grp = __match_any_sync(FULL, hb);
             if (hb < SAMPLE_HIST_BINS && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_exp[hb], __popc(grp));
         }
@@ -360,6 +418,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         // threshold may lie (in value: that ratio to the power 1/tail-index)
         const double rho = static_cast<double>(R) / (mean > 1e-9 ? mean : 1e-9);
         rel_shift = rho <= 2.0 ? 10u : (rho <= 8.0 ? 11u : 12u);
+        if (p.rk.on) rel_shift = 10u;          // uniform 23-bit priorities: 4095 << 10 is half the range
     }
     if (R > m_total) {                         // the sample cannot bound the threshold
         if (t == 0) s.spec_key = 0;            // stage everything: the count check decides
@@ -402,7 +461,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         const uint32_t higher = block_excl_scan(mine_e, s_w, tot);
         if (t == 0) s_flag = 0;
         __syncthreads();
-        if (higher < R && higher + mine_e >= R) s_flag = hb << SAMPLE_HIST_SHIFT;
+        if (higher < R && higher + mine_e >= R) s_flag = hb << p.sample_shift;
         __syncthreads();
         bound = s_flag;
         __syncthreads();
@@ -427,7 +486,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     // everything >= bound is on the lists, so counts over the lists equal counts over the
     // sample for any candidate >= bound; lane l of warp w looks at slots l, l+32, ...
 #pragma unroll 1
-    for (int bit = SAMPLE_HIST_SHIFT - 1; bit >= 7; --bit) {
+    for (int bit = static_cast<int>(p.sample_shift) - 1; bit >= static_cast<int>(p.bound_low_bit); --bit) {
         const uint32_t cand = bound | (1u << bit);
         uint32_t tot = 0;
         if (fits) {
@@ -452,10 +511,10 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
 // otherwise (and in the tile that holds the end of the vector) gradients are read entry by
 // entry.  SPEC: stage the entries whose key reaches sel[i].spec_key.
 // ------------------------------------------------------------------------------------------
-template <int GT, bool ALIGNED, bool SPEC>
+template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
 __global__ void __launch_bounds__(BLOCK)
 ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
-                     uint64_t d, float alpha, SelectState *__restrict__ sel,
+                     uint64_t d, float alpha, RandParams rk, SelectState *__restrict__ sel,
                      deco_pair *__restrict__ stage, uint64_t stage_cap,
                      uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
                      uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
@@ -554,9 +613,20 @@ ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__res
     for (int u = 0; u < U; ++u) {
         const uint64_t j = wbase + u * (32 * V) + lane * V;
         m[u] = 0;
+        uint32_t keys[V];
+        if (RANDK) {
+#pragma unroll
+            for (int q = 0; q < V / 4; ++q) {
+                const uint4 r4 = rand_keys4(rk, i, (j >> 2) + q);
+                keys[4 * q] = r4.x; keys[4 * q + 1] = r4.y; keys[4 * q + 2] = r4.z; keys[4 * q + 3] = r4.w;
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < V; ++c) keys[c] = mag_key(x[u][c]);
+        }
 #pragma unroll
         for (int c = 0; c < V; ++c)
-            if (mag_key(x[u][c]) >= bound && (full || j + c < d)) m[u] |= 1u << c;
+            if (keys[c] >= bound && (full || j + c < d)) m[u] |= 1u << c;
         cnt[u] = __popc(m[u]);
         any |= m[u];
     }
@@ -639,16 +709,18 @@ stage_hist_a_kernel(Sel p)
         const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
         for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
              base += gridDim.x * (4 * BLOCK)) {
-            float v[4];
+            deco_pair v[4];
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const uint32_t q = base + r * BLOCK + threadIdx.x;
-                v[r] = q < n_staged ? src[q].val : 0.0f;
+                v[r].idx = 0;
+                v[r].val = 0.0f;
+                if (q < n_staged) v[r] = src[q];
             }
 #pragma unroll
             for (int r = 0; r < 4; ++r)
                 if (base + r * BLOCK + threadIdx.x < n_staged)
-                    atomicAdd(&h[rel_bin_a(mag_key(v[r]), spec, shift)], 1u);
+                    atomicAdd(&h[rel_bin_a(key_of(p, i, v[r]), spec, shift)], 1u);
         }
         __syncthreads();
         uint32_t *out = hist_of(p, i, 0, 0);
@@ -690,16 +762,18 @@ stage_hist_b_kernel(Sel p)
     __syncthreads();
     for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
          base += gridDim.x * (4 * BLOCK)) {
-        float v[4];
+        deco_pair v[4];
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const uint32_t q = base + r * BLOCK + threadIdx.x;
-            v[r] = q < n_staged ? src[q].val : 0.0f;
+            v[r].idx = 0;
+            v[r].val = 0.0f;
+            if (q < n_staged) v[r] = src[q];
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             if (base + r * BLOCK + threadIdx.x >= n_staged) continue;
-            const uint32_t key = mag_key(v[r]);
+            const uint32_t key = key_of(p, i, v[r]);
             if (rel_bin_a(key, spec, shift) == a_sel) atomicAdd(&h[(key - spec) & low_mask], 1u);
         }
     }
@@ -856,9 +930,9 @@ stage_classify_kernel(Sel p, uint32_t walk_here)
         for (int r = 0; r < 4; ++r) {
             // neighbours in the staging area mostly belong to the same tile: lanes with the
             // same (tile, class) elect one of them to add the group's size
-            const uint32_t key = mag_key(prs[r].val);
-            const uint32_t tile = prs[r].idx / TILE;
             const bool in = base + r * BLOCK + threadIdx.x < n_staged;
+            const uint32_t key = in ? key_of(p, i, prs[r]) : 0x7FFFFFFFu;
+            const uint32_t tile = prs[r].idx / TILE;
             const uint32_t cls = !in ? 0u : (key < T ? 1u : (key == T ? 2u : 0u));
             const uint32_t grp = __match_any_sync(FULL, cls ? (tile * 2 + cls - 1) : 0xFFFFFFFFu);
             if (cls && lane == __ffs(grp) - 1)
@@ -875,7 +949,7 @@ stage_classify_kernel(Sel p, uint32_t walk_here)
                 const uint32_t q = base + r * BLOCK + threadIdx.x;
                 if (q < n_staged) {
                     const deco_pair pr = src[q];
-                    if (mag_key(pr.val) < T) erow[pr.idx] = pr.val;
+                    if (key_of(p, i, pr) < T) erow[pr.idx] = pr.val;
                 }
             }
         }
@@ -949,7 +1023,7 @@ __device__ __forceinline__ void emit_segment_warp(const Sel &p, uint32_t i, uint
             const deco_pair pr = prs[r];
             bool gt = false, eq = false;
             if (base + r * 32 + lane < cnt) {
-                const uint32_t key = mag_key(pr.val);
+                const uint32_t key = key_of(p, i, pr);
                 gt = key > T;
                 eq = key == T;
             }
@@ -1017,7 +1091,7 @@ emit_stage_chunk_kernel(Sel p)
         uint32_t written = 0, ties_seen = 0;
         for (uint32_t q = 0; q < t.cnt; ++q) {
             const deco_pair pr = src[q];
-            const uint32_t key = mag_key(pr.val);
+            const uint32_t key = key_of(p, i, pr);
             const bool eq = key == T;
             const bool pick = key > T || (eq && ties_seen < t.take);
             ties_seen += eq ? 1u : 0u;
@@ -1055,12 +1129,18 @@ __device__ __forceinline__ void hist_e_body(const Sel &p, uint32_t i, uint32_t p
     const uint64_t nvec = (p.d + 3) >> 2;
     for (uint64_t v = static_cast<uint64_t>(part) * BLOCK + threadIdx.x; v < nvec;
          v += static_cast<uint64_t>(nparts) * BLOCK) {
-        const float4 q = row[v];
         const uint64_t j = v << 2;
-        radix_bin<LEVEL>(mag_key(q.x), prefix, h);
-        if (j + 1 < p.d) radix_bin<LEVEL>(mag_key(q.y), prefix, h);
-        if (j + 2 < p.d) radix_bin<LEVEL>(mag_key(q.z), prefix, h);
-        if (j + 3 < p.d) radix_bin<LEVEL>(mag_key(q.w), prefix, h);
+        uint4 kq;
+        if (p.rk.on) {
+            kq = rand_keys4(p.rk, i, v);
+        } else {
+            const float4 q = row[v];
+            kq = make_uint4(mag_key(q.x), mag_key(q.y), mag_key(q.z), mag_key(q.w));
+        }
+        radix_bin<LEVEL>(kq.x, prefix, h);
+        if (j + 1 < p.d) radix_bin<LEVEL>(kq.y, prefix, h);
+        if (j + 2 < p.d) radix_bin<LEVEL>(kq.z, prefix, h);
+        if (j + 3 < p.d) radix_bin<LEVEL>(kq.w, prefix, h);
     }
     __syncthreads();
     uint32_t *out = hist_of(p, i, 1, LEVEL);
@@ -1079,11 +1159,17 @@ __device__ __forceinline__ void count_e_tile(const Sel &p, uint32_t i, uint32_t 
 #pragma unroll
     for (int r = 0; r < TILE / (4 * BLOCK); ++r) {
         const uint64_t j = base + (static_cast<uint64_t>(r) * BLOCK + threadIdx.x) * 4;
-        const float4 q = *reinterpret_cast<const float4 *>(row + j);
-        const float xs[4] = {q.x, q.y, q.z, q.w};
+        uint4 kq;
+        if (p.rk.on) {
+            kq = rand_keys4(p.rk, i, j >> 2);
+        } else {
+            const float4 q = *reinterpret_cast<const float4 *>(row + j);
+            kq = make_uint4(mag_key(q.x), mag_key(q.y), mag_key(q.z), mag_key(q.w));
+        }
+        const uint32_t ks[4] = {kq.x, kq.y, kq.z, kq.w};
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const uint32_t key = mag_key(xs[c]);
+            const uint32_t key = ks[c];
             const bool in = j + c < p.d;
             gt += (in && key > T);
             eq += (in && key == T);
@@ -1215,9 +1301,12 @@ __device__ __forceinline__ void emit_e_tile(const Sel &p, uint32_t i, uint32_t t
         const float4 q = *reinterpret_cast<const float4 *>(erow + j);
         x[u][0] = q.x; x[u][1] = q.y; x[u][2] = q.z; x[u][3] = q.w;
         gt[u] = eq[u] = 0;
+        uint4 kq = make_uint4(mag_key(q.x), mag_key(q.y), mag_key(q.z), mag_key(q.w));
+        if (p.rk.on) kq = rand_keys4(p.rk, i, j >> 2);
+        const uint32_t ks[4] = {kq.x, kq.y, kq.z, kq.w};
 #pragma unroll
         for (int c = 0; c < V; ++c) {
-            const uint32_t key = mag_key(x[u][c]);
+            const uint32_t key = ks[c];
             if (j + c < p.d) {
                 gt[u] |= (key > T) ? (1u << c) : 0u;
                 eq[u] |= (key == T) ? (1u << c) : 0u;
@@ -1387,6 +1476,17 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
     }
 }
 
+RandParams make_rand(const deco_ctx *c)
+{
+    RandParams rk;
+    rk.on = c->compressor == DECO_COMPRESSOR_RANDK ? 1u : 0u;
+    rk.seed_lo = static_cast<uint32_t>(c->seed);
+    rk.seed_hi = static_cast<uint32_t>(c->seed >> 32);
+    rk.step_lo = static_cast<uint32_t>(c->t);
+    rk.step_hi = static_cast<uint32_t>(c->t >> 32);
+    return rk;
+}
+
 Sel make_sel(const deco_ctx *c)
 {
     Sel p;
@@ -1419,6 +1519,9 @@ Sel make_sel(const deco_ctx *c)
     p.stage = c->stage;
     p.stage_cap = c->stage_cap;
     p.status = c->dev_status;
+    p.rk = make_rand(c);
+    p.sample_shift = p.rk.on ? 13u : static_cast<uint32_t>(SAMPLE_HIST_SHIFT);
+    p.bound_low_bit = p.rk.on ? 0u : 7u;
     return p;
 }
 
@@ -1450,18 +1553,26 @@ cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s)
     return cudaGetLastError();
 }
 
+template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
+static void launch_acc_variant(deco_ctx *c, const void *grads, float alpha, cudaStream_t s)
+{
+    dim3 grid(c->ntiles, c->n);
+    ef_accumulate_kernel<GT, ALIGNED, SPEC, RANDK><<<grid, BLOCK, 0, s>>>(
+        c->e, c->e_stride, grads, c->d, alpha, make_rand(c), c->sel, c->stage, c->stage_cap,
+        c->tile_off, c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
+}
+
 template <int GT, bool ALIGNED>
 static void launch_acc(deco_ctx *c, const void *grads, float alpha, cudaStream_t s)
 {
-    dim3 grid(c->ntiles, c->n);
-    if (streaming_route(c))
-        ef_accumulate_kernel<GT, ALIGNED, true><<<grid, BLOCK, 0, s>>>(
-            c->e, c->e_stride, grads, c->d, alpha, c->sel, c->stage, c->stage_cap, c->tile_off,
-            c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
-    else
-        ef_accumulate_kernel<GT, ALIGNED, false><<<grid, BLOCK, 0, s>>>(
-            c->e, c->e_stride, grads, c->d, alpha, c->sel, c->stage, c->stage_cap, c->tile_off,
-            c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
+    const bool randk = c->compressor == DECO_COMPRESSOR_RANDK;
+    if (streaming_route(c)) {
+        if (randk) launch_acc_variant<GT, ALIGNED, true, true>(c, grads, alpha, s);
+        else launch_acc_variant<GT, ALIGNED, true, false>(c, grads, alpha, s);
+    } else {
+        // the multi-pass route derives the keys itself: nothing is staged here
+        launch_acc_variant<GT, ALIGNED, false, false>(c, grads, alpha, s);
+    }
 }
 
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s)

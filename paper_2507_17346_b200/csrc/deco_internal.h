@@ -72,6 +72,8 @@ struct deco_ctx {
     int grad_dtype = DECO_F32;
     int lr_at_server = 0;
     int select_mode = DECO_SELECT_AUTO;
+    int compressor = DECO_COMPRESSOR_TOPK;
+    uint64_t seed = 0;                  // Random-k: key of the priority stream
     int device = 0;
     // derived
     uint64_t k = 0, k_cap = 0;

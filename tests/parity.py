@@ -58,7 +58,7 @@ def close(a, b64, scale_terms, rtol):
 
 def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mode=None,
                policy_plan=None, lr_at_server=False, tau_max=0, delta_max=0.0, device=0,
-               check_every=1, expect_exact=None):
+               check_every=1, expect_exact=None, compressor="topk", seed=0):
     """grad_fn(step) -> torch CUDA tensor [n, d] (float32 or bfloat16).
 
     policy_plan: {step: (delta, tau)} applied before that step on both sides."""
@@ -67,9 +67,12 @@ def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mo
     ctx = B.deco_init(d, n, delta, tau, lr,
                       grad_dtype=B.DECO_F32 if grad_dtype == "f32" else B.DECO_BF16,
                       tau_max=tau_max, delta_max=delta_max, lr_at_server=lr_at_server,
-                      device=device, select_mode=mode)
+                      device=device, select_mode=mode,
+                      compressor=B.DECO_COMPRESSOR_RANDK if compressor == "randk"
+                      else B.DECO_COMPRESSOR_TOPK, seed=seed)
     try:
-        orc = O.DDEFSGD(d, n, delta, tau, lr, lr_in_compress=not lr_at_server)
+        orc = O.DDEFSGD(d, n, delta, tau, lr, lr_in_compress=not lr_at_server,
+                        compressor=compressor, seed=seed)
         assert B.deco_get_k(ctx) == orc.k
         abs_S, mass = {}, np.zeros(d)
         scale = float(np.float32(1.0 if not lr_at_server else lr) / np.float32(n))

@@ -157,6 +157,25 @@ def test_many_workers_and_odd_length(mode):
                select_mode=mode)
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_random_k_sparsifier(mode):
+    """Random-k in place of Top-k: the same Philox priorities on both sides give the same index
+    sets; everything downstream (residual, aggregate, update) is shared with Top-k."""
+    seed = 0x5EED0123456789AB
+    for d, n, delta, dtype, name in [(4097, 2, 0.01, torch.float32, "f32"),
+                                     (20001, 3, 0.3, torch.bfloat16, "bf16"),
+                                     (300_000, 4, 0.01, torch.float32, "f32"),
+                                     (300_000, 2, 0.0005, torch.float32, "f32"),
+                                     (50_000, 2, 1.0, torch.float32, "f32")]:
+        run_parity(d, n, delta, 2, 0.1, lambda t: _values("normal", n, d, t, dtype), steps=5,
+                   grad_dtype=name, select_mode=mode, compressor="randk", seed=seed)
+    wl = W.make_workload("resnet18", 0.25)
+    st = run_parity(wl.d, wl.n, wl.delta, wl.tau, wl.lr, lambda t: W.gradients(wl, t, "cuda"),
+                    steps=6, select_mode=mode, compressor="randk", seed=7)
+    if mode == B.DECO_SELECT_AUTO:
+        assert st["exact_pass_workers"] == 0          # the sampled bound holds for uniform priorities
+
+
 def test_call_order_and_capacity_errors():
     d, n = 10_000, 2
     ctx = B.deco_init(d, n, 0.01, 1, 0.1, tau_max=2, delta_max=0.05)
