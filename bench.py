@@ -269,6 +269,7 @@ def run_ours(args):
     ev0.record(stream)
     for t in range(steps):
         B.deco_step(ctx, pool[(warmup + t) % pool_n], stream)
+    B.deco_join(ctx, stream)            # the last aggregation ends inside the timed region
     ev1.record(stream)
     torch.cuda.synchronize()
     t_wall1 = time.time()
@@ -301,6 +302,7 @@ def run_ours(args):
         e0.record(stream)
         for t in range(e_steps):
             B.deco_step_host(ctx, host_g[t % 2], host_msg, None, stream)
+        B.deco_join(ctx, stream)
         e1.record(stream)
         torch.cuda.synchronize()
         e_ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")

@@ -85,6 +85,7 @@ SIGNATURES = {
     "deco_aggregate_stale": (_i32, [_vp, _vp]),
     "deco_apply_update": (_i32, [_vp, _vp]),
     "deco_step": (_i32, [_vp, _vp, _vp]),
+    "deco_join": (_i32, [_vp, _vp]),
     "deco_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "deco_set_policy": (_i32, [_vp, _f64, _u32]),
     "deco_set_lr": (_i32, [_vp, _f32]),
@@ -202,6 +203,10 @@ def deco_apply_update(ctx, stream=None):
 
 def deco_step(ctx, grads, stream=None):
     _check(load().deco_step(ctx, _ptr(grads), _stream(stream)), "deco_step")
+
+
+def deco_join(ctx, stream=None):
+    _check(load().deco_join(ctx, _stream(stream)), "deco_join")
 
 
 def deco_step_host(ctx, grads_host, msg_host_out=None, params_host_out=None, stream=None):

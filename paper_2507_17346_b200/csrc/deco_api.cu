@@ -68,7 +68,10 @@ void free_all(deco_ctx *c)
     c->events.clear();
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->ev_emit) cudaEventDestroy(c->ev_emit);
+    if (c->ev_agg) cudaEventDestroy(c->ev_agg);
     if (c->side_stream) cudaStreamDestroy(c->side_stream);
+    if (c->agg_stream) cudaStreamDestroy(c->agg_stream);
 }
 
 deco_status zero_state(deco_ctx *c, cudaStream_t s)
@@ -92,6 +95,16 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
 }
 
 inline cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
+
+// Host-side wait for whatever deco_step left on the internal stream (for calls that read the
+// cache or the device status from the host, or hand out pointers).
+inline cudaError_t drain_internal(deco_ctx *c)
+{
+    c->agg_pending = false;
+    if (!c->side_stream) return cudaSuccess;
+    const cudaError_t err = cudaStreamSynchronize(c->side_stream);
+    return err != cudaSuccess ? err : cudaStreamSynchronize(c->agg_stream);
+}
 
 constexpr size_t MAX_TIMED_ITERS = 4096;
 
@@ -220,8 +233,11 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     if (st == DECO_OK && query_fallback_grid(c) != cudaSuccess) st = DECO_ERR_CUDA;
     if (st == DECO_OK &&
         (cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+         cudaStreamCreateWithFlags(&c->agg_stream, cudaStreamNonBlocking) != cudaSuccess ||
          cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-         cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
+         cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&c->ev_emit, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&c->ev_agg, cudaEventDisableTiming) != cudaSuccess))
         st = DECO_ERR_CUDA;
     if (st == DECO_OK) st = zero_state(c, nullptr);
     if (st == DECO_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = DECO_ERR_CUDA;
@@ -249,6 +265,7 @@ extern "C" deco_status deco_reset(deco_ctx *c, void *stream)
     if (!c) return DECO_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
+    if (drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
     return zero_state(c, as_stream(stream));
 }
 
@@ -282,6 +299,7 @@ extern "C" deco_status deco_aggregate_stale(deco_ctx *c, void *stream)
     Slot &sl = c->slot_info[si];
     if (sl.valid) return DECO_ERR_STATE;    // cannot happen while tau <= tau_max
     deco_pair *slot = c->slots + static_cast<uint64_t>(si) * c->n * c->k_cap;
+    if (wait_for_aggregate(c, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
     mark(c, 3, as_stream(stream));
     if (launch_aggregate(c, slot, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
     mark(c, 4, as_stream(stream));
@@ -329,6 +347,7 @@ extern "C" deco_status deco_apply_update(deco_ctx *c, void *stream)
     if (c->phase != 2) return DECO_ERR_STATE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
+    if (wait_for_aggregate(c, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
     mark(c, 5, as_stream(stream));
     const deco_status st = apply_due(c, as_stream(stream));
     if (st != DECO_OK) return st;
@@ -354,6 +373,7 @@ extern "C" deco_status deco_get_kernel_timing(deco_ctx *c, void *stream, double 
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
     if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    if (drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
     static const int pairs[4][2] = {{0, 1}, {1, 2}, {3, 4}, {5, 6}};
     for (int p = 0; p < 4; ++p) ms_sum[p] = 0.0;
     for (size_t it = 0; it < c->timed_iters; ++it)
@@ -382,24 +402,46 @@ extern "C" deco_status deco_step(deco_ctx *c, const void *grads, void *stream)
     }
     // tau >= 1: the aggregates due now were cached in earlier iterations and touch neither e
     // nor the messages, so their update runs on an internal stream next to the streaming
-    // pass.  It is forked from and joined back into the caller's stream inside this call:
-    // everything is complete, in stream order, when the caller's stream passes the call.
+    // pass.  It is forked from and joined back into the caller's stream inside this call: e,
+    // the messages and the parameters are complete, in stream order, when the caller's stream
+    // passes the call.
     if (reinterpret_cast<uintptr_t>(grads) & 15u) return DECO_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);
     if (cudaEventRecord(c->ev_fork, s) != cudaSuccess) return DECO_ERR_CUDA;
     if (cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0) != cudaSuccess) return DECO_ERR_CUDA;
+    // the only aggregation that can still be running is that of iteration t - 1, which is
+    // due now only if tau = 1
+    if (c->tau <= 1 && cudaStreamWaitEvent(c->side_stream, c->ev_agg, 0) != cudaSuccess)
+        return DECO_ERR_CUDA;
     mark(c, 5, c->side_stream);
     deco_status st = apply_due(c, c->side_stream);
     mark(c, 6, c->side_stream);
     if (cudaEventRecord(c->ev_join, c->side_stream) != cudaSuccess) return DECO_ERR_CUDA;
     if (st == DECO_OK) st = deco_ef_compress(c, grads, stream);
-    if (st == DECO_OK) st = deco_aggregate_stale(c, stream);
-    if (cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) return DECO_ERR_CUDA;
     if (st != DECO_OK) return st;
+    // This iteration's aggregate is not needed before iteration t + tau: it goes onto a second
+    // internal stream behind the messages and may run next to whatever the caller's stream
+    // does next (the streaming pass of the following iteration).  Every later launch that
+    // rewrites the messages or reads the cache orders itself after ev_agg.
+    if (cudaEventRecord(c->ev_emit, s) != cudaSuccess) return DECO_ERR_CUDA;
+    if (cudaStreamWaitEvent(c->agg_stream, c->ev_emit, 0) != cudaSuccess) return DECO_ERR_CUDA;
+    st = deco_aggregate_stale(c, c->agg_stream);
+    if (st != DECO_OK) return st;
+    if (cudaEventRecord(c->ev_agg, c->agg_stream) != cudaSuccess) return DECO_ERR_CUDA;
+    c->agg_pending = true;
+    if (cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) return DECO_ERR_CUDA;
     finish_iteration(c);
     return DECO_OK;
+}
+
+extern "C" deco_status deco_join(deco_ctx *c, void *stream)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return DECO_ERR_CUDA;
+    return wait_for_aggregate(c, as_stream(stream)) == cudaSuccess ? DECO_OK : DECO_ERR_CUDA;
 }
 
 extern "C" deco_status deco_step_host(deco_ctx *c, const void *grads_host, deco_pair *msg_out,
@@ -488,6 +530,10 @@ extern "C" deco_status deco_get_aggregate(deco_ctx *c, uint64_t step, const deco
     if (!c || !entries || !positions) return DECO_ERR_INVALID_ARG;
     const Slot &sl = c->slot_info[step % c->ring];
     if (!sl.valid || sl.step != step) return DECO_ERR_STATE;
+    {
+        DeviceGuard guard(c->device);
+        if (!guard.ok || drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
+    }
     *entries = c->slots + (step % c->ring) * c->n * c->k_cap;
     *positions = sl.positions;
     return DECO_OK;
@@ -522,6 +568,7 @@ extern "C" deco_status deco_get_stats(deco_ctx *c, void *stream, deco_stats *out
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
     if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    if (drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
     uint32_t st[4] = {0, 0, 0, 0};
     if (cudaMemcpy(st, c->dev_status, sizeof st, cudaMemcpyDeviceToHost) != cudaSuccess)
         return DECO_ERR_CUDA;
@@ -595,6 +642,7 @@ extern "C" deco_status deco_export_state(deco_ctx *c, void *buf, uint64_t bytes,
     if (bytes < state_size(c)) return DECO_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
+    if (drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);
     char *out = static_cast<char *>(buf);
     StateHeader h;
@@ -663,6 +711,7 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
     if (bytes < need) return DECO_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
+    if (drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);
     deco_status st = zero_state(c, s);                       // padding of e, status, counters
     if (st != DECO_OK) return st;

@@ -1610,6 +1610,7 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     Sel p = make_sel(c);
     dim3 tgrid(c->ntiles, c->n);
     if (!streaming_route(c)) {
+        if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();
         dim3 hgrid(part_blocks(c, (c->d + 3) / 4, BLOCK * 8), c->n);
         radix_hist_e_kernel<0><<<hgrid, BLOCK, 0, s>>>(p);
         radix_pick_kernel<0><<<c->n, BLOCK, 0, s>>>(p);
@@ -1634,6 +1635,9 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
         chunk_sums_kernel<<<dim3((c->nchunks + WARPS - 1) / WARPS, c->n), BLOCK, 0, s>>>(p);
         c->launches += 1;
     }
+    // the kernels from here on rewrite the messages and their directory, which the previous
+    // iteration's aggregation may still be reading on the internal stream
+    if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();
     // about 1.3 k staged entries spread over ntiles tiles: a warp per tile when a tile holds
     // many, a warp per chunk of tiles when it holds few
     if (13 * c->k >= 240ull * c->ntiles) {

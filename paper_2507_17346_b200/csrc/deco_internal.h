@@ -117,8 +117,14 @@ struct deco_ctx {
     uint64_t launches = 0;
     uint64_t k_of_msg = 0;              // k used by the last compress
     // internal stream of deco_step: the stale update runs next to the streaming pass
-    cudaStream_t side_stream = nullptr;
+    cudaStream_t side_stream = nullptr;      // stale update next to the worker side
+    cudaStream_t agg_stream = nullptr;       // aggregation left running past the end of deco_step
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // deco_step leaves the aggregation of its iteration running on agg_stream: ev_emit marks
+    // the messages complete, ev_agg the aggregation done; agg_pending says that a later launch
+    // which rewrites the messages or reads the cache has to wait for ev_agg first
+    cudaEvent_t ev_emit = nullptr, ev_agg = nullptr;
+    bool agg_pending = false;
     // optional event timing: 8 events per recorded iteration
     bool timing = false;
     std::vector<cudaEvent_t> events;
@@ -132,6 +138,14 @@ cudaError_t query_fallback_grid(deco_ctx *c);
 cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s);
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s);
 cudaError_t launch_selection(deco_ctx *c, cudaStream_t s);
+
+// Order stream s after the aggregation that deco_step left running on the internal stream.
+inline cudaError_t wait_for_aggregate(deco_ctx *c, cudaStream_t s)
+{
+    if (!c->agg_pending) return cudaSuccess;
+    c->agg_pending = false;
+    return cudaStreamWaitEvent(s, c->ev_agg, 0);
+}
 // --- kernel launchers (deco_server.cu) ---------------------------------------------------
 cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s);
 cudaError_t launch_apply(deco_ctx *c, const deco_pair *slot, uint64_t positions, float neg_scale,

@@ -231,9 +231,10 @@ def test_two_runs_give_the_same_bits():
 
 
 def test_fused_step_equals_the_three_calls():
-    """deco_step runs the stale update on an internal stream next to the worker side; the
-    result must be the bits of compress -> aggregate -> apply issued one after the other,
-    also across changes of tau (including tau = 0, where nothing may overlap)."""
+    """deco_step runs the stale update on an internal stream next to the worker side and leaves
+    its aggregation running there; the result must be the bits of compress -> aggregate ->
+    apply issued one after the other, also across changes of tau (including tau = 0, where
+    nothing may overlap) and when the two forms are mixed on one context."""
     wl = W.make_workload("resnet18", 0.25)
     kw = dict(tau_max=3, delta_max=0.02)
     a = B.deco_init(wl.d, wl.n, wl.delta, 2, wl.lr, **kw)
@@ -241,14 +242,19 @@ def test_fused_step_equals_the_three_calls():
     side = torch.cuda.Stream()
     try:
         plan = {3: (0.02, 0), 5: (0.005, 3), 8: (0.01, 1)}
-        for t in range(11):
+        for t in range(14):
             if t in plan:
                 B.deco_set_policy(a, *plan[t])
                 B.deco_set_policy(b, *plan[t])
             g = W.gradients(wl, t, "cuda")
             torch.cuda.synchronize()
             with torch.cuda.stream(side):                       # a non-default caller stream
-                B.deco_step(a, g)
+                if t % 4 == 3:                                  # the three calls right behind a
+                    B.deco_ef_compress(a, g)                    # fused step: they have to order
+                    B.deco_aggregate_stale(a)                   # themselves after its aggregation
+                    B.deco_apply_update(a)
+                else:
+                    B.deco_step(a, g)
             B.deco_ef_compress(b, g)
             B.deco_aggregate_stale(b)
             B.deco_apply_update(b)
@@ -258,7 +264,7 @@ def test_fused_step_equals_the_three_calls():
             assert torch.equal(B.view_i32(ba["e"], (wl.n, ba["e_stride"])),
                                B.view_i32(bb["e"], (wl.n, bb["e_stride"]))), t
         sa, sb = B.deco_get_stats(a), B.deco_get_stats(b)
-        assert sa["step"] == sb["step"] == 11 and sa["cached_aggregates"] == sb["cached_aggregates"]
+        assert sa["step"] == sb["step"] == 14 and sa["cached_aggregates"] == sb["cached_aggregates"]
         assert sa["device_status"] == 0 and sb["device_status"] == 0
     finally:
         B.deco_destroy(a)
