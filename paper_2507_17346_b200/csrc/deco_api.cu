@@ -45,6 +45,7 @@ void free_all(deco_ctx *c)
     cudaFree(c->msg);
     cudaFree(c->slots);
     cudaFree(c->stage);
+    cudaFree(c->work);
     cudaFree(c->hist);
     cudaFree(c->sel);
     cudaFree(c->tile_gt);
@@ -212,6 +213,9 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->msg, static_cast<uint64_t>(n) * c->k_cap));
     need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * n * c->k_cap));
     need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
+    // slices of 256 staged entries, plus one partial slice for every tile that has any
+    c->work_cap = c->stage_cap / 256 + (c->stage_cap / 17 < c->ntiles ? c->stage_cap / 17 : c->ntiles) + 32;
+    need(dev_alloc(c, &c->work, static_cast<uint64_t>(n) * c->work_cap));
     need(dev_alloc(c, &c->hist, static_cast<uint64_t>(n) * 2 * RADIX_LEVELS * RADIX_BINS));
     need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * DONE_SLOTS));
     need(dev_alloc(c, &c->sample_keys, static_cast<uint64_t>(n) * SAMPLE_KEYS));

@@ -98,6 +98,8 @@ struct Sel {
     uint64_t k_cap;
     deco_pair *stage;
     uint64_t stage_cap;
+    uint2 *work;             // [n][work_cap] (tile, slice) entries of the emit work list
+    uint64_t work_cap;
     uint32_t *status;        // [0] latched status, [1..2] detail, [3] "some worker needs the multi-pass route"
     RandParams rk;
     uint32_t sample_shift;   // sample histogram bin = key >> sample_shift (top 10 key bits)
@@ -328,6 +330,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     if (part == 0) {
         if (t < 3) p.done[i * DONE_SLOTS + t] = 0;          // levels A, B, classification
         if (t == 4) p.done[i * DONE_SLOTS + 4] = 0;         // chunk sums
+        if (t == 5) p.done[i * DONE_SLOTS + 5] = 0;         // length of the emit work list
         if (i == 0 && t == 0) p.status[3] = exact_all;
         if (t == 0) {
             s.prefix = 0;
@@ -687,6 +690,46 @@ __device__ __forceinline__ uint32_t rel_bin_a(uint32_t key, uint32_t spec, uint3
 
 __device__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w, bool streaming);
 
+// Emit works on slices: EMIT_SLICE consecutive staged entries of one tile.  A tile with at most
+// EMIT_LANE_MAX staged entries is walked by a single lane; every other tile is cut into slices
+// that are listed (in no particular order) in a per-worker work list, so that a layer whose
+// tiles hold thousands of candidates is spread over as many warps as it has slices.
+constexpr uint32_t EMIT_SLICE = 256;
+constexpr uint32_t EMIT_LANE_MAX = 16;
+
+__device__ __forceinline__ uint32_t emit_items_of(uint32_t cnt)
+{
+    return cnt > EMIT_LANE_MAX ? (cnt + EMIT_SLICE - 1) / EMIT_SLICE : 0u;
+}
+
+// Work list of a worker: one (tile, slice) entry per slice; every thread looks at one tile, a
+// warp reserves its entries with one atomic.  Called by all threads of the CTAs of a kernel
+// that runs between the streaming pass and emit.
+__device__ __forceinline__ void build_emit_work(const Sel &p, uint32_t i)
+{
+    const int lane = threadIdx.x & 31;
+    uint32_t *count = &p.done[i * DONE_SLOTS + 5];
+    uint2 *work = p.work + static_cast<size_t>(i) * p.work_cap;
+    const uint32_t tiles_up = (p.ntiles + 31u) & ~31u;       // whole warps stay together
+    for (uint32_t tile = blockIdx.x * BLOCK + threadIdx.x; tile < tiles_up;
+         tile += gridDim.x * BLOCK) {
+        const uint32_t items =
+            tile < p.ntiles ? emit_items_of(p.tile_cnt[static_cast<size_t>(i) * p.ntiles + tile]) : 0u;
+        const uint32_t incl = warp_incl_scan(items);
+        const uint32_t total = __shfl_sync(FULL, incl, 31);
+        if (total == 0) continue;
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(count, total);
+        base = __shfl_sync(FULL, base, 0) + incl - items;
+        if (base + items > p.work_cap) {
+            if (items) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x320u, tile);
+            continue;
+        }
+        for (uint32_t j = 0; j < items; ++j) work[base + j] = make_uint2(tile, j);
+    }
+}
+
+
 // Level A: histogram of the coarse bins of all staged keys.  The last CTA of a worker to
 // arrive takes the decision: is the staged set usable (at least k entries, so it contains the
 // k largest, and no overflow of the staging area), and which coarse bin holds the k-th
@@ -759,6 +802,7 @@ stage_hist_b_kernel(Sel p)
     const uint32_t low_mask = (1u << shift) - 1u;
     const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
+    build_emit_work(p, i);                              // independent of the histogram
     __syncthreads();
     for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
          base += gridDim.x * (4 * BLOCK)) {
@@ -971,6 +1015,7 @@ struct TileInfo {
     uint32_t start;   // message position of the tile's first entry
 };
 
+template <bool WRITE_DIR>
 __device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint32_t chunk)
 {
     const int lane = threadIdx.x & 31;
@@ -992,37 +1037,42 @@ __device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint3
     t.take = min(eq, left);
     t.sel = cnt - rej - eq + t.take;
     t.start = start0 + warp_incl_scan(t.sel) - t.sel;
-    // the directory the aggregation reads: message position of every tile
-    if (tile < p.ntiles) p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile] = t.start;
-    if (tile == p.ntiles - 1) p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + p.ntiles] = t.start + t.sel;
+    if (WRITE_DIR) {
+        // the directory the aggregation reads: message position of every tile
+        if (tile < p.ntiles) p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile] = t.start;
+        if (tile == p.ntiles - 1)
+            p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + p.ntiles] = t.start + t.sel;
+    }
     return t;
 }
 
-// The whole warp filters one tile's staged segment, in order, into the message.  The selected
-// entries are already +0 in e; ties that are not taken get their value back.
-__device__ __forceinline__ void emit_segment_warp(const Sel &p, uint32_t i, uint32_t tile,
-                                                  uint32_t off, uint32_t cnt, uint32_t start,
-                                                  uint32_t want, uint32_t take, uint32_t T)
+// The whole warp filters staged entries [begin, end) of one tile's segment, in order, into the
+// message; `written` entries of the tile were emitted and `ties_seen` ties met before `begin`.
+// The selected entries are already +0 in e; ties that are not taken get their value back.
+// Returns the number of entries written.
+__device__ __forceinline__ uint32_t emit_segment_warp(const Sel &p, uint32_t i, uint32_t tile,
+                                                      uint32_t off, uint32_t begin, uint32_t end,
+                                                      uint32_t start, uint32_t written,
+                                                      uint32_t ties_seen, uint32_t take, uint32_t T)
 {
     const int lane = threadIdx.x & 31;
     const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
     deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
     float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
-    uint32_t written = 0, ties_seen = 0;
-    for (uint32_t base = 0; base < cnt; base += 128) {       // four loads in flight per lane
+    for (uint32_t base = begin; base < end; base += 128) {     // four loads in flight per lane
         deco_pair prs[4];
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const uint32_t q = base + r * 32 + lane;
             prs[r].idx = 0;
             prs[r].val = 0.f;
-            if (q < cnt) prs[r] = src[q];
+            if (q < end) prs[r] = src[q];
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const deco_pair pr = prs[r];
             bool gt = false, eq = false;
-            if (base + r * 32 + lane < cnt) {
+            if (base + r * 32 + lane < end) {
                 const uint32_t key = key_of(p, i, pr);
                 gt = key > T;
                 eq = key == T;
@@ -1044,47 +1094,27 @@ __device__ __forceinline__ void emit_segment_warp(const Sel &p, uint32_t i, uint
             ties_seen += __popc(eq_mask);
         }
     }
-    if (lane == 0 && written != want) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x311u, tile);
+    return written;
 }
 
-// Emit, many staged entries per tile: one warp per tile.
+// Emit.  CTAs [0, dir_ctas) of a worker: one warp per chunk of CHUNK_TILES tiles writes the
+// directory and each lane walks its own tile if that holds at most EMIT_LANE_MAX staged
+// entries.  The remaining CTAs: their warps stride over the work list; a warp that gets slice
+// j > 0 of a tile first counts, with independent loads, what the slices before it emit.
 __global__ void __launch_bounds__(BLOCK)
-emit_stage_tile_kernel(Sel p)
+emit_stage_kernel(Sel p, uint32_t dir_ctas)
 {
     const uint32_t i = blockIdx.y;
     if (p.sel[i].exact) return;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t tile = blockIdx.x * WARPS + w;
-    if (tile >= p.ntiles) return;
-    const uint32_t my = tile % CHUNK_TILES;
-    const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
-    if (my != 0 && p.tile_cnt[ti] == 0) return;               // lane-0 warps write the directory
-    const TileInfo t = chunk_header(p, i, tile / CHUNK_TILES);
-    const uint32_t cnt = __shfl_sync(FULL, t.cnt, my);
-    if (cnt == 0) return;
-    const uint32_t start = __shfl_sync(FULL, t.start, my), want = __shfl_sync(FULL, t.sel, my);
-    const uint32_t take = __shfl_sync(FULL, t.take, my);
-    (void)lane;
-    emit_segment_warp(p, i, tile, p.tile_off[ti], cnt, start, want, take, p.sel[i].threshold);
-}
-
-// Emit, few staged entries per tile: one warp per chunk, each lane walks its own tile's few
-// entries; a tile with many entries is done by the whole warp.
-__global__ void __launch_bounds__(BLOCK)
-emit_stage_chunk_kernel(Sel p)
-{
-    constexpr uint32_t LANE_MAX = 16;
-    const uint32_t i = blockIdx.y;
-    if (p.sel[i].exact) return;
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t chunk = blockIdx.x * WARPS + w;
-    if (chunk >= p.nchunks) return;
-    const TileInfo t = chunk_header(p, i, chunk);
-    const uint32_t tile = chunk * CHUNK_TILES + lane;
     const uint32_t T = p.sel[i].threshold;
-    uint32_t off = 0;
-    if (t.cnt) off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
-    if (t.cnt && t.cnt <= LANE_MAX) {
+    if (blockIdx.x < dir_ctas) {
+        const uint32_t chunk = blockIdx.x * WARPS + w;
+        if (chunk >= p.nchunks) return;
+        const TileInfo t = chunk_header<true>(p, i, chunk);
+        const uint32_t tile = chunk * CHUNK_TILES + lane;
+        if (t.cnt == 0 || t.cnt > EMIT_LANE_MAX) return;
+        const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
         const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
         deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
         float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
@@ -1104,14 +1134,56 @@ emit_stage_chunk_kernel(Sel p)
             }
         }
         if (written != t.sel) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x313u, tile);
+        return;
     }
-    uint32_t big = __ballot_sync(FULL, t.cnt > LANE_MAX);
-    while (big) {
-        const int b = __ffs(big) - 1;
-        big &= big - 1;
-        emit_segment_warp(p, i, chunk * CHUNK_TILES + b, __shfl_sync(FULL, off, b),
-                          __shfl_sync(FULL, t.cnt, b), __shfl_sync(FULL, t.start, b),
-                          __shfl_sync(FULL, t.sel, b), __shfl_sync(FULL, t.take, b), T);
+    const uint32_t n_items = min(p.done[i * DONE_SLOTS + 5], static_cast<uint32_t>(p.work_cap));
+    const uint2 *work = p.work + static_cast<size_t>(i) * p.work_cap;
+    const uint32_t warps = (gridDim.x - dir_ctas) * WARPS;
+    for (uint32_t q = (blockIdx.x - dir_ctas) * WARPS + w; q < n_items; q += warps) {
+        const uint2 item = work[q];
+        const uint32_t tile = item.x, slice = item.y;
+        if (tile >= p.ntiles) {
+            if (lane == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x321u, q);
+            continue;
+        }
+        const TileInfo t = chunk_header<false>(p, i, tile / CHUNK_TILES);
+        const uint32_t my = tile % CHUNK_TILES;
+        const uint32_t cnt = __shfl_sync(FULL, t.cnt, my), start = __shfl_sync(FULL, t.start, my);
+        const uint32_t want = __shfl_sync(FULL, t.sel, my), take = __shfl_sync(FULL, t.take, my);
+        const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
+        const uint32_t begin = slice * EMIT_SLICE;
+        if (begin >= cnt) {
+            if (lane == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x322u, tile);
+            continue;
+        }
+        const uint32_t end = min(cnt, begin + EMIT_SLICE);
+        uint32_t written = 0, ties_seen = 0;
+        if (begin) {
+            // what slices 0..slice-1 emit: the entries above the threshold plus the ties
+            // that are still granted; whole slices, so every load is in range
+            const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
+            uint32_t g = 0, e = 0;
+            for (uint32_t base = 0; base < begin; base += EMIT_SLICE) {
+                deco_pair prs[EMIT_SLICE / 32];
+#pragma unroll
+                for (uint32_t r = 0; r < EMIT_SLICE / 32; ++r) prs[r] = src[base + r * 32 + lane];
+#pragma unroll
+                for (uint32_t r = 0; r < EMIT_SLICE / 32; ++r) {
+                    const uint32_t key = key_of(p, i, prs[r]);
+                    g += key > T ? 1u : 0u;
+                    e += key == T ? 1u : 0u;
+                }
+            }
+            for (int o = 16; o > 0; o >>= 1) {
+                g += __shfl_xor_sync(FULL, g, o);
+                e += __shfl_xor_sync(FULL, e, o);
+            }
+            written = g + min(e, take);
+            ties_seen = e;
+        }
+        written = emit_segment_warp(p, i, tile, off, begin, end, start, written, ties_seen, take, T);
+        if (end == cnt && lane == 0 && written != want)
+            latch(p.status, DECO_ERR_DEVICE_CHECK, 0x311u, tile);
     }
 }
 
@@ -1518,6 +1590,8 @@ Sel make_sel(const deco_ctx *c)
     p.k_cap = c->k_cap;
     p.stage = c->stage;
     p.stage_cap = c->stage_cap;
+    p.work = c->work;
+    p.work_cap = c->work_cap;
     p.status = c->dev_status;
     p.rk = make_rand(c);
     p.sample_shift = p.rk.on ? 13u : static_cast<uint32_t>(SAMPLE_HIST_SHIFT);
@@ -1638,14 +1712,17 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     // the kernels from here on rewrite the messages and their directory, which the previous
     // iteration's aggregation may still be reading on the internal stream
     if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();
-    // about 1.3 k staged entries spread over ntiles tiles: a warp per tile when a tile holds
-    // many, a warp per chunk of tiles when it holds few
-    if (13 * c->k >= 240ull * c->ntiles) {
-        dim3 wgrid((c->ntiles + WARPS - 1) / WARPS, c->n);
-        emit_stage_tile_kernel<<<wgrid, BLOCK, 0, s>>>(p);
-    } else {
-        dim3 wgrid((c->nchunks + WARPS - 1) / WARPS, c->n);
-        emit_stage_chunk_kernel<<<wgrid, BLOCK, 0, s>>>(p);
+    // directory CTAs (a warp per chunk), then the CTAs whose warps stride over the work list:
+    // enough of them for one slice per warp at about 1.3 k staged entries, capped at a few
+    // waves of the device
+    {
+        const uint32_t dir_ctas = (c->nchunks + WARPS - 1) / WARPS;
+        const uint64_t staged = 13 * c->k / 10, many = staged / (EMIT_LANE_MAX + 1);
+        const uint64_t est_items = staged / EMIT_SLICE + (many < c->ntiles ? many : c->ntiles);
+        uint64_t item_ctas = (est_items + WARPS - 1) / WARPS + 1;
+        const uint64_t cap = (148ull * 8 * 8 + c->n - 1) / c->n;
+        if (item_ctas > cap) item_ctas = cap;
+        emit_stage_kernel<<<dim3(dir_ctas + static_cast<uint32_t>(item_ctas), c->n), BLOCK, 0, s>>>(p, dir_ctas);
     }
     c->launches += 4;
     cudaError_t err = cudaGetLastError();

@@ -24,9 +24,9 @@ constexpr int WARP_ELEMS = TILE / WARPS;   // 1024
 constexpr int RADIX_BINS = 4096;
 constexpr int RADIX_LEVELS = 3;
 
-// Arrival counters per worker: level A, level B, classification, sampling (resets itself),
-// chunk sums.
-constexpr int DONE_SLOTS = 5;
+// Counters per worker: CTA arrivals at level A, level B, classification, sampling (resets
+// itself) and chunk sums; the length of the emit work list.
+constexpr int DONE_SLOTS = 6;
 
 // Per-worker selection record (device).  One 64-byte line per worker.
 struct SelectState {
@@ -88,6 +88,8 @@ struct deco_ctx {
     deco_pair *msg = nullptr;
     deco_pair *slots = nullptr;         // [ring][n * k_cap]
     deco_pair *stage = nullptr;         // [n][stage_cap]
+    uint2 *work = nullptr;              // [n][work_cap] emit work list: (tile, slice)
+    uint64_t work_cap = 0;
     uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
     uint32_t *done = nullptr;           // [n][DONE_SLOTS] CTA arrival counters
     uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
