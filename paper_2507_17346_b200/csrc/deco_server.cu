@@ -27,6 +27,128 @@ __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t 
     }
 }
 
+// One tile by the whole CTA: dense fp32 accumulator and touched-bit mask in shared memory (both
+// all-zero on entry and on exit), workers added in order, output in index order.
+__device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, uint64_t k_cap,
+                                           const uint32_t *__restrict__ tile_start, uint32_t ntiles,
+                                           uint32_t n, deco_pair *__restrict__ slot,
+                                           uint64_t positions, uint32_t *__restrict__ status,
+                                           uint32_t tile, float *acc, uint32_t *mask, uint32_t *s_w)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint64_t out_off = 0;
+    uint32_t cap = 0, longest = 0;
+    for (uint32_t i = 0; i < n; ++i) {
+        const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
+        const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+        out_off += a;
+        cap += b - a;
+        longest = max(longest, b - a);
+    }
+    if (cap == 0) return;
+    if (out_off + cap > positions) {
+        if (threadIdx.x == 0) latch(status, DECO_ERR_DEVICE_CHECK, 0x400u, tile);
+        return;
+    }
+    const uint32_t first = tile * static_cast<uint32_t>(TILE);
+    if (n <= PREFETCH_WORKERS && longest <= static_cast<uint32_t>(BLOCK)) {
+        // At most one entry per thread and worker.  All loads are issued before the first
+        // barrier, then the workers are added in order from registers.
+        deco_pair pre[PREFETCH_WORKERS];
+#pragma unroll
+        for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
+            pre[i].idx = DECO_NO_INDEX;
+            pre[i].val = 0.0f;
+            if (i < n) {
+                const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
+                const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+                if (a + threadIdx.x < b) pre[i] = msg[static_cast<size_t>(i) * k_cap + a + threadIdx.x];
+            }
+        }
+#pragma unroll
+        for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
+            if (i >= n) break;
+            if (pre[i].idx != DECO_NO_INDEX) {
+                const uint32_t loc = pre[i].idx - first;
+                if (loc >= static_cast<uint32_t>(TILE)) {
+                    latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pre[i].idx);
+                } else {
+                    acc[loc] = acc[loc] + pre[i].val;      // indices are unique per worker
+                    atomicOr(&mask[loc >> 5], 1u << (loc & 31));
+                }
+            }
+            __syncthreads();
+        }
+    } else {
+        for (uint32_t i = 0; i < n; ++i) {                 // worker order 0..n-1
+            const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
+            const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+            if (b == a) continue;
+            const deco_pair *src = msg + static_cast<size_t>(i) * k_cap;
+            for (uint32_t p0 = a; p0 < b; p0 += 4 * BLOCK) {   // four loads in flight
+                deco_pair prs[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const uint32_t p = p0 + r * BLOCK + threadIdx.x;
+                    prs[r].idx = DECO_NO_INDEX;
+                    prs[r].val = 0.0f;
+                    if (p < b) prs[r] = src[p];
+                }
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if (prs[r].idx == DECO_NO_INDEX) continue;
+                    const uint32_t loc = prs[r].idx - first;
+                    if (loc >= static_cast<uint32_t>(TILE)) {
+                        latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, prs[r].idx);
+                        continue;
+                    }
+                    acc[loc] = acc[loc] + prs[r].val;      // indices are unique per worker
+                    atomicOr(&mask[loc >> 5], 1u << (loc & 31));
+                }
+            }
+            __syncthreads();
+        }
+    }
+    uint32_t word = mask[threadIdx.x];
+    const uint32_t c = __popc(word);
+    uint32_t incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(FULL, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) s_w[w] = incl;
+    __syncthreads();
+    uint32_t before = 0, uniq = 0;
+#pragma unroll
+    for (int ww = 0; ww < WARPS; ++ww) {
+        const uint32_t v = s_w[ww];
+        before += (ww < w) ? v : 0u;
+        uniq += v;
+    }
+    deco_pair *out = slot + out_off;
+    uint32_t p = before + incl - c;
+    while (word) {
+        const uint32_t b = __ffs(word) - 1;
+        word &= word - 1;
+        const uint32_t loc = threadIdx.x * 32 + b;
+        deco_pair pr;
+        pr.idx = first + loc;
+        pr.val = acc[loc];
+        out[p++] = pr;
+        acc[loc] = 0.0f;
+    }
+    mask[threadIdx.x] = 0;
+    for (uint32_t q = uniq + threadIdx.x; q < cap; q += BLOCK) {
+        deco_pair pr;
+        pr.idx = DECO_NO_INDEX;
+        pr.val = 0.0f;
+        out[q] = pr;
+    }
+    __syncthreads();
+}
+
+// Persistent CTAs, every tile by the whole CTA: for messages with many entries per tile.
 __global__ void __launch_bounds__(BLOCK)
 aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
                  const uint32_t *__restrict__ tile_start, uint32_t ntiles, uint32_t n,
@@ -39,120 +161,170 @@ aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     for (int q = threadIdx.x; q < TILE; q += BLOCK) acc[q] = 0.0f;
     mask[threadIdx.x] = 0;
     __syncthreads();
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
+        dense_tile(msg, k_cap, tile_start, ntiles, n, slot, positions, status, tile, acc, mask, s_w);
+}
 
-    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        uint64_t out_off = 0;
-        uint32_t cap = 0, longest = 0;
-        for (uint32_t i = 0; i < n; ++i) {
-            const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-            const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
-            out_off += a;
-            cap += b - a;
-            longest = max(longest, b - a);
+// The entries a warp holds (one per lane, at most 32, worker-major and index-sorted within a
+// worker; lanes without one pass valid = false) merged into out[0 .. uniq): entries with the
+// same index are summed in worker order starting from +0, the sums are written in index order.
+// Returns uniq.
+__device__ __forceinline__ uint32_t warp_merge(bool valid, uint32_t idx, float val,
+                                               deco_pair *__restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    // lanes without an entry get keys of their own, so that they match nobody
+    const uint32_t grp = __match_any_sync(FULL, valid ? idx : (0xFFFFFF00u | lane));
+    const bool head = valid && lane == __ffs(grp) - 1;
+    float sum = 0.0f;
+    uint32_t rest = valid ? grp : 0u;
+    while (__any_sync(FULL, rest != 0)) {                     // ascending lanes = worker order
+        const int src = rest ? __ffs(rest) - 1 : 0;
+        const float v = __shfl_sync(FULL, val, src);
+        if (rest) {
+            sum = sum + v;
+            rest &= rest - 1;
         }
-        if (cap == 0) continue;
-        if (out_off + cap > positions) {
-            if (threadIdx.x == 0) latch(status, DECO_ERR_DEVICE_CHECK, 0x400u, tile);
-            continue;
+    }
+    const uint32_t heads = __ballot_sync(FULL, head);
+    uint32_t rank = 0;
+    for (uint32_t h = heads; h; h &= h - 1) {
+        const uint32_t other = __shfl_sync(FULL, idx, __ffs(h) - 1);
+        rank += other < idx ? 1u : 0u;
+    }
+    if (head) {
+        deco_pair pr;
+        pr.idx = idx;
+        pr.val = sum;
+        out[rank] = pr;
+    }
+    return __popc(heads);
+}
+
+// Sparse messages (a few entries per tile): one warp per tile, no accumulator.  Lane i first
+// holds worker i's range of the tile.  At most 32 entries in all are merged in one go;
+// otherwise the tile's index range is cut into SPARSE_WINDOWS windows that are merged one
+// after the other, each with at most 32 entries.  A tile that does not fit is left to the
+// whole CTA afterwards (dense_tile).
+constexpr int SPARSE_WINDOWS = 4;
+
+__global__ void __launch_bounds__(BLOCK)
+aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
+                        const uint32_t *__restrict__ tile_start, uint32_t ntiles, uint32_t n,
+                        deco_pair *__restrict__ slot, uint64_t positions,
+                        uint32_t *__restrict__ status)
+{
+    __shared__ float acc[TILE];
+    __shared__ uint32_t mask[TILE / 32];
+    __shared__ uint32_t s_w[WARPS];
+    __shared__ uint32_t s_heavy;
+    if (threadIdx.x == 0) s_heavy = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t tile = blockIdx.x * WARPS + w;
+    if (tile < ntiles) {
+        uint32_t a = 0, b = 0;
+        if (static_cast<uint32_t>(lane) < n) {
+            a = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile];
+            b = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile + 1];
         }
-        const uint32_t first = tile * static_cast<uint32_t>(TILE);
-        if (n <= PREFETCH_WORKERS && longest <= static_cast<uint32_t>(BLOCK)) {
-            // Sparse case: at most one entry per thread and worker.  All loads are issued
-            // before the first barrier, then the workers are added in order from registers.
-            deco_pair pre[PREFETCH_WORKERS];
-#pragma unroll
-            for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
-                pre[i].idx = DECO_NO_INDEX;
-                pre[i].val = 0.0f;
-                if (i < n) {
-                    const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-                    const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
-                    if (a + threadIdx.x < b) pre[i] = msg[static_cast<size_t>(i) * k_cap + a + threadIdx.x];
-                }
-            }
-#pragma unroll
-            for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
-                if (i >= n) break;
-                if (pre[i].idx != DECO_NO_INDEX) {
-                    const uint32_t loc = pre[i].idx - first;
-                    if (loc >= static_cast<uint32_t>(TILE)) {
-                        latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pre[i].idx);
-                    } else {
-                        acc[loc] = acc[loc] + pre[i].val;      // indices are unique per worker
-                        atomicOr(&mask[loc >> 5], 1u << (loc & 31));
-                    }
-                }
-                __syncthreads();
-            }
-        } else {
-            for (uint32_t i = 0; i < n; ++i) {                 // worker order 0..n-1
-                const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-                const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
-                if (b == a) continue;
-                const deco_pair *src = msg + static_cast<size_t>(i) * k_cap;
-                for (uint32_t p0 = a; p0 < b; p0 += 4 * BLOCK) {   // four loads in flight
-                    deco_pair prs[4];
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const uint32_t p = p0 + r * BLOCK + threadIdx.x;
-                        prs[r].idx = DECO_NO_INDEX;
-                        prs[r].val = 0.0f;
-                        if (p < b) prs[r] = src[p];
-                    }
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        if (prs[r].idx == DECO_NO_INDEX) continue;
-                        const uint32_t loc = prs[r].idx - first;
-                        if (loc >= static_cast<uint32_t>(TILE)) {
-                            latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, prs[r].idx);
-                            continue;
-                        }
-                        acc[loc] = acc[loc] + prs[r].val;      // indices are unique per worker
-                        atomicOr(&mask[loc >> 5], 1u << (loc & 31));
-                    }
-                }
-                __syncthreads();
-            }
-        }
-        uint32_t word = mask[threadIdx.x];
-        const uint32_t c = __popc(word);
-        uint32_t incl = c;
+        const uint32_t len = b - a;
+        uint32_t cap = len, longest = len;
+        uint64_t out_off = a;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t t = __shfl_up_sync(FULL, incl, o);
-            if (lane >= o) incl += t;
+            cap += __shfl_xor_sync(FULL, cap, o);
+            longest = max(longest, __shfl_xor_sync(FULL, longest, o));
+            out_off += __shfl_xor_sync(FULL, out_off, o);
         }
-        if (lane == 31) s_w[w] = incl;
-        __syncthreads();
-        uint32_t before = 0, uniq = 0;
+        const uint32_t first = tile * static_cast<uint32_t>(TILE);
+        if (cap == 0) {
+        } else if (out_off + cap > positions) {
+            if (lane == 0) latch(status, DECO_ERR_DEVICE_CHECK, 0x400u, tile);
+        } else if (cap > 32u * SPARSE_WINDOWS || longest > 32) {
+            if (lane == 0) atomicOr(&s_heavy, 1u << w);
+        } else {
+            // lane i: how many of worker i's entries lie below the end of each window
+            // (every lane looks at one entry of each worker in turn: ranges are at most 32 long)
+            uint32_t below[SPARSE_WINDOWS + 1];
+            below[0] = 0;
 #pragma unroll
-        for (int ww = 0; ww < WARPS; ++ww) {
-            const uint32_t v = s_w[ww];
-            before += (ww < w) ? v : 0u;
-            uniq += v;
+            for (int q = 1; q <= SPARSE_WINDOWS; ++q) below[q] = len;
+            if (cap > 32) {
+                for (uint32_t i = 0; i < n; ++i) {
+                    const uint32_t ai = __shfl_sync(FULL, a, i), li = __shfl_sync(FULL, len, i);
+                    uint32_t loc = DECO_NO_INDEX;
+                    if (static_cast<uint32_t>(lane) < li)
+                        loc = msg[static_cast<size_t>(i) * k_cap + ai + lane].idx - first;
+#pragma unroll
+                    for (int q = 1; q < SPARSE_WINDOWS; ++q) {
+                        const uint32_t cnt = __popc(__ballot_sync(FULL, loc < q * (TILE / SPARSE_WINDOWS)));
+                        if (static_cast<uint32_t>(lane) == i) below[q] = cnt;
+                    }
+                }
+            }
+            // per window: entries of the workers before lane's own, and in all
+            uint32_t before[SPARSE_WINDOWS], total[SPARSE_WINDOWS];
+            bool fits = true;
+#pragma unroll
+            for (int q = 0; q < SPARSE_WINDOWS; ++q) {
+                const uint32_t mine = below[q + 1] - below[q];
+                uint32_t incl = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(FULL, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                before[q] = incl - mine;
+                total[q] = __shfl_sync(FULL, incl, 31);
+                fits = fits && total[q] <= 32;
+            }
+            if (!fits) {
+                if (lane == 0) atomicOr(&s_heavy, 1u << w);
+            } else {
+                deco_pair *out = slot + out_off;
+                uint32_t uniq = 0;
+#pragma unroll
+                for (int q = 0; q < SPARSE_WINDOWS; ++q) {
+                    if (total[q] == 0) continue;
+                    const uint32_t part_a = a + below[q], part_len = below[q + 1] - below[q];
+                    deco_pair pr;
+                    pr.idx = DECO_NO_INDEX;
+                    pr.val = 0.0f;
+                    bool valid = false;
+                    for (uint32_t i = 0; i < n; ++i) {
+                        const uint32_t pb = __shfl_sync(FULL, before[q], i);
+                        const uint32_t pl = __shfl_sync(FULL, part_len, i);
+                        const uint32_t pa = __shfl_sync(FULL, part_a, i);
+                        if (static_cast<uint32_t>(lane) >= pb && static_cast<uint32_t>(lane) < pb + pl) {
+                            pr = msg[static_cast<size_t>(i) * k_cap + pa + (lane - pb)];
+                            valid = true;
+                        }
+                    }
+                    if (valid && pr.idx - first >= static_cast<uint32_t>(TILE)) {
+                        latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pr.idx);
+                        valid = false;
+                    }
+                    uniq += warp_merge(valid, pr.idx, pr.val, out + uniq);
+                }
+                for (uint32_t q = uniq + lane; q < cap; q += 32) {
+                    deco_pair pr;
+                    pr.idx = DECO_NO_INDEX;
+                    pr.val = 0.0f;
+                    out[q] = pr;
+                }
+            }
         }
-        deco_pair *out = slot + out_off;
-        uint32_t p = before + incl - c;
-        while (word) {
-            const uint32_t b = __ffs(word) - 1;
-            word &= word - 1;
-            const uint32_t loc = threadIdx.x * 32 + b;
-            deco_pair pr;
-            pr.idx = first + loc;
-            pr.val = acc[loc];
-            out[p++] = pr;
-            acc[loc] = 0.0f;
-        }
-        mask[threadIdx.x] = 0;
-        for (uint32_t q = uniq + threadIdx.x; q < cap; q += BLOCK) {
-            deco_pair pr;
-            pr.idx = DECO_NO_INDEX;
-            pr.val = 0.0f;
-            out[q] = pr;
-        }
-        __syncthreads();
     }
+    __syncthreads();
+    uint32_t heavy = s_heavy;
+    if (heavy == 0) return;
+    for (int q = threadIdx.x; q < TILE; q += BLOCK) acc[q] = 0.0f;
+    mask[threadIdx.x] = 0;
+    __syncthreads();
+    for (; heavy; heavy &= heavy - 1)
+        dense_tile(msg, k_cap, tile_start, ntiles, n, slot, positions, status,
+                   blockIdx.x * WARPS + __ffs(heavy) - 1, acc, mask, s_w);
 }
 
 __global__ void __launch_bounds__(256)
@@ -176,14 +348,20 @@ apply_kernel(const deco_pair *__restrict__ slot, uint64_t positions, float neg_s
 
 cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s)
 {
+    const uint64_t positions = static_cast<uint64_t>(c->n) * c->k_of_msg;
+    c->launches += 1;
+    if (c->n <= 32 && positions <= 80ull * c->ntiles) {
+        // on average at most 80 entries per tile over all workers: a warp per tile
+        aggregate_sparse_kernel<<<(c->ntiles + WARPS - 1) / WARPS, BLOCK, 0, s>>>(
+            c->msg, c->k_cap, c->tile_start, c->ntiles, c->n, slot, positions, c->dev_status);
+        return cudaGetLastError();
+    }
     // next to the streaming pass of the following iteration the aggregation takes half the
     // CTA slots it could hold, so that the pass keeps most of its loads in flight
     const uint32_t per_sm = (c->agg_stream && s == c->agg_stream) ? 3u : 6u;
     const uint32_t blocks = c->ntiles < 148u * per_sm ? c->ntiles : 148u * per_sm;
     aggregate_kernel<<<blocks, BLOCK, 0, s>>>(c->msg, c->k_cap, c->tile_start, c->ntiles, c->n,
-                                              slot, static_cast<uint64_t>(c->n) * c->k_of_msg,
-                                              c->dev_status);
-    c->launches += 1;
+                                              slot, positions, c->dev_status);
     return cudaGetLastError();
 }
 

@@ -157,6 +157,28 @@ def test_many_workers_and_odd_length(mode):
                select_mode=mode)
 
 
+@pytest.mark.parametrize("n", [3, 8, 20])
+def test_sparse_messages_take_every_aggregation_path(n):
+    """A few entries per tile: the aggregation merges a tile in one warp, in one go (at most 32
+    entries), window by window (at most 32 per quarter of the tile), or hands it to the whole
+    CTA (a hot tile).  Workers share most of their large entries, so sums of 2..n terms, in
+    worker order, are the rule."""
+    d, delta = 200_003, 0.002
+
+    def grads(t):
+        g = torch.Generator(device="cuda")
+        g.manual_seed(77 + t)
+        base = torch.randn((1, d), generator=g, device="cuda")
+        x = base * (1.0 + 0.2 * torch.randn((n, d), generator=g, device="cuda"))
+        x[:, 3 * 8192:4 * 8192] *= 50.0                      # hot tile: hundreds of entries
+        x[:, 10 * 8192:10 * 8192 + 2048] *= 4.0              # one crowded quarter
+        x[:, 17 * 8192:19 * 8192] *= 2.0                     # 30..100 entries per tile
+        return x.contiguous()
+
+    st = run_parity(d, n, delta, 1, 0.1, grads, steps=4)
+    assert st["device_status"] == 0
+
+
 @pytest.mark.parametrize("mode", MODES)
 def test_random_k_sparsifier(mode):
     """Random-k in place of Top-k: the same Philox priorities on both sides give the same index
