@@ -85,7 +85,7 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
     if (err == cudaSuccess)
         err = cudaMemsetAsync(c->done, 0, sizeof(uint32_t) * c->n * DONE_SLOTS, s);
     if (err == cudaSuccess)
-        err = cudaMemsetAsync(c->sample_hist, 0, sizeof(uint32_t) * c->n * 1024, s);
+        err = cudaMemsetAsync(c->sample_hist, 0, sizeof(uint32_t) * c->n * SAMPLE_BINS, s);
     if (err == cudaSuccess)
         err = cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n * (c->ntiles + 1), s);
     c->launches += 5;
@@ -219,7 +219,7 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     need(dev_alloc(c, &c->hist, static_cast<uint64_t>(n) * 2 * RADIX_LEVELS * RADIX_BINS));
     need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * DONE_SLOTS));
     need(dev_alloc(c, &c->sample_keys, static_cast<uint64_t>(n) * SAMPLE_KEYS));
-    need(dev_alloc(c, &c->sample_hist, static_cast<uint64_t>(n) * 1024));
+    need(dev_alloc(c, &c->sample_hist, static_cast<uint64_t>(n) * SAMPLE_BINS));
     need(dev_alloc(c, &c->sel, n));
     need(dev_alloc(c, &c->tile_gt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_eq, static_cast<uint64_t>(n) * c->ntiles));

@@ -88,7 +88,7 @@ struct Sel {
     uint32_t *hist;          // [n][2][RADIX_LEVELS][RADIX_BINS]: 0 = staged route, 1 = multi-pass
     uint32_t *done;          // [n][DONE_SLOTS] CTA arrival counters
     uint32_t *sample_keys;   // [n][4 * SAMPLE_CHUNKS] keys of the sample
-    uint32_t *sample_hist;   // [n][1024] sample keys per top-10-bit bin; cleared by its reader
+    uint32_t *sample_hist;   // [n][SAMPLE_BINS] sample keys per bin of their top bits; cleared by its reader
     uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt, *tile_rej;
     uint32_t nchunks;        // chunks of CHUNK_TILES tiles
     uint32_t *chunk_cnt, *chunk_rej, *chunk_eq;   // [n][nchunks] staged / rejected / ties
@@ -102,7 +102,7 @@ struct Sel {
     uint64_t work_cap;
     uint32_t *status;        // [0] latched status, [1..2] detail, [3] "some worker needs the multi-pass route"
     RandParams rk;
-    uint32_t sample_shift;   // sample histogram bin = key >> sample_shift (top 10 key bits)
+    uint32_t sample_shift;   // sample histogram bin = key >> sample_shift
     uint32_t bound_low_bit;  // lowest key bit the bound is refined to
 };
 
@@ -303,29 +303,46 @@ __device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *
 }
 
 // ------------------------------------------------------------------------------------------
-// Start of an iteration.  SAMPLE_CTAS CTAs per worker: together they clear the histograms and,
+// Start of an iteration.  Up to SAMPLE_CTAS CTAs per worker: together they clear the histograms and,
 // on the streaming route, draw the sample (each thread one group of 4 consecutive entries,
 // groups evenly spread over [0, d)) and leave its keys in global memory; CTA 0 re-arms the
 // selection record; the last CTA of a worker to arrive fixes spec_key from the sample.
 // ------------------------------------------------------------------------------------------
 constexpr int BEGIN_BLOCK = 1024;
-constexpr int SAMPLE_CTAS = 8;
-constexpr int SAMPLE_CHUNKS = SAMPLE_CTAS * BEGIN_BLOCK;   // 8192 groups of 4 entries
-constexpr int SAMPLE_KEYS_PER_THREAD = 4 * SAMPLE_CTAS;    // keys per thread in the search
-constexpr int SAMPLE_HIST_SHIFT = 21;                      // 31-bit key -> its top 10 bits
-constexpr uint32_t SAMPLE_HIST_BINS = 1u << (31 - SAMPLE_HIST_SHIFT);
-static_assert(SAMPLE_HIST_BINS == BEGIN_BLOCK, "one histogram bin per thread");
+constexpr int SAMPLE_CTAS = 32;
+constexpr int SAMPLE_CHUNKS = SAMPLE_CTAS * BEGIN_BLOCK;   // at most 32768 groups of 4 entries
+constexpr int SAMPLE_HIST_BITS = 12;                       // top key bits the histogram resolves
+constexpr uint32_t SAMPLE_HIST_BINS = 1u << SAMPLE_HIST_BITS;
+constexpr int SAMPLE_BINS_PER_THREAD = SAMPLE_HIST_BINS / BEGIN_BLOCK;
+constexpr int SAMPLE_WARP_LIST = 256;                      // list slots per warp in the search
+static_assert(4 * SAMPLE_CHUNKS == SAMPLE_KEYS, "sample buffer size");
+static_assert(SAMPLE_HIST_BINS == SAMPLE_BINS, "sample histogram size");
+static_assert(SAMPLE_HIST_BINS <= (BEGIN_BLOCK / 32) * SAMPLE_WARP_LIST, "histogram shares the list storage");
+
+// Number of sample groups S.  A group costs two random line fetches (e and g); a candidate
+// that is staged and then rejected costs about as much (its +0 guess is undone), and their
+// number falls like 5 k / sqrt(4 S k / d).  The sum is smallest near S = (k d)^(1/3); the
+// factor is fitted to measurements.  Between a quarter of the maximum and the maximum, never
+// more than the vector has.
+static uint32_t sample_groups(uint64_t d, uint64_t k)
+{
+    const uint64_t nchunks = (d + 3) >> 2;
+    uint64_t want = static_cast<uint64_t>(0.6 * cbrt(static_cast<double>(d) * static_cast<double>(k)));
+    if (want < SAMPLE_CHUNKS / 4) want = SAMPLE_CHUNKS / 4;
+    if (want > SAMPLE_CHUNKS) want = SAMPLE_CHUNKS;
+    return static_cast<uint32_t>(nchunks < want ? nchunks : want);
+}
 
 template <int GT>
-__global__ void __launch_bounds__(BEGIN_BLOCK)
-begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t exact_all)
+__global__ void __launch_bounds__(BEGIN_BLOCK, 2)
+begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t exact_all, uint32_t S)
 {
     const uint32_t i = blockIdx.y, part = blockIdx.x;
     const int t = threadIdx.x;
     SelectState &s = p.sel[i];
     uint32_t *hz = hist_of(p, i, 0, 0);
     for (int q = part * BEGIN_BLOCK + t; q < 2 * RADIX_LEVELS * RADIX_BINS;
-         q += SAMPLE_CTAS * BEGIN_BLOCK)
+         q += gridDim.x * BEGIN_BLOCK)
         hz[q] = 0;
     if (part == 0) {
         if (t < 3) p.done[i * DONE_SLOTS + t] = 0;          // levels A, B, classification
@@ -347,13 +364,15 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     }
     if (exact_all) return;
 
+    constexpr int NW = BEGIN_BLOCK / 32;
+    __shared__ uint32_t s_buf[NW * SAMPLE_WARP_LIST];        // histogram, later the warp lists
+    __shared__ uint32_t s_cnt[NW];
     __shared__ uint32_t s_w[33];
     __shared__ uint32_t s_flag;
     const float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     const char *grow = reinterpret_cast<const char *>(grads) +
                        static_cast<size_t>(i) * p.d * (GT ? 2 : 4);
     const uint64_t nchunks = (p.d + 3) >> 2;
-    const uint32_t S = nchunks < SAMPLE_CHUNKS ? static_cast<uint32_t>(nchunks) : SAMPLE_CHUNKS;
     uint4 *skeys = reinterpret_cast<uint4 *>(p.sample_keys) + static_cast<size_t>(i) * SAMPLE_CHUNKS;
     {
         const uint32_t sidx = part * BEGIN_BLOCK + t;
@@ -376,35 +395,31 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
             }
         }
         skeys[sidx] = make_uint4(kk[0], kk[1], kk[2], kk[3]);
-        // histogram of the top SAMPLE_HIST_BITS key bits (exponent and two mantissa bits) of
-        // this CTA's nonzero keys: lanes with the same bin elect one of them to add the
-        // group's size
-        __shared__ uint32_t s_exp[SAMPLE_HIST_BINS];
-        s_exp[t] = 0;
-        __syncthreads();
+        // histogram of the top SAMPLE_HIST_BITS key bits of this CTA's nonzero keys: lanes
+        // with the same bin elect one of them to add the group's size
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint32_t hb = kk[c] ? min(kk[c] >> p.sample_shift, SAMPLE_HIST_BINS - 1) : SAMPLE_HIST_BINS;
-            const uint32_t grp = __match_any_sync(FULL, hb);
-            if (hb < SAMPLE_HIST_BINS && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_exp[hb], __popc(grp));
+        for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) s_buf[c * BEGIN_BLOCK + t] = 0;
+        __syncthreads();
+        {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t hb = kk[c] ? min(kk[c] >> p.sample_shift, SAMPLE_HIST_BINS - 1) : SAMPLE_HIST_BINS;
+                const uint32_t grp = __match_any_sync(FULL, hb);
+                if (hb < SAMPLE_HIST_BINS && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_buf[hb], __popc(grp));
+            }
         }
         __syncthreads();
-        if (s_exp[t]) atomicAdd(&p.sample_hist[i * SAMPLE_HIST_BINS + t], s_exp[t]);
+#pragma unroll
+        for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) {
+            const uint32_t v = s_buf[c * BEGIN_BLOCK + t];
+            if (v) atomicAdd(&p.sample_hist[i * SAMPLE_HIST_BINS + c * BEGIN_BLOCK + t], v);
+        }
     }
     // the arrival counter resets itself: only the last CTA touches it afterwards
     uint32_t *arrive = &p.done[i * DONE_SLOTS + 3];
     if (!last_cta_to_arrive(arrive, &s_flag)) return;
     if (t == 0) *arrive = 0;
 
-    uint32_t keys[SAMPLE_KEYS_PER_THREAD];
-#pragma unroll
-    for (int q = 0; q < SAMPLE_CTAS; ++q) {
-        const uint4 v = __ldcg(skeys + q * BEGIN_BLOCK + t);
-        keys[q * 4 + 0] = v.x;
-        keys[q * 4 + 1] = v.y;
-        keys[q * 4 + 2] = v.z;
-        keys[q * 4 + 3] = v.w;
-    }
     // every sampled group is complete unless the sample is the whole vector
     const uint32_t m_total = (S == nchunks) ? static_cast<uint32_t>(p.d) : 4u * S;
     // rank inside the sample: mean + 5 sigma + 2 of a binomial with p = k/d (exact when the
@@ -423,87 +438,135 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         rel_shift = rho <= 2.0 ? 10u : (rho <= 8.0 ? 11u : 12u);
         if (p.rk.on) rel_shift = 10u;          // uniform 23-bit priorities: 4095 << 10 is half the range
     }
+    uint32_t *gh = p.sample_hist + i * SAMPLE_HIST_BINS;
     if (R > m_total) {                         // the sample cannot bound the threshold
         if (t == 0) s.spec_key = 0;            // stage everything: the count check decides
-        p.sample_hist[i * SAMPLE_HIST_BINS + t] = 0;
+#pragma unroll
+        for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) gh[c * BEGIN_BLOCK + t] = 0;
         return;
     }
-    // Largest 24-bit key prefix v with  #(sample keys >= v) >= R.  The top bits come from
-    // the histogram the sampling CTAs filled; the keys that survive (those in the threshold's octave and
-    // above, a few percent) go onto per-warp lists in shared memory and the mantissa bits are
-    // settled on those.  Zero keys never count: every candidate is positive.
-    constexpr int WARP_LIST = 128;
-    constexpr int NW = BEGIN_BLOCK / 32;
-    __shared__ uint32_t s_list[NW * WARP_LIST];
-    __shared__ uint32_t s_cnt[NW];
-    auto count_all = [&](uint32_t cand) {
-        uint32_t c = 0;
+    // Largest key prefix v (a multiple of 2^bound_low_bit) with  #(sample keys >= v) >= R.
+    // The top bits come from the histogram the sampling CTAs filled: thread t looks at bins
+    // BINS-1-4t .. BINS-4-4t, so that the prefix over threads counts the higher bins.
+    uint32_t bound = 0, above = 0;                           // above = #(keys in higher bins)
+    {
+        uint32_t cnt[SAMPLE_BINS_PER_THREAD];
+        uint32_t mine = 0;
 #pragma unroll
-        for (int q = 0; q < SAMPLE_KEYS_PER_THREAD; ++q) c += (keys[q] >= cand) ? 1u : 0u;
-        for (int o = 16; o > 0; o >>= 1) c += __shfl_down_sync(FULL, c, o);
-        if ((t & 31) == 0) s_w[t >> 5] = c;
-        __syncthreads();
-        if (t < 32) {
-            uint32_t v = s_w[t];
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(FULL, v, o);
-            if (t == 0) s_w[32] = v;
+        for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) {
+            const uint32_t hb = SAMPLE_HIST_BINS - 1 - (t * SAMPLE_BINS_PER_THREAD + c);
+            cnt[c] = __ldcg(&gh[hb]);
+            gh[hb] = 0;                                       // ready for the next iteration
+            mine += cnt[c];
+        }
+        uint32_t tot;
+        uint32_t higher = block_excl_scan(mine, s_w, tot);
+        if (t == 0) {
+            s_flag = 0;
+            s_cnt[0] = 0;
         }
         __syncthreads();
-        const uint32_t tot = s_w[32];
-        __syncthreads();
-        return tot;
-    };
-    // top bits of the R-th largest sample key from the histogram; thread t looks at the
-    // mirrored bin so that the prefix over threads counts the higher bins
-    uint32_t bound = 0;
-    {
-        const uint32_t hb = SAMPLE_HIST_BINS - 1 - t;
-        const uint32_t mine_e = __ldcg(&p.sample_hist[i * SAMPLE_HIST_BINS + hb]);
-        p.sample_hist[i * SAMPLE_HIST_BINS + hb] = 0;           // ready for the next iteration
-        uint32_t tot;
-        const uint32_t higher = block_excl_scan(mine_e, s_w, tot);
-        if (t == 0) s_flag = 0;
-        __syncthreads();
-        if (higher < R && higher + mine_e >= R) s_flag = hb << p.sample_shift;
+#pragma unroll
+        for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) {
+            if (higher < R && higher + cnt[c] >= R) {
+                s_flag = (SAMPLE_HIST_BINS - 1 - (t * SAMPLE_BINS_PER_THREAD + c)) << p.sample_shift;
+                s_cnt[0] = higher;
+            }
+            higher += cnt[c];
+        }
         __syncthreads();
         bound = s_flag;
+        above = s_cnt[0];
         __syncthreads();
     }
+    // The sample keys of that bin go onto per-warp lists in shared memory and the remaining
+    // bits are settled on those.  Zero keys never count: every candidate is positive.
     const int lane = t & 31, w = t >> 5;
+    const uint32_t bin_end = bound + (1u << p.sample_shift);    // no overflow: keys have 31 bits
+    const int parts = static_cast<int>((S + BEGIN_BLOCK - 1) / BEGIN_BLOCK);
     uint32_t mine = 0;                                       // warp-uniform running count
+    for (int q0 = 0; q0 < parts; q0 += 4) {
+        uint4 v[4];
 #pragma unroll
-    for (int q = 0; q < SAMPLE_KEYS_PER_THREAD; ++q) {
-        const bool keep = keys[q] >= bound && keys[q] != 0;
-        const uint32_t m = __ballot_sync(FULL, keep);
-        const uint32_t at = mine + __popc(m & ((1u << lane) - 1u));
-        if (keep && at < WARP_LIST) s_list[w * WARP_LIST + at] = keys[q];
-        mine += __popc(m);
+        for (int q = 0; q < 4; ++q)
+            v[q] = q0 + q < parts ? __ldcg(skeys + (q0 + q) * BEGIN_BLOCK + t) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t ks[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const bool keep = ks[c] >= bound && ks[c] < bin_end && ks[c] != 0;
+                const uint32_t m = __ballot_sync(FULL, keep);
+                if (m == 0) continue;
+                const uint32_t at = mine + __popc(m & ((1u << lane) - 1u));
+                if (keep && at < SAMPLE_WARP_LIST) s_buf[w * SAMPLE_WARP_LIST + at] = ks[c];
+                mine += __popc(m);
+            }
+        }
     }
     if (lane == 0) s_cnt[w] = mine;
     __syncthreads();
     uint32_t longest = 0;
 #pragma unroll
     for (int ww = 0; ww < NW; ++ww) longest = max(longest, s_cnt[ww]);
-    const bool fits = longest <= WARP_LIST;
-    const int rounds = (longest + 31) / 32;                  // same for every thread
-    // everything >= bound is on the lists, so counts over the lists equal counts over the
-    // sample for any candidate >= bound; lane l of warp w looks at slots l, l+32, ...
-#pragma unroll 1
-    for (int bit = static_cast<int>(p.sample_shift) - 1; bit >= static_cast<int>(p.bound_low_bit); --bit) {
-        const uint32_t cand = bound | (1u << bit);
-        uint32_t tot = 0;
-        if (fits) {
-            for (int r = 0; r < rounds; ++r) {
-                const uint32_t slot = r * 32 + lane;
-                tot += __syncthreads_count(slot < mine && s_list[w * WARP_LIST + slot] >= cand);
+    __syncthreads();
+    const int nbits = static_cast<int>(p.sample_shift) - static_cast<int>(p.bound_low_bit);
+    if (longest <= SAMPLE_WARP_LIST) {
+        // two rounds of a 64-bin histogram over the listed keys settle the remaining bits
+        __shared__ uint32_t s_h[64];
+        const uint32_t listed = min(mine, static_cast<uint32_t>(SAMPLE_WARP_LIST));
+        uint32_t settled = 0;                                // bits below sample_shift, settled so far
+        int done_bits = 0;
+        for (int round = 0; round < 2; ++round) {
+            const int take = round == 0 ? nbits - 6 : 6;      // nbits is 11 or 12
+            const int low = static_cast<int>(p.sample_shift) - done_bits - take;
+            if (t < 64) s_h[t] = 0;
+            __syncthreads();
+            for (uint32_t slot = lane; slot < listed; slot += 32) {
+                const uint32_t sub = s_buf[w * SAMPLE_WARP_LIST + slot] - bound;
+                // keys that agree with the bits settled so far
+                if (done_bits == 0 || (sub >> (low + take)) == (settled >> (low + take)))
+                    atomicAdd(&s_h[(sub >> low) & ((1u << take) - 1u)], 1u);
             }
-        } else {
-            tot = count_all(cand);
+            __syncthreads();
+            if (t == 0) {
+                uint32_t acc = above;
+                int pick = 0;
+                for (int bnum = (1 << take) - 1; bnum >= 0; --bnum) {
+                    if (acc + s_h[bnum] >= R) {
+                        pick = bnum;
+                        break;
+                    }
+                    acc += s_h[bnum];
+                }
+                s_w[0] = static_cast<uint32_t>(pick);
+                s_w[1] = acc;
+            }
+            __syncthreads();
+            settled |= s_w[0] << low;
+            above = s_w[1];
+            done_bits += take;
+            __syncthreads();
         }
-        if (tot >= R) bound = cand;
+        bound += settled;
+    } else {
+        // a list overflowed (very many sample keys in one bin): settle the bits one by one with
+        // counts over the whole sample
+#pragma unroll 1
+        for (int bit = static_cast<int>(p.sample_shift) - 1; bit >= static_cast<int>(p.bound_low_bit); --bit) {
+            const uint32_t cand = bound | (1u << bit);
+            uint32_t c = 0;
+            for (int q = 0; q < parts; ++q) {
+                const uint4 v = __ldcg(skeys + q * BEGIN_BLOCK + t);
+                c += (v.x >= cand) + (v.y >= cand) + (v.z >= cand) + (v.w >= cand);
+            }
+            uint32_t all;
+            (void)block_excl_scan(c, s_w, all);
+            if (all >= R) bound = cand;
+        }
     }
     if (t == 0) {
-        s.spec_key = bound;                    // a multiple of 128: lower edge of a 24-bit bin
+        s.spec_key = bound;                    // lower edge of a 2^bound_low_bit-wide key bin
         s.rel_shift = rel_shift;
     }
 }
@@ -1594,7 +1657,8 @@ Sel make_sel(const deco_ctx *c)
     p.work_cap = c->work_cap;
     p.status = c->dev_status;
     p.rk = make_rand(c);
-    p.sample_shift = p.rk.on ? 13u : static_cast<uint32_t>(SAMPLE_HIST_SHIFT);
+    // Top-k keys have 31 bits, Random-k priorities 23
+    p.sample_shift = (p.rk.on ? 23u : 31u) - SAMPLE_HIST_BITS;
     p.bound_low_bit = p.rk.on ? 0u : 7u;
     return p;
 }
@@ -1618,11 +1682,13 @@ cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s)
 {
     const float alpha = c->lr_at_server ? 1.0f : c->lr;
     const uint32_t exact_all = streaming_route(c) ? 0u : 1u;
-    const dim3 grid(SAMPLE_CTAS, c->n);
+    // one CTA per BEGIN_BLOCK sample groups
+    const uint32_t S = sample_groups(c->d, c->k);
+    const dim3 grid((S + BEGIN_BLOCK - 1) / BEGIN_BLOCK, c->n);
     if (c->grad_dtype == DECO_BF16)
-        begin_step_kernel<1><<<grid, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
+        begin_step_kernel<1><<<grid, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all, S);
     else
-        begin_step_kernel<0><<<grid, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all);
+        begin_step_kernel<0><<<grid, BEGIN_BLOCK, 0, s>>>(make_sel(c), grads, alpha, exact_all, S);
     c->launches += 1;
     return cudaGetLastError();
 }

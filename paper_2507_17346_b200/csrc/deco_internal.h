@@ -52,7 +52,8 @@ constexpr uint32_t SPEC_DISABLED = 0x80000000u;   // above every 31-bit key
 constexpr uint32_t CHUNK_TILES = 32;
 
 // Keys of the per-iteration sample kept per worker (8192 groups of 4 entries).
-constexpr uint32_t SAMPLE_KEYS = 32768;
+constexpr uint32_t SAMPLE_KEYS = 131072;
+constexpr uint32_t SAMPLE_BINS = 4096;                  // bins of the sample histogram
 
 struct Slot {
     uint64_t step = 0;
@@ -93,7 +94,7 @@ struct deco_ctx {
     uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
     uint32_t *done = nullptr;           // [n][DONE_SLOTS] CTA arrival counters
     uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
-    uint32_t *sample_hist = nullptr;    // [n][1024] sample keys per top-10-bit bin (self-clearing)
+    uint32_t *sample_hist = nullptr;    // [n][SAMPLE_BINS] sample keys per bin of their top bits (self-clearing)
     uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
     deco::SelectState *sel = nullptr;   // [n]
     uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
