@@ -179,6 +179,42 @@ def test_sparse_messages_take_every_aggregation_path(n):
     assert st["device_status"] == 0
 
 
+@pytest.mark.parametrize("seed", [11, 12, 13, 14])
+def test_seeded_random_configurations(seed):
+    """Shapes, worker counts, densities, staleness, dtypes and value structure drawn from a seeded
+    generator: every draw must match the oracle bit for bit like the hand-picked cases."""
+    rng = np.random.default_rng(seed)
+    for _ in range(8):
+        d = int(rng.choice([rng.integers(1, 3000), rng.integers(3000, 70_000),
+                            rng.integers(70_000, 400_000)]))
+        n = int(rng.integers(1, 25))
+        delta = float(min(1.0, 10.0 ** rng.uniform(-4, 0.1)))
+        tau = int(rng.integers(0, 4))
+        dtype, name = ((torch.float32, "f32"), (torch.bfloat16, "bf16"))[int(rng.integers(0, 2))]
+        kind = str(rng.choice(["normal", "coarse", "hot", "shared"]))
+        hot_lo = int(rng.integers(0, d))
+        hot_hi = min(d, hot_lo + int(rng.integers(1, 20_000)))
+        case_seed = int(rng.integers(0, 1 << 30))
+        delta2 = float(min(1.0, 10.0 ** rng.uniform(-4, 0.1)))
+
+        def grads(t):
+            g = torch.Generator(device="cuda")
+            g.manual_seed(case_seed + t)
+            if kind == "coarse":
+                x = torch.randint(-8, 9, (n, d), generator=g, device="cuda").float() / 8.0
+            else:
+                x = torch.randn((n, d), generator=g, device="cuda")
+            if kind == "shared":                                  # workers agree on the large entries
+                x = x[:1] * (1.0 + 0.1 * x)
+            if kind in ("hot", "shared"):
+                x[:, hot_lo:hot_hi] *= 30.0
+            return x.to(dtype).contiguous()
+
+        dmax = max(delta, delta2)
+        run_parity(d, n, delta, tau, 0.1, grads, steps=4, grad_dtype=name,
+                   policy_plan={2: (delta2, int(rng.integers(0, 4)))}, tau_max=3, delta_max=dmax)
+
+
 @pytest.mark.parametrize("mode", MODES)
 def test_random_k_sparsifier(mode):
     """Random-k in place of Top-k: the same Philox priorities on both sides give the same index
