@@ -330,8 +330,8 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "ef_accumulate_kernel", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
-                "traffic": NCU_TRAFFIC_BYTES.get(wl.name) if args.scale == 1.0 and args.compressor == "topk" else None
-                if (args.delta is None and args.compressor == "topk") else None,
+                "traffic": NCU_TRAFFIC_BYTES.get(wl.name)
+                if (args.scale == 1.0 and args.delta is None and args.compressor == "topk") else None,
                 "algorithmic_bytes_per_launch": algorithmic_bytes_accumulate(wl),
                 "avg_launch_ms": acc_ms, "launches_timed": iters}
     step_alg_bytes = algorithmic_bytes_accumulate(wl)

@@ -308,6 +308,58 @@ deco_status deco_get_kernel_timing(deco_ctx *ctx, void *stream, double *ms_sum /
 /* Number of kernels and memset/memcpy nodes the library has enqueued so far. */
 uint64_t deco_launch_count(const deco_ctx *ctx);
 
+/* ------------------------------------------------------------- per-layer Top-k (variant) */
+
+/*
+ * The paper applies "Top-k ... to gradients" (Section 5, implementation) without saying whether
+ * k counts over the whole model or per tensor; the contexts above take the whole flat vector.
+ * This variant takes it per layer: the vector is cut into n_layers ranges
+ * [layer_offsets[l], layer_offsets[l+1]) and C_delta keeps, for every worker, the
+ * k_l = k(delta, d_l) largest entries of each range (ties by increasing index).  Nothing else in
+ * Algorithm 1 couples entries of different layers, so a layered context is a batch of ordinary
+ * contexts, one per layer, sharing policy, stepsize, gradient buffer and parameter vector.
+ *   layer_offsets  HOST, [n_layers + 1], strictly increasing, first 0, last d
+ *   opt            as for deco_init; opt->params (DEVICE, [d], 16-byte aligned) or NULL;
+ *                  tau_max and delta_max apply to every layer
+ * Random-k: layer l uses seed + l.
+ */
+typedef struct deco_layered deco_layered;
+deco_status deco_layered_init(deco_layered **out, uint64_t d, uint32_t n,
+                              const uint64_t *layer_offsets, uint32_t n_layers, double delta,
+                              uint32_t tau, float lr, const deco_options *opt);
+
+/* Frees the layered context and every layer's context (waits for the device first). */
+void deco_layered_destroy(deco_layered *ctx);
+
+/*
+ * One iteration of every layer (deco_step per layer).  grads: DEVICE, [n][d] row-major, dtype =
+ * grad_dtype, 16-byte aligned base.  The layers run round-robin on internal streams forked
+ * from `stream` at the start of the call and joined back at its end; like deco_step, each
+ * layer may leave its aggregation running (deco_layered_join orders `stream` after them).
+ * The first error of a layer is returned; layers after it are not stepped.
+ */
+deco_status deco_layered_step(deco_layered *ctx, const void *grads, void *stream);
+deco_status deco_layered_join(deco_layered *ctx, void *stream);
+
+/* deco_set_policy / deco_set_lr for all layers; the policy changes all layers or none
+ * (DECO_ERR_CAPACITY if any layer lacks the capacity). */
+deco_status deco_layered_set_policy(deco_layered *ctx, double delta, uint32_t tau);
+deco_status deco_layered_set_lr(deco_layered *ctx, float lr);
+
+/*
+ * The context of one layer, for the getters above (deco_get_k, deco_get_buffers,
+ * deco_get_aggregate, deco_get_stats, ...): its indices are relative to the layer's offset.
+ * It stays owned by the layered context: do not destroy it and do not step it on its own.
+ * Every out pointer may be NULL.
+ */
+deco_status deco_layered_layer(deco_layered *ctx, uint32_t layer, deco_ctx **layer_ctx,
+                               uint64_t *offset, uint64_t *length);
+
+/* Number of layers, sum of the layers' k, the parameter vector (DEVICE, [d]) and the number of
+ * completed iterations.  Every out pointer may be NULL. */
+deco_status deco_layered_info(deco_layered *ctx, uint32_t *n_layers, uint64_t *k_total,
+                              float **params, uint64_t *step);
+
 /*
  * Top-k compression of one vector without any allocation.  (The paper has no counterpart:
  * this entry point exists for callers that cannot allocate device memory at the moment they

@@ -13,7 +13,8 @@ Readings taken where the paper is silent (each is also listed in the design note
   * "largest" is by |a|, compared through the IEEE-754 bit pattern with the sign cleared;
     among equal magnitudes the lower index wins;
   * k = ceil(delta * d), clamped to [1, d] (the Top-k contraction lemma needs k/d >= delta);
-  * Top-k is global over the flat length-d vector;
+  * Top-k is global over the flat length-d vector; the per-layer variant (`layer_offsets`)
+    keeps k(delta, d_l) entries in each range [offset_l, offset_{l+1}) instead;
   * iterations are numbered from 0 and update t applies the aggregate of step t - tau iff
     t - tau >= 0 (the paper's "g_{t-tau} = e_{t-tau} = 0 if t - tau <= 0" boundary);
   * when tau changes between steps the server drains its cache exactly once, oldest first:
@@ -84,6 +85,16 @@ def topk_select(a, k):
     return sel
 
 
+def topk_select_per_layer(a, layer_offsets, delta):
+    """Per-layer variant of C_delta: the k(delta, d_l) largest-|a| entries of every range
+    [layer_offsets[l], layer_offsets[l+1]), same tie rule inside a range.  Indices ascending."""
+    parts = []
+    for lo, hi in zip(layer_offsets[:-1], layer_offsets[1:]):
+        lo, hi = int(lo), int(hi)
+        parts.append(topk_select(a[lo:hi], k_from_delta(delta, hi - lo)).astype(np.uint64) + lo)
+    return np.concatenate(parts).astype(np.uint32)
+
+
 def compress(a, k, sel=None):
     """C_delta(a) as (indices ascending, values) and the residual a - C_delta(a).  `sel`
     overrides the Top-k choice (Random-k passes its own index set)."""
@@ -118,14 +129,18 @@ class DDEFSGD:
     False moves the stepsize to the server (a = e + g, update scale gamma/n)."""
 
     def __init__(self, d, n, delta, tau, lr, x0=None, lr_in_compress=True, compressor="topk",
-                 seed=0):
+                 seed=0, layer_offsets=None):
         self.d, self.n = int(d), int(n)
+        self.layer_offsets = None if layer_offsets is None else [int(v) for v in layer_offsets]
+        if self.layer_offsets is not None:
+            assert compressor == "topk" and self.layer_offsets[0] == 0
+            assert self.layer_offsets[-1] == self.d
         self.lr = np.float32(lr)
         self.lr_in_compress = bool(lr_in_compress)
         assert compressor in ("topk", "randk")
         self.compressor, self.seed = compressor, int(seed)
         self.delta, self.tau = float(delta), int(tau)
-        self.k = k_from_delta(delta, d)
+        self.k = self._k_of(delta)
         self.x = (np.zeros(d, np.float32) if x0 is None
                   else np.array(x0, dtype=np.float32, copy=True))
         self.x64 = self.x.astype(np.float64)
@@ -133,10 +148,17 @@ class DDEFSGD:
         self.cache = []                                   # server cache: (step, S, S64), FIFO
         self.t = 0
 
+    def _k_of(self, delta):
+        """Entries per message: k(delta, d), or the sum of the layers' k(delta, d_l)."""
+        if self.layer_offsets is None:
+            return k_from_delta(delta, self.d)
+        return sum(k_from_delta(delta, hi - lo)
+                   for lo, hi in zip(self.layer_offsets[:-1], self.layer_offsets[1:]))
+
     def set_policy(self, delta, tau):
         """New (delta, tau) from the next iteration on (Algorithm 2's broadcast)."""
         self.delta, self.tau = float(delta), int(tau)
-        self.k = k_from_delta(delta, self.d)
+        self.k = self._k_of(delta)
 
     def set_lr(self, lr):
         self.lr = np.float32(lr)
@@ -156,6 +178,8 @@ class DDEFSGD:
             if self.compressor == "randk":
                 from . import random_k
                 chosen = random_k.randk_select(d, self.k, self.seed, self.t, i)
+            elif self.layer_offsets is not None:
+                chosen = topk_select_per_layer(a, self.layer_offsets, self.delta)
             sel, vals, resid = compress(a, self.k, chosen)
             self.e[i] = resid
             msgs.append((sel, vals))

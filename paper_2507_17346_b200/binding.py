@@ -108,6 +108,14 @@ SIGNATURES = {
     "deco_import_state": (_i32, [_vp, _vp, _u64, _vp]),
     "deco_launch_count": (_u64, [_vp]),
     "deco_topk_compress_static": (_i32, [_vp, _u64, _u64, _vp, _vp]),
+    "deco_layered_init": (_i32, [_P(_vp), _u64, _u32, _P(_u64), _u32, _f64, _u32, _f32, _vp]),
+    "deco_layered_destroy": (None, [_vp]),
+    "deco_layered_step": (_i32, [_vp, _vp, _vp]),
+    "deco_layered_join": (_i32, [_vp, _vp]),
+    "deco_layered_set_policy": (_i32, [_vp, _f64, _u32]),
+    "deco_layered_set_lr": (_i32, [_vp, _f32]),
+    "deco_layered_layer": (_i32, [_vp, _u32, _P(_vp), _P(_u64), _P(_u64)]),
+    "deco_layered_info": (_i32, [_vp, _P(_u32), _P(_u64), _P(_vp), _P(_u64)]),
     "deco_status_string": (ctypes.c_char_p, [_i32]),
 }
 
@@ -160,10 +168,8 @@ def _stream(stream):
 
 # ------------------------------------------------------------------ entry points
 
-def deco_init(d, n, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0, delta_max=0.0,
-              lr_at_server=False, params=None, device=0, select_mode=DECO_SELECT_AUTO,
-              compressor=DECO_COMPRESSOR_TOPK, seed=0):
-    """-> opaque context handle (int).  `params`: optional fp32 CUDA tensor of length d."""
+def _options(grad_dtype, tau_max, delta_max, lr_at_server, params, device, select_mode,
+             compressor, seed):
     opt = deco_options()
     opt.grad_dtype = grad_dtype
     opt.tau_max = tau_max
@@ -175,10 +181,67 @@ def deco_init(d, n, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0, delta_max=0.
     opt.compressor = compressor
     opt.seed_lo = seed & 0xFFFFFFFF
     opt.seed_hi = (seed >> 32) & 0xFFFFFFFF
+    return opt
+
+
+def deco_init(d, n, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0, delta_max=0.0,
+              lr_at_server=False, params=None, device=0, select_mode=DECO_SELECT_AUTO,
+              compressor=DECO_COMPRESSOR_TOPK, seed=0):
+    """-> opaque context handle (int).  `params`: optional fp32 CUDA tensor of length d."""
+    opt = _options(grad_dtype, tau_max, delta_max, lr_at_server, params, device, select_mode,
+                   compressor, seed)
     ctx = _vp()
     _check(load().deco_init(ctypes.byref(ctx), d, n, delta, tau, lr, ctypes.byref(opt)),
            "deco_init")
     return ctx.value
+
+
+def deco_layered_init(d, n, layer_offsets, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0,
+                      delta_max=0.0, lr_at_server=False, params=None, device=0,
+                      select_mode=DECO_SELECT_AUTO, compressor=DECO_COMPRESSOR_TOPK, seed=0):
+    """Per-layer Top-k: `layer_offsets` = [0, ..., d] (len = layers + 1).  -> opaque handle."""
+    opt = _options(grad_dtype, tau_max, delta_max, lr_at_server, params, device, select_mode,
+                   compressor, seed)
+    offs = (_u64 * len(layer_offsets))(*[int(x) for x in layer_offsets])
+    ctx = _vp()
+    _check(load().deco_layered_init(ctypes.byref(ctx), d, n, offs, len(layer_offsets) - 1, delta,
+                                    tau, lr, ctypes.byref(opt)), "deco_layered_init")
+    return ctx.value
+
+
+def deco_layered_destroy(ctx):
+    load().deco_layered_destroy(ctx)
+
+
+def deco_layered_step(ctx, grads, stream=None):
+    _check(load().deco_layered_step(ctx, _ptr(grads), _stream(stream)), "deco_layered_step")
+
+
+def deco_layered_join(ctx, stream=None):
+    _check(load().deco_layered_join(ctx, _stream(stream)), "deco_layered_join")
+
+
+def deco_layered_set_policy(ctx, delta, tau):
+    _check(load().deco_layered_set_policy(ctx, delta, tau), "deco_layered_set_policy")
+
+
+def deco_layered_set_lr(ctx, lr):
+    _check(load().deco_layered_set_lr(ctx, lr), "deco_layered_set_lr")
+
+
+def deco_layered_layer(ctx, layer):
+    """-> (layer context handle, offset, length); the handle works with every deco_get_*."""
+    c, off, ln = _vp(), _u64(), _u64()
+    _check(load().deco_layered_layer(ctx, layer, ctypes.byref(c), ctypes.byref(off),
+                                     ctypes.byref(ln)), "deco_layered_layer")
+    return c.value, off.value, ln.value
+
+
+def deco_layered_info(ctx):
+    nl, kt, pp, st = _u32(), _u64(), _vp(), _u64()
+    _check(load().deco_layered_info(ctx, ctypes.byref(nl), ctypes.byref(kt), ctypes.byref(pp),
+                                    ctypes.byref(st)), "deco_layered_info")
+    return {"n_layers": nl.value, "k_total": kt.value, "params": pp.value, "step": st.value}
 
 
 def deco_destroy(ctx):

@@ -142,7 +142,14 @@ extern "C" const char *deco_status_string(deco_status s)
 extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double delta,
                                  uint32_t tau, float lr, const deco_options *opt)
 {
+    return deco::init_context(out, d, n, delta, tau, lr, opt, 0);
+}
+
+deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double delta, uint32_t tau,
+                               float lr, const deco_options *opt, uint64_t g_stride)
+{
     if (!out) return DECO_ERR_INVALID_ARG;
+    if (g_stride != 0 && g_stride < d) return DECO_ERR_INVALID_ARG;
     deco_options o;
     std::memset(&o, 0, sizeof o);
     if (opt) o = *opt;
@@ -159,7 +166,7 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
         return DECO_ERR_INVALID_ARG;
     if (o.tau_max != 0 && o.tau_max < tau) return DECO_ERR_INVALID_ARG;
     if (o.tau_max > (1u << 20) || tau > (1u << 20)) return DECO_ERR_INVALID_ARG;
-    if (o.params && (reinterpret_cast<uintptr_t>(o.params) & 15u)) return DECO_ERR_INVALID_ARG;
+    if (o.params && (reinterpret_cast<uintptr_t>(o.params) & (g_stride ? 3u : 15u))) return DECO_ERR_INVALID_ARG;
 
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) {
@@ -173,6 +180,7 @@ extern "C" deco_status deco_init(deco_ctx **out, uint64_t d, uint32_t n, double 
     deco_ctx *c = new (std::nothrow) deco_ctx();
     if (!c) return DECO_ERR_OOM;
     c->d = d;
+    c->g_stride = g_stride ? g_stride : d;
     c->n = n;
     c->delta = delta;
     c->delta_max = o.delta_max != 0.0 ? o.delta_max : delta;
@@ -276,7 +284,7 @@ extern "C" deco_status deco_reset(deco_ctx *c, void *stream)
 extern "C" deco_status deco_ef_compress(deco_ctx *c, const void *grads, void *stream)
 {
     if (!c || !grads) return DECO_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(grads) & 15u) return DECO_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(grads) & (c->g_stride != c->d ? 1u : 15u)) return DECO_ERR_INVALID_ARG;
     if (c->phase != 0) return DECO_ERR_STATE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
@@ -409,7 +417,7 @@ extern "C" deco_status deco_step(deco_ctx *c, const void *grads, void *stream)
     // pass.  It is forked from and joined back into the caller's stream inside this call: e,
     // the messages and the parameters are complete, in stream order, when the caller's stream
     // passes the call.
-    if (reinterpret_cast<uintptr_t>(grads) & 15u) return DECO_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(grads) & (c->g_stride != c->d ? 1u : 15u)) return DECO_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);

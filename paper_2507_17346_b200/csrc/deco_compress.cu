@@ -81,6 +81,7 @@ struct Sel {
     float *e;
     uint64_t e_stride;
     uint64_t d;
+    uint64_t g_stride;       // entries between gradient rows
     uint32_t n;
     uint32_t ntiles;
     uint32_t k;
@@ -371,7 +372,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     __shared__ uint32_t s_flag;
     const float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     const char *grow = reinterpret_cast<const char *>(grads) +
-                       static_cast<size_t>(i) * p.d * (GT ? 2 : 4);
+                       static_cast<size_t>(i) * p.g_stride * (GT ? 2 : 4);
     const uint64_t nchunks = (p.d + 3) >> 2;
     uint4 *skeys = reinterpret_cast<uint4 *>(p.sample_keys) + static_cast<size_t>(i) * SAMPLE_CHUNKS;
     {
@@ -580,7 +581,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
 template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
 __global__ void __launch_bounds__(BLOCK)
 ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
-                     uint64_t d, float alpha, RandParams rk, SelectState *__restrict__ sel,
+                     uint64_t d, uint64_t g_stride, float alpha, RandParams rk, SelectState *__restrict__ sel,
                      deco_pair *__restrict__ stage, uint64_t stage_cap,
                      uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
                      uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
@@ -591,7 +592,7 @@ ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__res
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     float *erow = e + static_cast<size_t>(i) * e_stride;
     const char *grow = reinterpret_cast<const char *>(grads) +
-                       static_cast<size_t>(i) * d * (GT ? 2 : 4);
+                       static_cast<size_t>(i) * g_stride * (GT ? 2 : 4);
     const uint64_t tile_base = static_cast<uint64_t>(tile) * TILE;
     const uint64_t wbase = tile_base + static_cast<uint64_t>(w) * WARP_ELEMS;
     const bool full = ALIGNED && (tile_base + TILE <= d);
@@ -1628,6 +1629,7 @@ Sel make_sel(const deco_ctx *c)
     p.e = c->e;
     p.e_stride = c->e_stride;
     p.d = c->d;
+    p.g_stride = c->g_stride;
     p.n = c->n;
     p.ntiles = c->ntiles;
     p.k = static_cast<uint32_t>(c->k);
@@ -1698,7 +1700,7 @@ static void launch_acc_variant(deco_ctx *c, const void *grads, float alpha, cuda
 {
     dim3 grid(c->ntiles, c->n);
     ef_accumulate_kernel<GT, ALIGNED, SPEC, RANDK><<<grid, BLOCK, 0, s>>>(
-        c->e, c->e_stride, grads, c->d, alpha, make_rand(c), c->sel, c->stage, c->stage_cap,
+        c->e, c->e_stride, grads, c->d, c->g_stride, alpha, make_rand(c), c->sel, c->stage, c->stage_cap,
         c->tile_off, c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
 }
 
@@ -1718,8 +1720,9 @@ static void launch_acc(deco_ctx *c, const void *grads, float alpha, cudaStream_t
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s)
 {
     const float alpha = c->lr_at_server ? 1.0f : c->lr;
-    const uint64_t row_bytes = c->d * (c->grad_dtype == DECO_BF16 ? 2 : 4);
-    const bool aligned = (c->n == 1) || (row_bytes % 16 == 0);
+    const uint64_t row_bytes = c->g_stride * (c->grad_dtype == DECO_BF16 ? 2 : 4);
+    const bool aligned = (reinterpret_cast<uintptr_t>(grads) % 16 == 0) &&
+                         ((c->n == 1) || (row_bytes % 16 == 0));
     if (c->grad_dtype == DECO_BF16) {
         if (aligned) launch_acc<1, true>(c, grads, alpha, s);
         else launch_acc<1, false>(c, grads, alpha, s);

@@ -76,6 +76,9 @@ struct deco_ctx {
     int compressor = DECO_COMPRESSOR_TOPK;
     uint64_t seed = 0;                  // Random-k: key of the priority stream
     int device = 0;
+    // entries between consecutive gradient rows: d, or the full vector length when the context
+    // works on one layer of a longer vector (then the rows need not be 16-byte aligned)
+    uint64_t g_stride = 0;
     // derived
     uint64_t k = 0, k_cap = 0;
     uint64_t e_stride = 0;      // floats per worker row of e (multiple of TILE)
@@ -141,6 +144,10 @@ cudaError_t query_fallback_grid(deco_ctx *c);
 cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s);
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s);
 cudaError_t launch_selection(deco_ctx *c, cudaStream_t s);
+
+// deco_init with the distance between gradient rows given (0: d)
+deco_status init_context(deco_ctx **out, uint64_t d, uint32_t n, double delta, uint32_t tau, float lr,
+                         const deco_options *opt, uint64_t g_stride);
 
 // Order stream s after the aggregation that deco_step left running on the internal stream.
 inline cudaError_t wait_for_aggregate(deco_ctx *c, cudaStream_t s)

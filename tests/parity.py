@@ -127,3 +127,61 @@ def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mo
         return st
     finally:
         B.deco_destroy(ctx)
+
+
+def run_layered_parity(layer_offsets, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32",
+                       policy_plan=None, tau_max=0, delta_max=0.0, device=0):
+    """Per-layer Top-k: the layered context (one library context per layer, stepped together)
+    against the oracle's per-layer variant, which keeps one flat state and only selects per
+    range.  Messages, residuals, aggregates and parameters must agree bit for bit."""
+    d = int(layer_offsets[-1])
+    ctx = B.deco_layered_init(d, n, layer_offsets, delta, tau, lr,
+                              grad_dtype=B.DECO_F32 if grad_dtype == "f32" else B.DECO_BF16,
+                              tau_max=tau_max, delta_max=delta_max, device=device)
+    try:
+        orc = O.DDEFSGD(d, n, delta, tau, lr, layer_offsets=layer_offsets)
+        info = B.deco_layered_info(ctx)
+        assert info["n_layers"] == len(layer_offsets) - 1 and info["k_total"] == orc.k
+        layers = [B.deco_layered_layer(ctx, l) for l in range(info["n_layers"])]
+        for t in range(steps):
+            if policy_plan and t in policy_plan:
+                B.deco_layered_set_policy(ctx, *policy_plan[t])
+                orc.set_policy(*policy_plan[t])
+                assert B.deco_layered_info(ctx)["k_total"] == orc.k
+            g = grad_fn(t)
+            ref = orc.step(W.to_numpy_bits(g))
+            B.deco_layered_step(ctx, g)
+            torch.cuda.synchronize()
+            idx_parts = [[] for _ in range(n)]
+            val_parts = [[] for _ in range(n)]
+            agg_idx, agg_val = [], []
+            for sub, off, ln in layers:
+                k_l = B.deco_get_k(sub)
+                idx, val = read_messages(sub, n, k_l, device)
+                for i in range(n):
+                    idx_parts[i].append(idx[i].astype(np.uint64) + off)
+                    val_parts[i].append(val[i])
+                e = read_e(sub, n, ln, device)
+                assert np.array_equal(bits(e), bits(orc.e[:, off:off + ln])), \
+                    "step %d layer at %d: residual" % (t, off)
+                aidx, aval = read_aggregate(sub, t, device)
+                agg_idx.append(aidx.astype(np.uint64) + off)
+                agg_val.append(aval)
+            for i, (sel, vals) in enumerate(ref["msgs"]):
+                assert np.array_equal(np.concatenate(idx_parts[i]), sel.astype(np.uint64)), \
+                    "step %d worker %d: index set" % (t, i)
+                assert np.array_equal(bits(np.concatenate(val_parts[i])), bits(vals)), \
+                    "step %d worker %d: message values" % (t, i)
+            touched = np.unique(np.concatenate([s for s, _ in ref["msgs"]]))
+            assert np.array_equal(np.concatenate(agg_idx), touched.astype(np.uint64)), \
+                "step %d: aggregate index set" % t
+            assert np.array_equal(bits(np.concatenate(agg_val)), bits(ref["S"][touched])), \
+                "step %d: aggregate" % t
+            x = B.view_f32(info["params"], (d,), device).cpu().numpy()
+            assert np.array_equal(bits(x), bits(orc.x)), "step %d: parameters" % t
+        for sub, _, _ in layers:
+            st = B.deco_get_stats(sub)
+            assert st["device_status"] == 0 and st["step"] == steps
+        assert B.deco_layered_info(ctx)["step"] == steps
+    finally:
+        B.deco_layered_destroy(ctx)

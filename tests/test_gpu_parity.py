@@ -6,7 +6,7 @@ import torch
 
 from paper_2507_17346_b200 import binding as B
 from paper_2507_17346_b200 import workloads as W
-from tests.parity import run_parity
+from tests.parity import run_layered_parity, run_parity
 
 pytestmark = pytest.mark.gpu
 
@@ -213,6 +213,28 @@ def test_seeded_random_configurations(seed):
         dmax = max(delta, delta2)
         run_parity(d, n, delta, tau, 0.1, grads, steps=4, grad_dtype=name,
                    policy_plan={2: (delta2, int(rng.integers(0, 4)))}, tau_max=3, delta_max=dmax)
+
+
+def test_per_layer_topk_variant():
+    """Top-k per tensor instead of over the flat vector: tiny tensors (k_l = 1), tensors that
+    start at odd offsets (gradient rows of a layer are then not 16-byte aligned), a loud layer,
+    a policy change; fp32 and bf16 gradients."""
+    wl = W.make_workload("resnet18", 0.125)                  # 62 tensors, ResNet-18 structure
+    offsets = [0]
+    for t in wl.tensors:
+        offsets.append(offsets[-1] + int(t.numel))
+    assert offsets[-1] == wl.d
+    run_layered_parity(offsets, 3, 0.01, 2, 0.1, lambda t: W.gradients(wl, t, "cuda")[:3].contiguous(),
+                       steps=4, policy_plan={2: (0.03, 1)}, tau_max=2, delta_max=0.03)
+    odd = [0, 1, 4, 1001, 1002, 30_003, 100_000, 100_007]
+    for dtype, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        def grads(t):
+            g = torch.Generator(device="cuda")
+            g.manual_seed(900 + t)
+            x = torch.randn((4, odd[-1]), generator=g, device="cuda")
+            x[:, 4:1001] *= 40.0
+            return x.to(dtype).contiguous()
+        run_layered_parity(odd, 4, 0.02, 1, 0.1, grads, steps=4, grad_dtype=name)
 
 
 @pytest.mark.parametrize("mode", MODES)
