@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--delta", type=float, default=None)
     ap.add_argument("--tau", type=int, default=None)
     ap.add_argument("--compressor", default="topk", choices=["topk", "randk"])
+    ap.add_argument("--shard-workers", action="store_true",
+                    help="N > 1: split the workers over the ranks (sparse all-gather per step) "
+                         "instead of running N replicas; strong scaling")
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink the workload's layer widths (profiling captures of the large shapes)")
     return ap.parse_args()
@@ -252,15 +255,29 @@ def run_ours(args):
     pool_n = args.pool if args.pool > 0 else max(2, min(8, int(6e9 // gbytes)))
     pool = [W.gradients(wl, p, "cuda") for p in range(pool_n)]
     mode = B.DECO_SELECT_AUTO if args.select_mode == "auto" else B.DECO_SELECT_EXACT_PASSES
-    ctx = B.deco_init(wl.d, wl.n, wl.delta, wl.tau, wl.lr,
+    sharded = args.shard_workers and world > 1
+    n_local, base = wl.n, 0
+    if sharded:
+        if wl.n % world:
+            raise SystemExit("--shard-workers needs the worker count to be a multiple of --gpus")
+        n_local, base = wl.n // world, rank * (wl.n // world)
+        pool = [p[base:base + n_local].clone() for p in pool]      # this rank's workers only
+    ctx = B.deco_init(wl.d, n_local, wl.delta, wl.tau, wl.lr,
                       grad_dtype=B.DECO_F32 if wl.grad_dtype == "f32" else B.DECO_BF16,
                       device=local, select_mode=mode,
                       compressor=B.DECO_COMPRESSOR_RANDK if args.compressor == "randk"
-                      else B.DECO_COMPRESSOR_TOPK, seed=wl.seed)
+                      else B.DECO_COMPRESSOR_TOPK, seed=wl.seed,
+                      n_total=wl.n if sharded else 0, worker_base=base)
     stream = torch.cuda.current_stream()
 
+    def one_step(g):
+        if sharded:
+            B.deco_step_sharded(ctx, g, None, stream, local)
+        else:
+            B.deco_step(ctx, g, stream)
+
     for t in range(warmup):
-        B.deco_step(ctx, pool[t % pool_n], stream)
+        one_step(pool[t % pool_n])
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local)
@@ -275,7 +292,7 @@ def run_ours(args):
     t_wall0 = time.time()
     ev0.record(stream)
     for t in range(steps):
-        B.deco_step(ctx, pool[(warmup + t) % pool_n], stream)
+        one_step(pool[(warmup + t) % pool_n])
     B.deco_join(ctx, stream)            # the last aggregation ends inside the timed region
     ev1.record(stream)
     torch.cuda.synchronize()
@@ -291,11 +308,12 @@ def run_ours(args):
 
     ms_max = max_over_ranks(ms_total, dist, "cuda")
     ms_per_step = ms_max / steps
-    value = whole_job_value(gbytes, world, ms_per_step)
+    # replicas: every rank steps the whole workload; sharded: the ranks share one workload
+    value = whole_job_value(gbytes, 1 if sharded else world, ms_per_step)
 
     # end to end through the host-buffer entry point: H2D gradients, step, D2H messages
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not sharded:
         k = B.deco_get_k(ctx)
         host_g = [p.cpu().pin_memory() for p in pool[:2]]
         host_msg = torch.empty((wl.n, k, 2), dtype=torch.int32).pin_memory()
@@ -326,25 +344,29 @@ def run_ours(args):
 
     peak, peak_kind = measured_peaks()
     acc_ms = parts["accumulate"] / max(1, iters)
-    achieved = algorithmic_bytes_accumulate(wl) / (acc_ms * 1e-3) / 1e9 if acc_ms > 0 else None
+    acc_bytes = algorithmic_bytes_accumulate(wl) * n_local // wl.n      # this rank's launch
+    achieved = acc_bytes / (acc_ms * 1e-3) / 1e9 if acc_ms > 0 else None
     roofline = {"bound": "hbm", "kernel": "ef_accumulate_kernel", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
                 "traffic": NCU_TRAFFIC_BYTES.get(wl.name)
                 if (args.scale == 1.0 and args.delta is None and args.compressor == "topk") else None,
-                "algorithmic_bytes_per_launch": algorithmic_bytes_accumulate(wl),
+                "algorithmic_bytes_per_launch": acc_bytes,
                 "avg_launch_ms": acc_ms, "launches_timed": iters}
     step_alg_bytes = algorithmic_bytes_accumulate(wl)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
             "config": {"workload": wl.name, "d": wl.d, "n": wl.n, "delta": wl.delta,
                        "tau": wl.tau, "lr": wl.lr, "grad_dtype": wl.grad_dtype,
                        "k": stats["k"], "select_mode": args.select_mode,
                        "compressor": args.compressor,
                        "l2": "inputs larger than L2 (e and g of one step exceed 126 MB)"
                        if 2 * gbytes > 126e6 else "working set fits in L2",
-                       "gradient_pool": pool_n, "replicas": world},
+                       "gradient_pool": pool_n, "replicas": 1 if sharded else world,
+                       "parallelism": ("workers sharded over %d ranks" % world) if sharded
+                       else "replicas only"},
             "step_algorithmic_GBps": step_alg_bytes / (ms_per_step * 1e-3) / 1e9,
             "step_frac_of_hbm_peak": step_alg_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
             "phases_ms": {k_: v / max(1, iters) for k_, v in parts.items()},

@@ -98,7 +98,9 @@ typedef struct {
     int32_t  compressor;     /* deco_compressor; default Top-k */
     uint32_t seed_lo;        /* Random-k: 64-bit seed of the priority stream, low word */
     uint32_t seed_hi;        /*           high word */
-    uint32_t reserved[5];    /* must be zero */
+    uint32_t n_total;        /* worker-sharded context: workers of the whole job (0: n) */
+    uint32_t worker_base;    /* ... and the global id of this context's first worker */
+    uint32_t reserved[3];    /* must be zero */
 } deco_options;
 
 typedef struct {
@@ -307,6 +309,32 @@ deco_status deco_get_kernel_timing(deco_ctx *ctx, void *stream, double *ms_sum /
 
 /* Number of kernels and memset/memcpy nodes the library has enqueued so far. */
 uint64_t deco_launch_count(const deco_ctx *ctx);
+
+/* ------------------------------------------------- workers sharded over several contexts */
+
+/*
+ * Algorithm 1's workers are separate machines that exchange only the sparse messages.  A
+ * context created with opt->n_total > n holds n of the job's n_total workers (global ids
+ * worker_base ... worker_base + n - 1: e, gradients and the worker side are local) and a full
+ * replica of the server side: its message buffer and tile directory have n_total rows,
+ * deco_ef_compress fills the context's own rows, the CALLER brings the other rows in (one
+ * all-gather of the two buffers among the contexts of the job: NCCL over NVLink between GPUs,
+ * plain copies between contexts on one GPU), then deco_aggregate_stale sums all n_total
+ * messages in global worker order and deco_apply_update scales by 1/n_total, so every replica
+ * of x stays bit-identical to the single-context run.  Random-k draws with the global id.
+ * deco_step is not available on such a context (the exchange sits between its parts):
+ * DECO_ERR_STATE.
+ *
+ * Buffers to exchange, valid for the context's lifetime (all DEVICE):
+ *   msg_all   [n_total][msg_row_pairs] pairs; row w = message of global worker w, the first
+ *             k pairs of a row are meaningful
+ *   dir_all   [n_total][dir_row_words] u32; row w = message position of every tile of worker w
+ *             (dir_row_words = tiles + 1)
+ * row0 / rows_local: the rows this context writes.  Every out pointer may be NULL.
+ */
+deco_status deco_get_exchange(deco_ctx *ctx, deco_pair **msg_all, uint64_t *msg_row_pairs,
+                              uint32_t **dir_all, uint64_t *dir_row_words, uint32_t *row0,
+                              uint32_t *rows_local, uint32_t *rows_total);
 
 /* ------------------------------------------------------------- per-layer Top-k (variant) */
 

@@ -45,7 +45,9 @@ class deco_options(ctypes.Structure):
                 ("compressor", ctypes.c_int32),
                 ("seed_lo", ctypes.c_uint32),
                 ("seed_hi", ctypes.c_uint32),
-                ("reserved", ctypes.c_uint32 * 5)]
+                ("n_total", ctypes.c_uint32),
+                ("worker_base", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32 * 3)]
 
 
 class deco_lut_entry(ctypes.Structure):
@@ -107,6 +109,8 @@ SIGNATURES = {
     "deco_export_state": (_i32, [_vp, _vp, _u64, _vp]),
     "deco_import_state": (_i32, [_vp, _vp, _u64, _vp]),
     "deco_launch_count": (_u64, [_vp]),
+    "deco_get_exchange": (_i32, [_vp, _P(_vp), _P(_u64), _P(_vp), _P(_u64), _P(_u32), _P(_u32),
+                                 _P(_u32)]),
     "deco_topk_compress_static": (_i32, [_vp, _u64, _u64, _vp, _vp]),
     "deco_layered_init": (_i32, [_P(_vp), _u64, _u32, _P(_u64), _u32, _f64, _u32, _f32, _vp]),
     "deco_layered_destroy": (None, [_vp]),
@@ -169,8 +173,10 @@ def _stream(stream):
 # ------------------------------------------------------------------ entry points
 
 def _options(grad_dtype, tau_max, delta_max, lr_at_server, params, device, select_mode,
-             compressor, seed):
+             compressor, seed, n_total=0, worker_base=0):
     opt = deco_options()
+    opt.n_total = n_total
+    opt.worker_base = worker_base
     opt.grad_dtype = grad_dtype
     opt.tau_max = tau_max
     opt.delta_max = delta_max
@@ -186,10 +192,11 @@ def _options(grad_dtype, tau_max, delta_max, lr_at_server, params, device, selec
 
 def deco_init(d, n, delta, tau, lr, grad_dtype=DECO_F32, tau_max=0, delta_max=0.0,
               lr_at_server=False, params=None, device=0, select_mode=DECO_SELECT_AUTO,
-              compressor=DECO_COMPRESSOR_TOPK, seed=0):
-    """-> opaque context handle (int).  `params`: optional fp32 CUDA tensor of length d."""
+              compressor=DECO_COMPRESSOR_TOPK, seed=0, n_total=0, worker_base=0):
+    """-> opaque context handle (int).  `params`: optional fp32 CUDA tensor of length d.
+    n_total / worker_base: this context holds n of the job's n_total workers (sharded job)."""
     opt = _options(grad_dtype, tau_max, delta_max, lr_at_server, params, device, select_mode,
-                   compressor, seed)
+                   compressor, seed, n_total, worker_base)
     ctx = _vp()
     _check(load().deco_init(ctypes.byref(ctx), d, n, delta, tau, lr, ctypes.byref(opt)),
            "deco_init")
@@ -392,6 +399,51 @@ def deco_import_state(ctx, blob, stream=None):
 
 def deco_launch_count(ctx):
     return load().deco_launch_count(ctx)
+
+
+def deco_get_exchange(ctx):
+    """Buffers a worker-sharded job all-gathers between compress and aggregate."""
+    m, mr, dd, dr = _vp(), _u64(), _vp(), _u64()
+    r0, rl, rt = _u32(), _u32(), _u32()
+    _check(load().deco_get_exchange(ctx, ctypes.byref(m), ctypes.byref(mr), ctypes.byref(dd),
+                                    ctypes.byref(dr), ctypes.byref(r0), ctypes.byref(rl),
+                                    ctypes.byref(rt)), "deco_get_exchange")
+    return {"msg_all": m.value, "msg_row_pairs": mr.value, "dir_all": dd.value,
+            "dir_row_words": dr.value, "row0": r0.value, "rows_local": rl.value,
+            "rows_total": rt.value}
+
+
+def exchange_views(ctx, device=0):
+    """torch views of the two exchange buffers: ([n_total, k_cap, 2] int32, [n_total, tiles+1]
+    int32), for torch.distributed collectives or plain copies."""
+    x = deco_get_exchange(ctx)
+    msg = view_i32(x["msg_all"], (x["rows_total"], x["msg_row_pairs"], 2), device)
+    dirs = view_i32(x["dir_all"], (x["rows_total"], x["dir_row_words"]), device)
+    return msg, dirs, x
+
+
+def all_gather_rows(full, row0, rows_local, group=None):
+    """In-place all-gather of a row-sharded tensor: this rank owns rows [row0, row0+rows_local)
+    of `full`, every rank the same number, in rank order.  Plumbing (torch.distributed)."""
+    import torch.distributed as dist
+    mine = full[row0:row0 + rows_local]
+    dist.all_gather_into_tensor(full, mine, group=group)
+
+
+def deco_step_sharded(ctx, grads, group=None, stream=None, device=0):
+    """One iteration of a worker-sharded context: compress the local workers, all-gather the
+    sparse messages and their tile directories among the ranks of `group` (NCCL on GPUs: the
+    collectives run on torch's current stream, which must be `stream`), aggregate, update."""
+    deco_ef_compress(ctx, grads, stream)
+    msg, dirs, x = exchange_views(ctx, device)
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        all_gather_rows(msg, x["row0"], x["rows_local"], group)
+        all_gather_rows(dirs, x["row0"], x["rows_local"], group)
+    elif x["rows_total"] != x["rows_local"]:
+        raise RuntimeError("a worker-sharded context needs an initialised process group")
+    deco_aggregate_stale(ctx, stream)
+    deco_apply_update(ctx, stream)
 
 
 DECO_STATIC_MAX_D = 16777216

@@ -87,7 +87,7 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
     if (err == cudaSuccess)
         err = cudaMemsetAsync(c->sample_hist, 0, sizeof(uint32_t) * c->n * SAMPLE_BINS, s);
     if (err == cudaSuccess)
-        err = cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n * (c->ntiles + 1), s);
+        err = cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n_total * (c->ntiles + 1), s);
     c->launches += 5;
     c->t = 0;
     c->phase = 0;
@@ -156,6 +156,9 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     for (uint32_t r : o.reserved)
         if (r != 0) return DECO_ERR_INVALID_ARG;
     if (d == 0 || d >= 0xFFFFFFFFull - TILE || n == 0 || n > 65535) return DECO_ERR_INVALID_ARG;
+    if (o.n_total == 0 && o.worker_base != 0) return DECO_ERR_INVALID_ARG;
+    if (o.n_total != 0 && (o.n_total > 65535 || static_cast<uint64_t>(o.worker_base) + n > o.n_total))
+        return DECO_ERR_INVALID_ARG;
     if (!(delta > 0.0) || !(delta <= 1.0) || !(lr == lr)) return DECO_ERR_INVALID_ARG;
     if (o.grad_dtype != DECO_F32 && o.grad_dtype != DECO_BF16) return DECO_ERR_INVALID_ARG;
     if (o.select_mode != DECO_SELECT_AUTO && o.select_mode != DECO_SELECT_EXACT_PASSES)
@@ -182,6 +185,8 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     c->d = d;
     c->g_stride = g_stride ? g_stride : d;
     c->n = n;
+    c->n_total = o.n_total ? o.n_total : n;
+    c->worker_base = o.worker_base;
     c->delta = delta;
     c->delta_max = o.delta_max != 0.0 ? o.delta_max : delta;
     c->tau = tau;
@@ -218,8 +223,8 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
         need(dev_alloc(c, &c->params, d));
         c->own_params = (st == DECO_OK);
     }
-    need(dev_alloc(c, &c->msg, static_cast<uint64_t>(n) * c->k_cap));
-    need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * n * c->k_cap));
+    need(dev_alloc(c, &c->msg, static_cast<uint64_t>(c->n_total) * c->k_cap));
+    need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * c->n_total * c->k_cap));
     need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
     // slices of 256 staged entries, plus one partial slice for every tile that has any
     c->work_cap = c->stage_cap / 256 + (c->stage_cap / 17 < c->ntiles ? c->stage_cap / 17 : c->ntiles) + 32;
@@ -232,7 +237,7 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     need(dev_alloc(c, &c->tile_gt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_eq, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_take, static_cast<uint64_t>(n) * c->ntiles));
-    need(dev_alloc(c, &c->tile_start, static_cast<uint64_t>(n) * (c->ntiles + 1)));
+    need(dev_alloc(c, &c->tile_start, static_cast<uint64_t>(c->n_total) * (c->ntiles + 1)));
     need(dev_alloc(c, &c->tile_off, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_cnt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_rej, static_cast<uint64_t>(n) * c->ntiles));
@@ -310,13 +315,13 @@ extern "C" deco_status deco_aggregate_stale(deco_ctx *c, void *stream)
     const uint32_t si = static_cast<uint32_t>(c->t % c->ring);
     Slot &sl = c->slot_info[si];
     if (sl.valid) return DECO_ERR_STATE;    // cannot happen while tau <= tau_max
-    deco_pair *slot = c->slots + static_cast<uint64_t>(si) * c->n * c->k_cap;
+    deco_pair *slot = c->slots + static_cast<uint64_t>(si) * c->n_total * c->k_cap;
     if (wait_for_aggregate(c, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
     mark(c, 3, as_stream(stream));
     if (launch_aggregate(c, slot, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
     mark(c, 4, as_stream(stream));
     sl.step = c->t;
-    sl.positions = static_cast<uint64_t>(c->n) * c->k_of_msg;
+    sl.positions = static_cast<uint64_t>(c->n_total) * c->k_of_msg;
     sl.valid = true;
     c->phase = 2;
     return DECO_OK;
@@ -329,7 +334,7 @@ namespace {
 deco_status apply_due(deco_ctx *c, cudaStream_t s)
 {
     const float beta = c->lr_at_server ? c->lr : 1.0f;
-    const float neg_scale = -(beta / static_cast<float>(c->n));
+    const float neg_scale = -(beta / static_cast<float>(c->n_total));
     if (c->t < c->tau) return DECO_OK;
     const uint64_t due = c->t - c->tau;
     // step ids still cached lie in (t - ring, t]
@@ -337,7 +342,7 @@ deco_status apply_due(deco_ctx *c, cudaStream_t s)
     for (uint64_t step = lo; step <= due; ++step) {
         Slot &sl = c->slot_info[step % c->ring];
         if (!sl.valid || sl.step != step) continue;
-        const deco_pair *slot = c->slots + (step % c->ring) * c->n * c->k_cap;
+        const deco_pair *slot = c->slots + (step % c->ring) * c->n_total * c->k_cap;
         if (launch_apply(c, slot, sl.positions, neg_scale, s) != cudaSuccess) return DECO_ERR_CUDA;
         sl.valid = false;
     }
@@ -405,6 +410,7 @@ extern "C" deco_status deco_step(deco_ctx *c, const void *grads, void *stream)
 {
     if (!c || !grads) return DECO_ERR_INVALID_ARG;
     if (c->phase != 0) return DECO_ERR_STATE;
+    if (c->n_total != c->n) return DECO_ERR_STATE;      // the exchange sits between the parts
     if (c->tau == 0 || !c->side_stream) {
         // the update of this iteration needs this iteration's aggregate: strictly in order
         deco_status st = deco_ef_compress(c, grads, stream);
@@ -482,7 +488,8 @@ extern "C" deco_status deco_step_host(deco_ctx *c, const void *grads_host, deco_
     if (st != DECO_OK) return st;
     if (msg_out) {
         // rows of k pairs, packed: [n][k]
-        if (cudaMemcpy2DAsync(msg_out, c->k_of_msg * sizeof(deco_pair), c->msg,
+        if (cudaMemcpy2DAsync(msg_out, c->k_of_msg * sizeof(deco_pair),
+                              c->msg + static_cast<uint64_t>(c->worker_base) * c->k_cap,
                               c->k_cap * sizeof(deco_pair), c->k_of_msg * sizeof(deco_pair), c->n,
                               cudaMemcpyDeviceToHost, s) != cudaSuccess)
             return DECO_ERR_CUDA;
@@ -530,7 +537,7 @@ extern "C" deco_status deco_get_buffers(deco_ctx *c, float **e, uint64_t *e_stri
     if (!c) return DECO_ERR_INVALID_ARG;
     if (e) *e = c->e;
     if (e_stride) *e_stride = c->e_stride;
-    if (msg) *msg = c->msg;
+    if (msg) *msg = c->msg + static_cast<uint64_t>(c->worker_base) * c->k_cap;   // the local rows
     if (k_cap) *k_cap = c->k_cap;
     if (params) *params = c->params;
     return DECO_OK;
@@ -546,7 +553,7 @@ extern "C" deco_status deco_get_aggregate(deco_ctx *c, uint64_t step, const deco
         DeviceGuard guard(c->device);
         if (!guard.ok || drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
     }
-    *entries = c->slots + (step % c->ring) * c->n * c->k_cap;
+    *entries = c->slots + (step % c->ring) * c->n_total * c->k_cap;
     *positions = sl.positions;
     return DECO_OK;
 }
@@ -608,6 +615,21 @@ extern "C" deco_status deco_get_stats(deco_ctx *c, void *stream, deco_stats *out
     return DECO_OK;
 }
 
+extern "C" deco_status deco_get_exchange(deco_ctx *c, deco_pair **msg_all, uint64_t *msg_row_pairs,
+                                         uint32_t **dir_all, uint64_t *dir_row_words,
+                                         uint32_t *row0, uint32_t *rows_local, uint32_t *rows_total)
+{
+    if (!c) return DECO_ERR_INVALID_ARG;
+    if (msg_all) *msg_all = c->msg;
+    if (msg_row_pairs) *msg_row_pairs = c->k_cap;
+    if (dir_all) *dir_all = c->tile_start;
+    if (dir_row_words) *dir_row_words = static_cast<uint64_t>(c->ntiles) + 1;
+    if (row0) *row0 = c->worker_base;
+    if (rows_local) *rows_local = c->n;
+    if (rows_total) *rows_total = c->n_total;
+    return DECO_OK;
+}
+
 extern "C" uint64_t deco_launch_count(const deco_ctx *c) { return c ? c->launches : 0; }
 
 // ------------------------------------------------------------------ checkpoint / resume
@@ -619,7 +641,7 @@ struct StateHeader {
     double delta;
     uint32_t tau, grad_dtype, lr_at_server, compressor;
     float lr;
-    uint32_t pad2;
+    uint32_t sharding;          // n_total << 16 | worker_base (both below 65536)
     uint64_t seed;
 };
 constexpr uint64_t STATE_MAGIC = 0x4F434544534F4345ull;   // "ECOSDECO"
@@ -665,6 +687,7 @@ extern "C" deco_status deco_export_state(deco_ctx *c, void *buf, uint64_t bytes,
     h.delta = c->delta; h.tau = c->tau; h.grad_dtype = c->grad_dtype;
     h.lr_at_server = c->lr_at_server; h.lr = c->lr;
     h.compressor = c->compressor; h.seed = c->seed;
+    h.sharding = (c->n_total << 16) | c->worker_base;
     std::memcpy(out, &h, sizeof h);
     out += sizeof h;
     for (const Slot &sl : c->slot_info) {
@@ -683,7 +706,7 @@ extern "C" deco_status deco_export_state(deco_ctx *c, void *buf, uint64_t bytes,
     for (uint32_t q = 0; q < c->ring; ++q) {
         const Slot &sl = c->slot_info[q];
         if (!sl.valid) continue;
-        if (cudaMemcpyAsync(out, c->slots + static_cast<uint64_t>(q) * c->n * c->k_cap,
+        if (cudaMemcpyAsync(out, c->slots + static_cast<uint64_t>(q) * c->n_total * c->k_cap,
                             sizeof(deco_pair) * sl.positions, cudaMemcpyDeviceToHost, s) != cudaSuccess)
             return DECO_ERR_CUDA;
         out += sizeof(deco_pair) * sl.positions;
@@ -703,7 +726,8 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
     if (h.magic != STATE_MAGIC || h.version != 1 || h.d != c->d || h.n != c->n ||
         h.k_cap != c->k_cap || h.ring != c->ring || h.grad_dtype != static_cast<uint32_t>(c->grad_dtype) ||
         h.lr_at_server != static_cast<uint32_t>(c->lr_at_server) || h.tau > c->tau_max || h.k > c->k_cap ||
-        h.compressor != static_cast<uint32_t>(c->compressor) || h.seed != c->seed)
+        h.compressor != static_cast<uint32_t>(c->compressor) || h.seed != c->seed ||
+        h.sharding != ((c->n_total << 16) | c->worker_base))
         return DECO_ERR_INVALID_ARG;
     if (bytes < sizeof(StateHeader) + sizeof(SlotRecord) * c->ring) return DECO_ERR_INVALID_ARG;
     std::vector<Slot> slots(c->ring);
@@ -713,7 +737,7 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
         SlotRecord r;
         std::memcpy(&r, in, sizeof r);
         in += sizeof r;
-        if (r.valid && (r.positions > static_cast<uint64_t>(c->n) * c->k_cap || r.step % c->ring != q))
+        if (r.valid && (r.positions > static_cast<uint64_t>(c->n_total) * c->k_cap || r.step % c->ring != q))
             return DECO_ERR_INVALID_ARG;
         slots[q].step = r.step;
         slots[q].positions = r.positions;
@@ -736,7 +760,7 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
     in += sizeof(float) * c->d;
     for (uint32_t q = 0; q < c->ring; ++q) {
         if (!slots[q].valid) continue;
-        if (cudaMemcpyAsync(c->slots + static_cast<uint64_t>(q) * c->n * c->k_cap, in,
+        if (cudaMemcpyAsync(c->slots + static_cast<uint64_t>(q) * c->n_total * c->k_cap, in,
                             sizeof(deco_pair) * slots[q].positions, cudaMemcpyHostToDevice, s) != cudaSuccess)
             return DECO_ERR_CUDA;
         in += sizeof(deco_pair) * slots[q].positions;

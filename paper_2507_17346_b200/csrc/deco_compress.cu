@@ -59,12 +59,13 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
 struct RandParams {
     uint32_t on;                 // 0: Top-k on |a|, 1: Random-k
     uint32_t seed_lo, seed_hi, step_lo, step_hi;
+    uint32_t worker_base;        // global id of the context's first worker
 };
 
 __device__ __forceinline__ uint4 rand_keys4(const RandParams &rk, uint32_t worker, uint64_t j4)
 {
     // priorities of the four entries 4*j4 .. 4*j4 + 3
-    uint4 o = philox4x32_10(make_uint4(static_cast<uint32_t>(j4), rk.step_lo, worker,
+    uint4 o = philox4x32_10(make_uint4(static_cast<uint32_t>(j4), rk.step_lo, rk.worker_base + worker,
                                        rk.step_hi ^ 0x52414E44u), rk.seed_lo, rk.seed_hi);
     return make_uint4(o.x >> 9, o.y >> 9, o.z >> 9, o.w >> 9);
 }
@@ -1620,6 +1621,7 @@ RandParams make_rand(const deco_ctx *c)
     rk.seed_hi = static_cast<uint32_t>(c->seed >> 32);
     rk.step_lo = static_cast<uint32_t>(c->t);
     rk.step_hi = static_cast<uint32_t>(c->t >> 32);
+    rk.worker_base = c->worker_base;
     return rk;
 }
 
@@ -1641,7 +1643,8 @@ Sel make_sel(const deco_ctx *c)
     p.tile_gt = c->tile_gt;
     p.tile_eq = c->tile_eq;
     p.tile_take = c->tile_take;
-    p.tile_start = c->tile_start;
+    // the context's own rows of the job-wide directory and message buffer
+    p.tile_start = c->tile_start + static_cast<size_t>(c->worker_base) * (c->ntiles + 1);
     p.tile_off = c->tile_off;
     p.tile_cnt = c->tile_cnt;
     p.tile_rej = c->tile_rej;
@@ -1651,7 +1654,7 @@ Sel make_sel(const deco_ctx *c)
     p.chunk_eq = c->chunk_eq;
     p.chunk_eqb = c->chunk_eqb;
     p.chunk_start = c->chunk_start;
-    p.msg = c->msg;
+    p.msg = c->msg + static_cast<size_t>(c->worker_base) * c->k_cap;
     p.k_cap = c->k_cap;
     p.stage = c->stage;
     p.stage_cap = c->stage_cap;

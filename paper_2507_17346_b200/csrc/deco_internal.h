@@ -67,6 +67,9 @@ struct deco_ctx {
     // problem
     uint64_t d = 0;
     uint32_t n = 0;
+    // worker-sharded context: n local workers with global ids worker_base .. worker_base+n-1
+    // of n_total; message buffer, directory, cache and update cover all n_total
+    uint32_t n_total = 0, worker_base = 0;
     double delta = 0, delta_max = 0;
     uint32_t tau = 0, tau_max = 0;
     float lr = 0;
@@ -89,8 +92,8 @@ struct deco_ctx {
     float *e = nullptr;
     float *params = nullptr;
     bool own_params = false;
-    deco_pair *msg = nullptr;
-    deco_pair *slots = nullptr;         // [ring][n * k_cap]
+    deco_pair *msg = nullptr;           // [n_total][k_cap]
+    deco_pair *slots = nullptr;         // [ring][n_total * k_cap]
     deco_pair *stage = nullptr;         // [n][stage_cap]
     uint2 *work = nullptr;              // [n][work_cap] emit work list: (tile, slice)
     uint64_t work_cap = 0;
@@ -103,7 +106,7 @@ struct deco_ctx {
     uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
     uint32_t *tile_eq = nullptr;        // [n][ntiles]  entries equal to it per tile
     uint32_t *tile_take = nullptr;      // [n][ntiles]  ties taken per tile
-    uint32_t *tile_start = nullptr;     // [n][ntiles + 1] message position of each tile
+    uint32_t *tile_start = nullptr;     // [n_total][ntiles + 1] message position of each tile
     uint32_t *tile_off = nullptr;       // [n][ntiles]  staging offset of each tile's candidates
     uint32_t *tile_cnt = nullptr;       // [n][ntiles]  staged candidates per tile
     uint32_t *tile_rej = nullptr;       // [n][ntiles]  staged candidates below the threshold

@@ -348,19 +348,19 @@ apply_kernel(const deco_pair *__restrict__ slot, uint64_t positions, float neg_s
 
 cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s)
 {
-    const uint64_t positions = static_cast<uint64_t>(c->n) * c->k_of_msg;
+    const uint64_t positions = static_cast<uint64_t>(c->n_total) * c->k_of_msg;
     c->launches += 1;
-    if (c->n <= 32 && positions <= 80ull * c->ntiles) {
+    if (c->n_total <= 32 && positions <= 80ull * c->ntiles) {
         // on average at most 80 entries per tile over all workers: a warp per tile
         aggregate_sparse_kernel<<<(c->ntiles + WARPS - 1) / WARPS, BLOCK, 0, s>>>(
-            c->msg, c->k_cap, c->tile_start, c->ntiles, c->n, slot, positions, c->dev_status);
+            c->msg, c->k_cap, c->tile_start, c->ntiles, c->n_total, slot, positions, c->dev_status);
         return cudaGetLastError();
     }
     // next to the streaming pass of the following iteration the aggregation takes half the
     // CTA slots it could hold, so that the pass keeps most of its loads in flight
     const uint32_t per_sm = (c->agg_stream && s == c->agg_stream) ? 3u : 6u;
     const uint32_t blocks = c->ntiles < 148u * per_sm ? c->ntiles : 148u * per_sm;
-    aggregate_kernel<<<blocks, BLOCK, 0, s>>>(c->msg, c->k_cap, c->tile_start, c->ntiles, c->n,
+    aggregate_kernel<<<blocks, BLOCK, 0, s>>>(c->msg, c->k_cap, c->tile_start, c->ntiles, c->n_total,
                                               slot, positions, c->dev_status);
     return cudaGetLastError();
 }

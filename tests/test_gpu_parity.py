@@ -237,6 +237,86 @@ def test_per_layer_topk_variant():
         run_layered_parity(odd, 4, 0.02, 1, 0.1, grads, steps=4, grad_dtype=name)
 
 
+@pytest.mark.parametrize("compressor", ["topk", "randk"])
+def test_worker_sharded_contexts_equal_the_single_job(compressor):
+    """Five workers split 2 + 3 over two contexts on one GPU.  Each compresses its own workers;
+    the rows of the two exchange buffers are then copied across (what the all-gather does
+    between GPUs), and both replicas aggregate and update.  Local messages and residuals, the
+    aggregate and both parameter replicas must equal the oracle's single five-worker job."""
+    from oracle import dd_ef_sgd as O
+    from tests.parity import bits, read_aggregate, read_e, read_messages, read_params
+    d, n, delta, tau, lr = 70_004, 5, 0.004, 1, 0.1
+    split = [(0, 2), (2, 3)]
+    comp = B.DECO_COMPRESSOR_RANDK if compressor == "randk" else B.DECO_COMPRESSOR_TOPK
+    ctxs = [B.deco_init(d, cnt, delta, tau, lr, n_total=n, worker_base=base, compressor=comp,
+                        seed=99, tau_max=2, delta_max=0.02) for base, cnt in split]
+    orc = O.DDEFSGD(d, n, delta, tau, lr, compressor=compressor, seed=99)
+    try:
+        with pytest.raises(B.DecoError):
+            B.deco_step(ctxs[0], torch.zeros((2, d), device="cuda"))
+        for t in range(6):
+            if t == 3:
+                for c in ctxs:
+                    B.deco_set_policy(c, 0.02, 2)
+                orc.set_policy(0.02, 2)
+            g = _values("normal", n, d, t, torch.float32)
+            ref = orc.step(W.to_numpy_bits(g))
+            views = []
+            for c, (base, cnt) in zip(ctxs, split):
+                B.deco_ef_compress(c, g[base:base + cnt])
+                views.append(B.exchange_views(c))
+            for me, (base, cnt) in enumerate(split):               # the exchange, by copies
+                for other in range(len(split)):
+                    if other != me:
+                        views[other][0][base:base + cnt].copy_(views[me][0][base:base + cnt])
+                        views[other][1][base:base + cnt].copy_(views[me][1][base:base + cnt])
+            touched = np.unique(np.concatenate([s for s, _ in ref["msgs"]]))
+            for c, (base, cnt) in zip(ctxs, split):
+                idx, val = read_messages(c, cnt, ref["k"])
+                for i in range(cnt):
+                    assert np.array_equal(idx[i], ref["msgs"][base + i][0]), (t, base + i)
+                    assert np.array_equal(bits(val[i]), bits(ref["msgs"][base + i][1]))
+                assert np.array_equal(bits(read_e(c, cnt, d)), bits(orc.e[base:base + cnt]))
+                B.deco_aggregate_stale(c)
+                aidx, aval = read_aggregate(c, t)
+                assert np.array_equal(aidx, touched), t
+                assert np.array_equal(bits(aval), bits(ref["S"][touched])), t
+                B.deco_apply_update(c)
+                assert np.array_equal(bits(read_params(c, d)), bits(orc.x)), t
+        for c in ctxs:
+            st = B.deco_get_stats(c)
+            assert st["device_status"] == 0 and st["step"] == 6
+    finally:
+        for c in ctxs:
+            B.deco_destroy(c)
+
+
+def test_sharded_step_through_nccl_with_one_rank():
+    """The binding's sharded step (compress, all-gather of the exchange buffers through
+    torch.distributed / NCCL, aggregate, update) with a world of one rank gives the bits of
+    the plain three calls."""
+    import torch.distributed as dist
+    from tests.parity import bits, read_params
+    d, n = 120_000, 4
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29541", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    a = B.deco_init(d, n, 0.01, 2, 0.1)
+    b = B.deco_init(d, n, 0.01, 2, 0.1)
+    try:
+        for t in range(5):
+            g = _values("normal", n, d, t, torch.float32)
+            B.deco_step_sharded(a, g)
+            B.deco_ef_compress(b, g)
+            B.deco_aggregate_stale(b)
+            B.deco_apply_update(b)
+            torch.cuda.synchronize()
+            assert np.array_equal(bits(read_params(a, d)), bits(read_params(b, d))), t
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
+        dist.destroy_process_group()
+
+
 @pytest.mark.parametrize("mode", MODES)
 def test_random_k_sparsifier(mode):
     """Random-k in place of Top-k: the same Philox priorities on both sides give the same index
