@@ -249,7 +249,7 @@ def run_ours(args):
     sz = 4 if wl.grad_dtype == "f32" else 2
     gbytes = grad_bytes(wl)
     # enough steps for a timed region that nvidia-smi can sample
-    steps = args.steps if args.steps is not None else max(50, min(3000, int(2.0e12 / (6 * gbytes))))
+    steps = args.steps if args.steps is not None else max(50, min(4000, int(8.0e12 / (6 * gbytes))))
     warmup = args.warmup if args.warmup is not None else 10
     warmup = max(3, warmup)
     pool_n = args.pool if args.pool > 0 else max(2, min(8, int(6e9 // gbytes)))
