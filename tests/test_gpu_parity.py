@@ -431,6 +431,38 @@ def test_fused_step_equals_the_three_calls():
         B.deco_destroy(b)
 
 
+@pytest.mark.parametrize("tau", [1, 2])
+def test_fused_step_with_a_long_aggregation(tau):
+    """Dense messages (delta = 0.05 of 4 M entries): the aggregation left behind by one fused
+    step is still running when the next step's worker side starts, so the orderings between
+    the internal streams (emit after the previous aggregation, update after the aggregate it
+    consumes) carry real waits.  Bits must equal the strictly sequential three calls."""
+    d, n = 4_000_000, 4
+    a = B.deco_init(d, n, 0.05, tau, 0.1)
+    b = B.deco_init(d, n, 0.05, tau, 0.1)
+    try:
+        pool = [_values("normal", n, d, t, torch.float32) for t in range(3)]
+        for t in range(12):
+            B.deco_step(a, pool[t % 3])                          # back to back, no host sync
+        for t in range(12):
+            B.deco_ef_compress(b, pool[t % 3])
+            B.deco_aggregate_stale(b)
+            B.deco_apply_update(b)
+        B.deco_join(a)
+        torch.cuda.synchronize()
+        ba, bb = B.deco_get_buffers(a), B.deco_get_buffers(b)
+        assert torch.equal(B.view_i32(ba["params"], (d,)), B.view_i32(bb["params"], (d,)))
+        assert torch.equal(B.view_i32(ba["e"], (n, ba["e_stride"])), B.view_i32(bb["e"], (n, bb["e_stride"])))
+        for s_ in range(12 - tau, 12):                           # the aggregates still cached
+            pa, na = B.deco_get_aggregate(a, s_)
+            pb, nb = B.deco_get_aggregate(b, s_)
+            assert na == nb and torch.equal(B.view_i32(pa, (na, 2)), B.view_i32(pb, (nb, 2)))
+        assert B.deco_get_stats(a)["device_status"] == 0
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
+
+
 def test_checkpoint_and_resume_give_the_same_bits():
     wl = W.make_workload("gpt2_small", 0.08)
     kw = dict(grad_dtype=B.DECO_BF16, tau_max=4, delta_max=0.01)
