@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--shard-workers", action="store_true",
                     help="N > 1: split the workers over the ranks (sparse all-gather per step) "
                          "instead of running N replicas; strong scaling")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="per-layer Top-k variant: k(delta, d_l) entries of every tensor of the workload "
+                         "(deco_layered_step); no per-kernel timing, no e2e")
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink the workload's layer widths (profiling captures of the large shapes)")
     return ap.parse_args()
@@ -262,6 +265,8 @@ def run_ours(args):
             raise SystemExit("--shard-workers needs the worker count to be a multiple of --gpus")
         n_local, base = wl.n // world, rank * (wl.n // world)
         pool = [p[base:base + n_local].clone() for p in pool]      # this rank's workers only
+    if args.per_layer:
+        return run_per_layer(args, wl, pool, pool_n, steps, warmup, local, world, rank, dist)
     ctx = B.deco_init(wl.d, n_local, wl.delta, wl.tau, wl.lr,
                       grad_dtype=B.DECO_F32 if wl.grad_dtype == "f32" else B.DECO_BF16,
                       device=local, select_mode=mode,
@@ -379,6 +384,67 @@ def run_ours(args):
         line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
                                 "sample": sample, "ms_per_step_sample": ms}
     print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_per_layer(args, wl, pool, pool_n, steps, warmup, local, world, rank, dist):
+    """The per-layer Top-k variant on the workload's tensors: whole-step timing only."""
+    import torch
+    from paper_2507_17346_b200 import binding as B
+    offsets = [0]
+    for t in wl.tensors:
+        offsets.append(offsets[-1] + int(t.numel))
+    ctx = B.deco_layered_init(wl.d, wl.n, offsets, wl.delta, wl.tau, wl.lr,
+                              grad_dtype=B.DECO_F32 if wl.grad_dtype == "f32" else B.DECO_BF16,
+                              device=local)
+    stream = torch.cuda.current_stream()
+    for t in range(warmup):
+        B.deco_layered_step(ctx, pool[t % pool_n], stream)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for t in range(steps):
+        B.deco_layered_step(ctx, pool[(warmup + t) % pool_n], stream)
+    B.deco_layered_join(ctx, stream)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    ms_per_step = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda") / steps
+    info = B.deco_layered_info(ctx)
+    fallbacks = 0
+    for l in range(info["n_layers"]):
+        sub, _, _ = B.deco_layered_layer(ctx, l)
+        st = B.deco_get_stats(sub, stream)
+        fallbacks += st["exact_pass_workers"]
+        assert st["device_status"] == 0, (l, st)
+    B.deco_layered_destroy(ctx)
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        alg = algorithmic_bytes_accumulate(wl)
+        line = {"metric": METRIC, "value": whole_job_value(grad_bytes(wl), world, ms_per_step), "unit": UNIT,
+                "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic",
+                "config": {"workload": wl.name, "variant": "per-layer Top-k", "layers": info["n_layers"],
+                           "d": wl.d, "n": wl.n, "delta": wl.delta, "tau": wl.tau, "lr": wl.lr,
+                           "grad_dtype": wl.grad_dtype, "k_total": info["k_total"],
+                           "gradient_pool": pool_n, "parallelism": "replicas only"},
+                "step_algorithmic_GBps": alg / (ms_per_step * 1e-3) / 1e9,
+                "step_frac_of_hbm_peak": alg / (ms_per_step * 1e-3) / 1e9 / peak,
+                "peak": peak, "peak_kind": peak_kind,
+                "exact_pass_worker_steps": fallbacks, "clocks": clocks}
+        print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 

@@ -346,6 +346,10 @@ deco_status deco_get_exchange(deco_ctx *ctx, deco_pair **msg_all, uint64_t *msg_
  * k_l = k(delta, d_l) largest entries of each range (ties by increasing index).  Nothing else in
  * Algorithm 1 couples entries of different layers, so a layered context is a batch of ordinary
  * contexts, one per layer, sharing policy, stepsize, gradient buffer and parameter vector.
+ * With Top-k on the streaming route the layers are not stepped one by one: every kernel of the
+ * path runs once for all layers (a table of the layers' buffers in device memory, grid rows
+ * = layer x worker), and layers of at most 8192 entries are done by one CTA per (layer, worker).
+ * With Random-k or DECO_SELECT_EXACT_PASSES each layer's context is stepped on its own.
  *   layer_offsets  HOST, [n_layers + 1], strictly increasing, first 0, last d
  *   opt            as for deco_init; opt->params (DEVICE, [d], 16-byte aligned) or NULL;
  *                  tau_max and delta_max apply to every layer
@@ -360,10 +364,10 @@ deco_status deco_layered_init(deco_layered **out, uint64_t d, uint32_t n,
 void deco_layered_destroy(deco_layered *ctx);
 
 /*
- * One iteration of every layer (deco_step per layer).  grads: DEVICE, [n][d] row-major, dtype =
- * grad_dtype, 16-byte aligned base.  The layers run round-robin on internal streams forked
- * from `stream` at the start of the call and joined back at its end; like deco_step, each
- * layer may leave its aggregation running (deco_layered_join orders `stream` after them).
+ * One iteration of every layer.  grads: DEVICE, [n][d] row-major, dtype = grad_dtype, 16-byte
+ * aligned base.  The work runs on internal streams forked from `stream` at the start of the
+ * call and joined back at its end; where layers are stepped one by one (deco_step per layer),
+ * each may leave its aggregation running (deco_layered_join orders `stream` after them).
  * The first error of a layer is returned; layers after it are not stepped.
  */
 deco_status deco_layered_step(deco_layered *ctx, const void *grads, void *stream);

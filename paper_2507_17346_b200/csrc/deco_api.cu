@@ -358,6 +358,37 @@ void finish_iteration(deco_ctx *c)
 
 }  // namespace
 
+deco_status deco::mark_compressed_external(deco_ctx *c)
+{
+    if (c->phase != 0) return DECO_ERR_STATE;
+    c->k_of_msg = c->k;
+    c->phase = 1;
+    return DECO_OK;
+}
+
+uint32_t deco::advance_iteration_external(deco_ctx *c, std::vector<uint32_t> *due)
+{
+    const uint32_t si = static_cast<uint32_t>(c->t % c->ring);
+    c->k_of_msg = c->k;
+    Slot &now = c->slot_info[si];
+    now.step = c->t;
+    now.positions = static_cast<uint64_t>(c->n_total) * c->k;
+    now.valid = true;
+    if (c->t >= c->tau) {
+        const uint64_t last = c->t - c->tau;
+        const uint64_t lo = c->t + 1 >= c->ring ? c->t + 1 - c->ring : 0;
+        for (uint64_t step = lo; step <= last; ++step) {
+            Slot &sl = c->slot_info[step % c->ring];
+            if (!sl.valid || sl.step != step) continue;
+            if (due) due->push_back(static_cast<uint32_t>(step % c->ring));
+            sl.valid = false;
+        }
+    }
+    c->t += 1;
+    c->phase = 0;
+    return si;
+}
+
 extern "C" deco_status deco_apply_update(deco_ctx *c, void *stream)
 {
     if (!c) return DECO_ERR_INVALID_ARG;

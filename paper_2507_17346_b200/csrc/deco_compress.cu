@@ -22,6 +22,9 @@
 // consecutive entries, and in round u lane l owns V consecutive ones, so each warp-level
 // load is one contiguous 512-byte request.
 #include <cooperative_groups.h>
+
+#include <algorithm>
+#include <new>
 #include <cuda_bf16.h>
 
 #include "deco_internal.h"
@@ -293,15 +296,20 @@ __device__ __forceinline__ void pick_body(SelectState &s, const uint32_t *h, uin
 }
 
 // true for exactly one CTA per counter: the last of gridDim.x to get here (nothing waits)
-__device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *s_flag)
+__device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *s_flag, uint32_t ctas)
 {
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) *s_flag = (atomicAdd(counter, 1u) == gridDim.x - 1) ? 1u : 0u;
+    if (threadIdx.x == 0) *s_flag = (atomicAdd(counter, 1u) == ctas - 1) ? 1u : 0u;
     __syncthreads();
     const bool last = *s_flag != 0;
     if (last) __threadfence();
     return last;
+}
+
+__device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *s_flag)
+{
+    return last_cta_to_arrive(counter, s_flag, gridDim.x);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -330,21 +338,29 @@ static uint32_t sample_groups(uint64_t d, uint64_t k)
 {
     const uint64_t nchunks = (d + 3) >> 2;
     uint64_t want = static_cast<uint64_t>(0.6 * cbrt(static_cast<double>(d) * static_cast<double>(k)));
-    if (want < SAMPLE_CHUNKS / 4) want = SAMPLE_CHUNKS / 4;
+    // at least a quarter of the maximum, but for short vectors (layers of the per-layer variant)
+    // no more than one group in 16, down to one CTA's worth
+    uint64_t least = nchunks / 16;
+    if (least > SAMPLE_CHUNKS / 4) least = SAMPLE_CHUNKS / 4;
+    if (least < BEGIN_BLOCK) least = BEGIN_BLOCK;
+    if (want < least) want = least;
     if (want > SAMPLE_CHUNKS) want = SAMPLE_CHUNKS;
     return static_cast<uint32_t>(nchunks < want ? nchunks : want);
 }
 
-template <int GT>
-__global__ void __launch_bounds__(BEGIN_BLOCK, 2)
-begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t exact_all, uint32_t S)
+// nparts: the CTAs (blockIdx.x = 0 .. nparts - 1) that work on worker i; others leave at once.
+// G: sample groups per thread (nparts * G * BEGIN_BLOCK >= S).
+template <int GT, int G>
+__device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, const void *__restrict__ grads,
+                                                float alpha, uint32_t exact_all, uint32_t S, const uint32_t nparts)
 {
-    const uint32_t i = blockIdx.y, part = blockIdx.x;
+    const uint32_t part = blockIdx.x;
+    if (part >= nparts) return;
     const int t = threadIdx.x;
     SelectState &s = p.sel[i];
     uint32_t *hz = hist_of(p, i, 0, 0);
     for (int q = part * BEGIN_BLOCK + t; q < 2 * RADIX_LEVELS * RADIX_BINS;
-         q += gridDim.x * BEGIN_BLOCK)
+         q += nparts * BEGIN_BLOCK)
         hz[q] = 0;
     if (part == 0) {
         if (t < 3) p.done[i * DONE_SLOTS + t] = 0;          // levels A, B, classification
@@ -377,35 +393,45 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     const uint64_t nchunks = (p.d + 3) >> 2;
     uint4 *skeys = reinterpret_cast<uint4 *>(p.sample_keys) + static_cast<size_t>(i) * SAMPLE_CHUNKS;
     {
-        const uint32_t sidx = part * BEGIN_BLOCK + t;
-        uint32_t kk[4] = {0, 0, 0, 0};                       // 0 = "not a sample"
-        if (sidx < S) {
-            const uint64_t j = ((static_cast<uint64_t>(sidx) * nchunks) / S) << 2;
-            if (p.rk.on) {
-                const uint4 r4 = rand_keys4(p.rk, i, j >> 2);
-                const uint32_t rs[4] = {r4.x, r4.y, r4.z, r4.w};
+        // G sample groups per thread, all loads issued before the first use
+        uint32_t kk[G][4];
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (j + c < p.d) kk[c] = rs[c];
-            } else {
-                const float4 ev = *reinterpret_cast<const float4 *>(erow + j);
-                const float es[4] = {ev.x, ev.y, ev.z, ev.w};
+        for (int gq = 0; gq < G; ++gq) {
+            const uint32_t sidx = (part * G + gq) * BEGIN_BLOCK + t;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (j + c < p.d)
-                        kk[c] = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
+            for (int c = 0; c < 4; ++c) kk[gq][c] = 0;           // 0 = "not a sample"
+            if (sidx < S) {
+                const uint64_t j = ((static_cast<uint64_t>(sidx) * nchunks) / S) << 2;
+                if (p.rk.on) {
+                    const uint4 r4 = rand_keys4(p.rk, i, j >> 2);
+                    const uint32_t rs[4] = {r4.x, r4.y, r4.z, r4.w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if (j + c < p.d) kk[gq][c] = rs[c];
+                } else {
+                    const float4 ev = *reinterpret_cast<const float4 *>(erow + j);
+                    const float es[4] = {ev.x, ev.y, ev.z, ev.w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if (j + c < p.d)
+                            kk[gq][c] = mag_key(__fmaf_rn(alpha, load_g<GT>(grow, j + c), es[c]));
+                }
             }
         }
-        skeys[sidx] = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+#pragma unroll
+        for (int gq = 0; gq < G; ++gq)
+            skeys[(part * G + gq) * BEGIN_BLOCK + t] = make_uint4(kk[gq][0], kk[gq][1], kk[gq][2], kk[gq][3]);
         // histogram of the top SAMPLE_HIST_BITS key bits of this CTA's nonzero keys: lanes
         // with the same bin elect one of them to add the group's size
 #pragma unroll
         for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) s_buf[c * BEGIN_BLOCK + t] = 0;
         __syncthreads();
-        {
+#pragma unroll
+        for (int gq = 0; gq < G; ++gq) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const uint32_t hb = kk[c] ? min(kk[c] >> p.sample_shift, SAMPLE_HIST_BINS - 1) : SAMPLE_HIST_BINS;
+                const uint32_t key = kk[gq][c];
+                const uint32_t hb = key ? min(key >> p.sample_shift, SAMPLE_HIST_BINS - 1) : SAMPLE_HIST_BINS;
                 const uint32_t grp = __match_any_sync(FULL, hb);
                 if (hb < SAMPLE_HIST_BINS && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_buf[hb], __popc(grp));
             }
@@ -419,7 +445,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     }
     // the arrival counter resets itself: only the last CTA touches it afterwards
     uint32_t *arrive = &p.done[i * DONE_SLOTS + 3];
-    if (!last_cta_to_arrive(arrive, &s_flag)) return;
+    if (!last_cta_to_arrive(arrive, &s_flag, nparts)) return;
     if (t == 0) *arrive = 0;
 
     // every sampled group is complete unless the sample is the whole vector
@@ -437,7 +463,7 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
         // how far the sampled rank sits above k/d decides how far above the bound the
         // threshold may lie (in value: that ratio to the power 1/tail-index)
         const double rho = static_cast<double>(R) / (mean > 1e-9 ? mean : 1e-9);
-        rel_shift = rho <= 2.0 ? 10u : (rho <= 8.0 ? 11u : 12u);
+        rel_shift = rho <= 1.5 ? 10u : (rho <= 1.75 ? 11u : 12u);
         if (p.rk.on) rel_shift = 10u;          // uniform 23-bit priorities: 4095 << 10 is half the range
     }
     uint32_t *gh = p.sample_hist + i * SAMPLE_HIST_BINS;
@@ -573,6 +599,13 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
     }
 }
 
+template <int GT>
+__global__ void __launch_bounds__(BEGIN_BLOCK, 2)
+begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t exact_all, uint32_t S)
+{
+    begin_step_body<GT, 1>(p, blockIdx.y, grads, alpha, exact_all, S, gridDim.x);
+}
+
 // ------------------------------------------------------------------------------------------
 // Streaming pass.  GT = 0: fp32 gradients; GT = 1: bfloat16 gradients.  ALIGNED: every
 // gradient row starts on a 16-byte boundary, so whole tiles are read with 128-bit loads;
@@ -580,23 +613,23 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
 // entry.  SPEC: stage the entries whose key reaches sel[i].spec_key.
 // ------------------------------------------------------------------------------------------
 template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
-__global__ void __launch_bounds__(BLOCK)
-ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
-                     uint64_t d, uint64_t g_stride, float alpha, RandParams rk, SelectState *__restrict__ sel,
-                     deco_pair *__restrict__ stage, uint64_t stage_cap,
-                     uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
-                     uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
-                     uint32_t ntiles)
+__device__ __forceinline__ void
+ef_accumulate_body(const uint32_t tile, const uint32_t i, const bool rows_aligned,
+                   float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
+                   uint64_t d, uint64_t g_stride, float alpha, const RandParams &rk, SelectState *__restrict__ sel,
+                   deco_pair *__restrict__ stage, uint64_t stage_cap,
+                   uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
+                   uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
+                   uint32_t ntiles)
 {
     constexpr int V = Geo<GT>::V, U = Geo<GT>::U;
-    const uint32_t tile = blockIdx.x, i = blockIdx.y;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     float *erow = e + static_cast<size_t>(i) * e_stride;
     const char *grow = reinterpret_cast<const char *>(grads) +
                        static_cast<size_t>(i) * g_stride * (GT ? 2 : 4);
     const uint64_t tile_base = static_cast<uint64_t>(tile) * TILE;
     const uint64_t wbase = tile_base + static_cast<uint64_t>(w) * WARP_ELEMS;
-    const bool full = ALIGNED && (tile_base + TILE <= d);
+    const bool full = ALIGNED && rows_aligned && (tile_base + TILE <= d);
 
     float x[U][V];
     if (full) {
@@ -735,6 +768,20 @@ ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__res
     }
 }
 
+template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
+__global__ void __launch_bounds__(BLOCK)
+ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
+                     uint64_t d, uint64_t g_stride, float alpha, RandParams rk, SelectState *__restrict__ sel,
+                     deco_pair *__restrict__ stage, uint64_t stage_cap,
+                     uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
+                     uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
+                     uint32_t ntiles)
+{
+    ef_accumulate_body<GT, ALIGNED, SPEC, RANDK>(blockIdx.x, blockIdx.y, true, e, e_stride, grads, d, g_stride,
+                                                 alpha, rk, sel, stage, stage_cap, tile_off, tile_cnt,
+                                                 tile_rej, tile_eq, ntiles);
+}
+
 // ------------------------------------------------------------------------------------------
 // Streaming route: exact selection among the staged pairs.
 // ------------------------------------------------------------------------------------------
@@ -800,10 +847,8 @@ __device__ __forceinline__ void build_emit_work(const Sel &p, uint32_t i)
 // k largest, and no overflow of the staging area), and which coarse bin holds the k-th
 // largest.  If the set is not usable, or the threshold falls into the shared top bin, the
 // worker is handed to the multi-pass route.
-__global__ void __launch_bounds__(BLOCK)
-stage_hist_a_kernel(Sel p)
+__device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i)
 {
-    const uint32_t i = blockIdx.y;
     SelectState &s = p.sel[i];
     if (s.exact) return;
     const uint32_t n_staged = s.n_staged, spec = s.spec_key, shift = s.rel_shift;
@@ -853,10 +898,10 @@ stage_hist_a_kernel(Sel p)
 
 // Level B: histogram of the low bits of the staged keys that fell into the chosen A bin; the
 // last CTA of a worker to arrive fixes the threshold key and the number of ties to take.
-__global__ void __launch_bounds__(BLOCK)
-stage_hist_b_kernel(Sel p)
+__global__ void __launch_bounds__(BLOCK) stage_hist_a_kernel(Sel p) { stage_hist_a_body(p, blockIdx.y); }
+
+__device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i)
 {
-    const uint32_t i = blockIdx.y;
     SelectState &s = p.sel[i];
     if (s.exact) return;
     __shared__ uint32_t h[RADIX_BINS];
@@ -907,6 +952,8 @@ stage_hist_b_kernel(Sel p)
         }
     }
 }
+
+__global__ void __launch_bounds__(BLOCK) stage_hist_b_kernel(Sel p) { stage_hist_b_body(p, blockIdx.y); }
 
 // One CTA: ties are granted to chunks in index order until ties_take are used up, then every
 // chunk gets its position in the message.  Per thread a contiguous range of chunks.  With
@@ -973,10 +1020,8 @@ __device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, 
 
 // Many chunks: their sums are taken in parallel, one warp per chunk (three coalesced loads
 // and a warp reduction), and the last CTA of a worker to arrive walks the chunks.
-__global__ void __launch_bounds__(BLOCK)
-chunk_sums_kernel(Sel p)
+__device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i)
 {
-    const uint32_t i = blockIdx.y;
     if (p.sel[i].exact) return;
     __shared__ uint32_t s_scan[33];
     __shared__ uint32_t s_flag;
@@ -1006,15 +1051,15 @@ chunk_sums_kernel(Sel p)
     chunk_walk(p, i, s_scan, true);
 }
 
+__global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p) { chunk_sums_body(p, blockIdx.y); }
+
 // Classification.  With the threshold known every staged entry below it is rejected: counted
 // for its tile and its chunk (CHUNK_TILES consecutive tiles) and given its value back in e;
 // entries equal to it are counted as ties.  With few chunks (walk_here) the last CTA of a worker
 // to arrive then walks the chunks once; with many, chunk_sums_kernel follows.  (The per-tile positions follow from these inside the
 // emit kernel, so nothing here is serial in the number of tiles.)
-__global__ void __launch_bounds__(BLOCK)
-stage_classify_kernel(Sel p, uint32_t walk_here)
+__device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t i, uint32_t walk_here)
 {
-    const uint32_t i = blockIdx.y;
     const SelectState &s = p.sel[i];
     if (s.exact) return;
     __shared__ uint32_t s_scan[33];
@@ -1069,6 +1114,11 @@ stage_classify_kernel(Sel p, uint32_t walk_here)
     }
     if (walk_here) chunk_walk(p, i, s_scan, false);
     write_back_rejected();
+}
+
+__global__ void __launch_bounds__(BLOCK) stage_classify_kernel(Sel p, uint32_t walk_here)
+{
+    stage_classify_body(p, blockIdx.y, walk_here);
 }
 
 // What a warp learns about the CHUNK_TILES tiles of one chunk from three coalesced loads and
@@ -1166,10 +1216,8 @@ __device__ __forceinline__ uint32_t emit_segment_warp(const Sel &p, uint32_t i, 
 // directory and each lane walks its own tile if that holds at most EMIT_LANE_MAX staged
 // entries.  The remaining CTAs: their warps stride over the work list; a warp that gets slice
 // j > 0 of a tile first counts, with independent loads, what the slices before it emit.
-__global__ void __launch_bounds__(BLOCK)
-emit_stage_kernel(Sel p, uint32_t dir_ctas)
+__device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, uint32_t dir_ctas)
 {
-    const uint32_t i = blockIdx.y;
     if (p.sel[i].exact) return;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t T = p.sel[i].threshold;
@@ -1250,6 +1298,11 @@ emit_stage_kernel(Sel p, uint32_t dir_ctas)
         if (end == cnt && lane == 0 && written != want)
             latch(p.status, DECO_ERR_DEVICE_CHECK, 0x311u, tile);
     }
+}
+
+__global__ void __launch_bounds__(BLOCK) emit_stage_kernel(Sel p, uint32_t dir_ctas)
+{
+    emit_stage_body(p, blockIdx.y, dir_ctas);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1548,12 +1601,9 @@ __global__ void __launch_bounds__(BLOCK) emit_e_kernel(Sel p)
 // ---- fallback of the streaming route: the whole multi-pass route in one cooperative launch.
 // Leaves at once unless some worker's staged set was rejected.  All CTAs take every
 // grid-wide barrier: the decision to leave is the same for the whole grid.
-__global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
+__device__ __forceinline__ void exact_fallback_body(const Sel &p, cg::grid_group &grid, uint32_t *h,
+                                                    uint32_t *s_a, uint32_t *s_b, uint32_t *s_out)
 {
-    if (__ldcg(&p.status[3]) == 0) return;
-    cg::grid_group grid = cg::this_grid();
-    __shared__ uint32_t h[RADIX_BINS];
-    __shared__ uint32_t s_a[33], s_b[WARPS], s_out[2];
     const uint32_t cta = blockIdx.x, ncta = gridDim.x;
     // The streaming pass wrote +0 over the staged entries of every tile whose segment fitted;
     // the passes below need the values back.
@@ -1610,6 +1660,146 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
             emit_e_tile(p, i, tile, s_b);
             __syncthreads();
         }
+    }
+}
+
+__global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
+{
+    if (__ldcg(&p.status[3]) == 0) return;
+    cg::grid_group grid = cg::this_grid();
+    __shared__ uint32_t h[RADIX_BINS];
+    __shared__ uint32_t s_a[33], s_b[WARPS], s_out[2];
+    exact_fallback_body(p, grid, h, s_a, s_b, s_out);
+}
+
+// ------------------------------------------------------------------------------------------
+// Many contexts in one launch (per-layer Top-k: one context per layer, all with n workers).
+// Row y of the grid is worker y % n of layer y / n; the layer's parameters come from a table
+// in device memory.  Every selection kernel above strides over its work by gridDim.x and
+// counts gridDim.x arrivals per worker, so one grid width serves layers of any size; the
+// sampling kernel is told how many CTAs each layer uses, and the streaming pass, which has one
+// CTA per tile, finds its layer from the tile number.
+// ------------------------------------------------------------------------------------------
+struct MultiLayer {
+    Sel p;
+    uint64_t g_off;          // entries from the start of a gradient row to the layer
+    uint32_t S;              // sample groups of begin_step
+    uint32_t walk_here;      // classification walks the chunks itself (few chunks)
+    uint32_t rows_aligned;   // the layer's gradient rows start on 16-byte boundaries
+    uint32_t pad;
+};
+
+// With hundreds of (layer, worker) rows the sampling kernel is bound by the number of CTAs it
+// has to get through, so each thread takes several sample groups.
+constexpr int MULTI_BEGIN_GROUPS = 4;
+
+template <int GT>
+__global__ void __launch_bounds__(BEGIN_BLOCK, 2)
+begin_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, const void *__restrict__ grads,
+                        float alpha)
+{
+    const MultiLayer &m = table[blockIdx.y / n];
+    constexpr uint32_t PER_CTA = MULTI_BEGIN_GROUPS * BEGIN_BLOCK;
+    if (blockIdx.x * PER_CTA >= m.S) return;
+    const Sel p = m.p;
+    const char *g = static_cast<const char *>(grads) + m.g_off * (GT ? 2 : 4);
+    begin_step_body<GT, MULTI_BEGIN_GROUPS>(p, blockIdx.y % n, g, alpha, 0u, m.S, (m.S + PER_CTA - 1) / PER_CTA);
+}
+
+// The streaming pass of many layers.  Its per-layer arguments travel as a kernel parameter
+// (constant bank: no dependent global load before the tile's own loads can be issued); the
+// layer of a tile is found by bisection over the layers' first tiles.  ALIGNED: the launch for
+// the layers whose gradient rows start on 16-byte boundaries (tiles of the other layers leave
+// at once); !ALIGNED: the launch for the others, if there are any.
+constexpr int ACC_LAYERS_MAX = 256;
+struct AccLayer {
+    float *e;
+    deco_pair *stage;
+    SelectState *sel;
+    uint32_t *tile_off, *tile_cnt, *tile_rej, *tile_eq;
+    uint64_t e_stride, stage_cap, d, g_off;
+    uint32_t ntiles, first_tile;     // first_tile: relative to the table's first layer
+    uint32_t rows_aligned, pad;
+};
+struct AccTable {
+    AccLayer L[ACC_LAYERS_MAX];
+    uint32_t count, pad;
+};
+static_assert(sizeof(AccTable) < 32000, "kernel parameters are limited to 32764 bytes");
+
+template <int GT, bool ALIGNED>
+__global__ void __launch_bounds__(BLOCK, 3)
+ef_accumulate_multi_kernel(const __grid_constant__ AccTable tab, const void *__restrict__ grads,
+                           uint64_t g_stride, float alpha)
+{
+    uint32_t lo = 0, hi = tab.count;                         // the layer lies in [lo, hi)
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (tab.L[mid].first_tile <= blockIdx.x) lo = mid;
+        else hi = mid;
+    }
+    const AccLayer &m = tab.L[lo];
+    if ((m.rows_aligned != 0) != ALIGNED) return;
+    const char *g = static_cast<const char *>(grads) + m.g_off * (GT ? 2 : 4);
+    RandParams rk;
+    rk.on = 0;
+    rk.seed_lo = rk.seed_hi = rk.step_lo = rk.step_hi = rk.worker_base = 0;
+    ef_accumulate_body<GT, ALIGNED, true, false>(blockIdx.x - m.first_tile, blockIdx.y, true, m.e, m.e_stride, g,
+                                                 m.d, g_stride, alpha, rk, m.sel, m.stage, m.stage_cap,
+                                                 m.tile_off, m.tile_cnt, m.tile_rej, m.tile_eq, m.ntiles);
+}
+
+__global__ void __launch_bounds__(BLOCK) stage_hist_a_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
+{
+    const Sel p = table[blockIdx.y / n].p;
+    stage_hist_a_body(p, blockIdx.y % n);
+}
+
+__global__ void __launch_bounds__(BLOCK) stage_hist_b_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
+{
+    const Sel p = table[blockIdx.y / n].p;
+    stage_hist_b_body(p, blockIdx.y % n);
+}
+
+__global__ void __launch_bounds__(BLOCK) stage_classify_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
+{
+    const MultiLayer &m = table[blockIdx.y / n];
+    const Sel p = m.p;
+    stage_classify_body(p, blockIdx.y % n, m.walk_here);
+}
+
+__global__ void __launch_bounds__(BLOCK) chunk_sums_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
+{
+    const MultiLayer &m = table[blockIdx.y / n];
+    if (m.walk_here) return;                                 // the classification did the walk
+    const Sel p = m.p;
+    chunk_sums_body(p, blockIdx.y % n);
+}
+
+__global__ void __launch_bounds__(BLOCK)
+emit_stage_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, uint32_t dir_ctas)
+{
+    const Sel p = table[blockIdx.y / n].p;
+    emit_stage_body(p, blockIdx.y % n, dir_ctas);
+}
+
+// Cooperative: the layers with a rejected staged set, one after the other.  Which layers those
+// are is read from memory that no CTA of this kernel writes, so every CTA takes the same
+// barriers.
+__global__ void __launch_bounds__(BLOCK) exact_fallback_multi_kernel(const MultiLayer *__restrict__ table, uint32_t layers)
+{
+    // nothing to do (the usual case): every thread looks at one layer's flag
+    int any = 0;
+    for (uint32_t l = threadIdx.x; l < layers; l += BLOCK) any |= __ldcg(&table[l].p.status[3]) != 0;
+    if (!__syncthreads_or(any)) return;
+    cg::grid_group grid = cg::this_grid();
+    __shared__ uint32_t h[RADIX_BINS];
+    __shared__ uint32_t s_a[33], s_b[WARPS], s_out[2];
+    for (uint32_t l = 0; l < layers; ++l) {
+        if (__ldcg(&table[l].p.status[3]) == 0) continue;
+        const Sel p = table[l].p;
+        exact_fallback_body(p, grid, h, s_a, s_b, s_out);
+        __syncthreads();
     }
 }
 
@@ -1803,6 +1993,174 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     err = cudaLaunchCooperativeKernel(reinterpret_cast<void *>(exact_fallback_kernel),
                                       dim3(c->fallback_grid), dim3(BLOCK), args, 0, s);
     c->launches += 1;
+    return err;
+}
+
+// ------------------------------------------------------------------------------------------
+// Worker side of many contexts (the layers of the per-layer variant) in a fixed number of
+// launches.
+// ------------------------------------------------------------------------------------------
+struct MultiPlan {
+    std::vector<deco_ctx *> layers;
+    std::vector<uint64_t> g_off;
+    std::vector<MultiLayer> host;
+    MultiLayer *dev = nullptr;
+    uint32_t n = 0;
+    int grad_dtype = DECO_F32;
+    uint32_t fallback_grid = 0;
+    bool dirty = true;
+    // streaming pass: the layers in groups of at most ACC_LAYERS_MAX, one launch (or two) each
+    struct AccGroup {
+        AccTable tab;
+        uint32_t tiles = 0;
+        bool any_aligned = false, any_unaligned = false;
+    };
+    std::vector<AccGroup> acc;
+    // grid widths shared by all layers
+    uint32_t begin_ctas = 1, stage_ctas = 1, chunk_ctas = 0, dir_ctas = 1, item_ctas = 1;
+};
+
+MultiPlan *multi_plan_create(const std::vector<deco_ctx *> &layers, const std::vector<uint64_t> &g_off,
+                             uint32_t n, int grad_dtype)
+{
+    if (layers.empty()) return nullptr;
+    MultiPlan *mp = new (std::nothrow) MultiPlan();
+    if (!mp) return nullptr;
+    try {
+        mp->layers = layers;
+        mp->g_off = g_off;
+        mp->host.resize(layers.size());
+        mp->n = n;
+        mp->grad_dtype = grad_dtype;
+        int per_sm = 0, sms = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, exact_fallback_multi_kernel, BLOCK, 0) !=
+                cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, layers[0]->device) != cudaSuccess ||
+            per_sm < 1)
+            throw 1;
+        mp->fallback_grid = static_cast<uint32_t>((per_sm > 4 ? 4 : per_sm) * sms);
+        if (cudaMalloc(reinterpret_cast<void **>(&mp->dev), sizeof(MultiLayer) * layers.size()) != cudaSuccess)
+            throw 2;
+    } catch (...) {
+        cudaGetLastError();
+        multi_plan_destroy(mp);
+        return nullptr;
+    }
+    return mp;
+}
+
+void multi_plan_destroy(MultiPlan *mp)
+{
+    if (!mp) return;
+    cudaFree(mp->dev);
+    delete mp;
+}
+
+void multi_plan_mark_dirty(MultiPlan *mp)
+{
+    if (mp) mp->dirty = true;
+}
+
+// Table and grid widths for the layers' current k (after a policy change).
+static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStream_t s)
+{
+    const uint32_t L = static_cast<uint32_t>(mp->layers.size());
+    const uint64_t esz = mp->grad_dtype == DECO_BF16 ? 2 : 4;
+    uint64_t begin_max = 1, stage_max = 1, chunk_max = 0, dir_max = 1, item_max = 1;
+    for (uint32_t l = 0; l < L; ++l) {
+        const deco_ctx *c = mp->layers[l];
+        MultiLayer &m = mp->host[l];
+        m.p = make_sel(c);
+        m.g_off = mp->g_off[l];
+        m.S = sample_groups(c->d, c->k);
+        m.walk_here = c->nchunks <= 256 ? 1u : 0u;
+        m.rows_aligned = ((mp->g_off[l] * esz) % 16 == 0 && (c->g_stride * esz) % 16 == 0) ? 1u : 0u;
+        begin_max = std::max<uint64_t>(begin_max, (m.S + MULTI_BEGIN_GROUPS * BEGIN_BLOCK - 1) /
+                                                      (MULTI_BEGIN_GROUPS * BEGIN_BLOCK));
+        stage_max = std::max<uint64_t>(stage_max, (2 * c->k + 65536 + BLOCK * 4 - 1) / (BLOCK * 4));
+        if (!m.walk_here) chunk_max = std::max<uint64_t>(chunk_max, (c->nchunks + WARPS - 1) / WARPS);
+        dir_max = std::max<uint64_t>(dir_max, (c->nchunks + WARPS - 1) / WARPS);
+        const uint64_t staged = 13 * c->k / 10, many = staged / (EMIT_LANE_MAX + 1);
+        const uint64_t est_items = staged / EMIT_SLICE + (many < c->ntiles ? many : c->ntiles);
+        item_max = std::max<uint64_t>(item_max, (est_items + WARPS - 1) / WARPS + 1);
+    }
+    mp->acc.assign((L + ACC_LAYERS_MAX - 1) / ACC_LAYERS_MAX, MultiPlan::AccGroup());
+    for (uint32_t l = 0; l < L; ++l) {
+        const MultiLayer &m = mp->host[l];
+        MultiPlan::AccGroup &grp = mp->acc[l / ACC_LAYERS_MAX];
+        AccLayer &a = grp.tab.L[l % ACC_LAYERS_MAX];
+        a.e = m.p.e;
+        a.stage = m.p.stage;
+        a.sel = m.p.sel;
+        a.tile_off = m.p.tile_off;
+        a.tile_cnt = m.p.tile_cnt;
+        a.tile_rej = m.p.tile_rej;
+        a.tile_eq = m.p.tile_eq;
+        a.e_stride = m.p.e_stride;
+        a.stage_cap = m.p.stage_cap;
+        a.d = m.p.d;
+        a.g_off = m.g_off;
+        a.ntiles = m.p.ntiles;
+        a.first_tile = grp.tiles;
+        a.rows_aligned = m.rows_aligned;
+        a.pad = 0;
+        grp.tiles += m.p.ntiles;
+        grp.tab.count = l % ACC_LAYERS_MAX + 1;
+        grp.tab.pad = 0;
+        (m.rows_aligned ? grp.any_aligned : grp.any_unaligned) = true;
+    }
+    // a few waves of the device in all: rows = layers * n
+    const uint64_t rows = static_cast<uint64_t>(L) * mp->n;
+    const uint64_t cap = std::max<uint64_t>(1, (148ull * 8 * 4 + rows - 1) / rows);
+    mp->begin_ctas = static_cast<uint32_t>(begin_max);
+    mp->stage_ctas = static_cast<uint32_t>(std::min(stage_max, cap));
+    mp->chunk_ctas = static_cast<uint32_t>(chunk_max);
+    mp->dir_ctas = static_cast<uint32_t>(dir_max);
+    mp->item_ctas = static_cast<uint32_t>(std::min(item_max, std::max<uint64_t>(1, 2 * cap)));
+    (void)grads;
+    // the host table is pageable: the copy has left it when the call returns
+    const cudaError_t err = cudaMemcpyAsync(mp->dev, mp->host.data(), sizeof(MultiLayer) * L,
+                                            cudaMemcpyHostToDevice, s);
+    if (err == cudaSuccess) mp->dirty = false;
+    return err;
+}
+
+cudaError_t multi_compress(MultiPlan *mp, const void *grads, float alpha, cudaStream_t s)
+{
+    if (mp->dirty) {
+        const cudaError_t err = multi_plan_refresh(mp, grads, s);
+        if (err != cudaSuccess) return err;
+    }
+    const uint32_t L = static_cast<uint32_t>(mp->layers.size()), n = mp->n, rows = L * n;
+    const bool bf16 = mp->grad_dtype == DECO_BF16;
+    if (bf16) begin_step_multi_kernel<1><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
+    else begin_step_multi_kernel<0><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
+    const uint64_t g_stride = mp->layers[0]->g_stride;
+    for (const MultiPlan::AccGroup &grp : mp->acc) {
+        const dim3 agrid(grp.tiles, n);
+        if (grp.any_aligned) {
+            if (bf16) ef_accumulate_multi_kernel<1, true><<<agrid, BLOCK, 0, s>>>(grp.tab, grads, g_stride, alpha);
+            else ef_accumulate_multi_kernel<0, true><<<agrid, BLOCK, 0, s>>>(grp.tab, grads, g_stride, alpha);
+        }
+        if (grp.any_unaligned) {
+            if (bf16) ef_accumulate_multi_kernel<1, false><<<agrid, BLOCK, 0, s>>>(grp.tab, grads, g_stride, alpha);
+            else ef_accumulate_multi_kernel<0, false><<<agrid, BLOCK, 0, s>>>(grp.tab, grads, g_stride, alpha);
+        }
+    }
+    const dim3 sgrid(mp->stage_ctas, rows);
+    stage_hist_a_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, n);
+    stage_hist_b_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, n);
+    stage_classify_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, n);
+    if (mp->chunk_ctas) chunk_sums_multi_kernel<<<dim3(mp->chunk_ctas, rows), BLOCK, 0, s>>>(mp->dev, n);
+    emit_stage_multi_kernel<<<dim3(mp->dir_ctas + mp->item_ctas, rows), BLOCK, 0, s>>>(mp->dev, n, mp->dir_ctas);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    const MultiLayer *tab = mp->dev;
+    uint32_t layers = L;
+    void *args[] = {&tab, &layers};
+    err = cudaLaunchCooperativeKernel(reinterpret_cast<void *>(exact_fallback_multi_kernel),
+                                      dim3(mp->fallback_grid), dim3(BLOCK), args, 0, s);
+    mp->layers[0]->launches += mp->chunk_ctas ? 9 : 8;
     return err;
 }
 

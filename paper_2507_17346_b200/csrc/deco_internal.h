@@ -159,6 +159,80 @@ inline cudaError_t wait_for_aggregate(deco_ctx *c, cudaStream_t s)
     c->agg_pending = false;
     return cudaStreamWaitEvent(s, c->ev_agg, 0);
 }
+// --- worker side of many contexts in a fixed number of launches (deco_compress.cu) ----------
+// All contexts have n workers, Top-k on the streaming route, and read their gradients from one
+// buffer of rows of g_stride entries, context l at entry g_off[l] of every row.
+struct MultiPlan;
+MultiPlan *multi_plan_create(const std::vector<deco_ctx *> &layers, const std::vector<uint64_t> &g_off,
+                             uint32_t n, int grad_dtype);
+void multi_plan_destroy(MultiPlan *mp);
+void multi_plan_mark_dirty(MultiPlan *mp);       // some context's k changed
+// begin_step .. fallback of every context on stream s; the contexts' host state is untouched
+cudaError_t multi_compress(MultiPlan *mp, const void *grads, float alpha, cudaStream_t s);
+// host state of c after its worker side was run by multi_compress: ready for deco_aggregate_stale
+deco_status mark_compressed_external(deco_ctx *c);
+
+// --- server side of many contexts in a fixed number of launches (deco_server.cu) ------------
+struct ServerLayer {
+    const deco_pair *msg;    // [n][k_cap]
+    uint64_t k_cap;
+    const uint32_t *tile_start;
+    deco_pair *slots;        // [ring][n * k_cap]
+    float *params;
+    uint32_t *status;
+    uint32_t *slot_pos;      // [ring] positions held by each cache slot (written on the device)
+    uint64_t d;
+    uint32_t ntiles, first_tile;
+    uint32_t k;              // entries kept per worker at the current delta
+    uint32_t dense;          // aggregate with the CTA-wide accumulator (many entries per tile)
+};
+bool aggregate_prefers_dense(const deco_ctx *c);
+// all layers' messages into cache slot slot_write of each (tiles numbered across the layers)
+cudaError_t launch_multi_aggregate(const ServerLayer *table, const uint32_t *tile_layer, uint32_t total_tiles,
+                                   uint32_t n, uint32_t slot_write, bool any_dense, bool any_sparse,
+                                   cudaStream_t s);
+// cache slot slot_read of every layer onto its parameters
+cudaError_t launch_multi_apply(const ServerLayer *table, uint32_t layers, uint32_t n, uint32_t ctas_per_layer,
+                               uint32_t slot_read, float neg_scale, cudaStream_t s);
+
+// --- batch of short layers (per-layer Top-k): deco_small.cu, deco_server.cu ---------------
+// One entry per layer of at most TILE entries; the table lives in device memory.  All pointers
+// are the buffers of that layer's own context, in their usual layouts.
+struct SmallLayer {
+    float *e;                // [n][e_stride]
+    uint64_t e_stride;
+    uint64_t g_off;          // entries from the start of a gradient row to the layer
+    deco_pair *msg;          // [n][k_cap]
+    uint64_t k_cap;
+    deco_pair *slots;        // [ring][n * k_cap]
+    uint32_t *tile_start;    // [n][2]
+    SelectState *sel;        // [n]
+    float *params;           // the layer's slice of the parameter vector
+    uint32_t *status;        // the context's device status words
+    uint32_t *slot_pos;      // [ring] positions held by each cache slot (written on the device)
+    uint32_t d;              // entries of the layer
+    uint32_t k;              // entries kept per worker at the current delta
+};
+
+constexpr int SMALL_DUE_MAX = 16;        // cache slots one server launch can apply
+struct SmallDue {
+    uint32_t count;
+    uint32_t slot[SMALL_DUE_MAX];        // slot numbers, oldest aggregate first
+};
+
+// worker side of every listed layer for all n workers: one CTA per (layer, worker)
+cudaError_t launch_small_workers(const SmallLayer *table, uint32_t layers, uint32_t n, const void *grads,
+                                 uint64_t g_stride, int grad_dtype, float alpha, cudaStream_t s);
+// server side of every listed layer: aggregate the n messages into cache slot `slot_write`
+// (unless aggregate is false), then apply the listed slots, oldest first; one CTA per layer
+cudaError_t launch_small_server(const SmallLayer *table, uint32_t layers, uint32_t n, bool aggregate,
+                                uint32_t slot_write, const SmallDue &due, float neg_scale, cudaStream_t s);
+
+// Host bookkeeping of one whole iteration of c whose device work is done by the batch kernels:
+// the cache slot of iteration t becomes valid, the slots due at t are appended to `due` (slot
+// numbers, oldest first) and marked applied, t advances.  Returns the slot written.
+uint32_t advance_iteration_external(deco_ctx *c, std::vector<uint32_t> *due);
+
 // --- kernel launchers (deco_server.cu) ---------------------------------------------------
 cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s);
 cudaError_t launch_apply(deco_ctx *c, const deco_pair *slot, uint64_t positions, float neg_scale,

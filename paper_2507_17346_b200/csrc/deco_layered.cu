@@ -6,8 +6,13 @@
 // layer's columns starting at its offset) and the parameter vector (the layer's slice).  The
 // layers are stepped round-robin on a few internal streams forked from and joined back into
 // the caller's stream.
+//
+// Layers of at most one tile (Top-k on the streaming route) are not stepped one by one: their
+// contexts only hold the buffers, and two launches do the device work of all of them (one CTA
+// per layer and worker for the worker side, one CTA per layer for aggregation and update).
 #include "deco_internal.h"
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -28,6 +33,24 @@ struct deco_layered {
     cudaEvent_t ev_fork = nullptr;
     cudaEvent_t ev_done[LAYER_STREAMS] = {};
     uint64_t t = 0;
+    // the short layers that are stepped as one batch
+    std::vector<uint32_t> small;                 // their layer numbers
+    std::vector<uint32_t> big;                   // all other layers
+    std::vector<deco::SmallLayer> small_host;    // the table, host copy
+    deco::SmallLayer *small_dev = nullptr;
+    uint32_t *small_slot_pos = nullptr;          // [small][ring]
+    bool small_dirty = true;                     // k changed: upload the table before the next step
+    // the other layers' worker side runs in a fixed number of launches when they all use
+    // Top-k on the streaming route
+    deco::MultiPlan *plan = nullptr;
+    std::vector<deco::ServerLayer> server_host;  // one entry per layer of `big`
+    deco::ServerLayer *server_dev = nullptr;
+    uint32_t *big_tile_layer = nullptr;          // device: layer (position in `big`) of every tile
+    uint32_t *big_slot_pos = nullptr;            // device: [big][ring]
+    uint32_t big_tiles = 0;
+    bool server_dirty = true;
+    bool any_dense = false, any_sparse = false;
+    uint32_t apply_ctas = 1;
 };
 
 namespace {
@@ -53,8 +76,189 @@ void release(deco_layered *L)
     for (cudaEvent_t e : L->ev_done)
         if (e) cudaEventDestroy(e);
     if (L->ev_fork) cudaEventDestroy(L->ev_fork);
+    deco::multi_plan_destroy(L->plan);
+    cudaFree(L->server_dev);
+    cudaFree(L->big_tile_layer);
+    cudaFree(L->big_slot_pos);
+    cudaFree(L->small_dev);
+    cudaFree(L->small_slot_pos);
     if (L->own_params) cudaFree(L->params);
     delete L;
+}
+
+// Sort the layers into the batch of short ones and the rest, and build the batch's table.
+cudaError_t build_small_batch(deco_layered *L)
+{
+    for (uint32_t l = 0; l < L->layers.size(); ++l) {
+        const deco_ctx *c = L->layers[l];
+        const bool is_small = c->d <= static_cast<uint64_t>(deco::TILE) &&
+                              c->compressor == DECO_COMPRESSOR_TOPK &&
+                              c->select_mode == DECO_SELECT_AUTO && c->n_total == c->n;
+        (is_small ? L->small : L->big).push_back(l);
+    }
+    bool batchable = !L->big.empty();
+    std::vector<deco_ctx *> ctxs;
+    std::vector<uint64_t> offs;
+    for (uint32_t l : L->big) {
+        const deco_ctx *c = L->layers[l];
+        batchable = batchable && c->compressor == DECO_COMPRESSOR_TOPK &&
+                    c->select_mode == DECO_SELECT_AUTO && c->n_total == c->n;
+        ctxs.push_back(L->layers[l]);
+        offs.push_back(L->offsets[l]);
+    }
+    if (batchable) {
+        L->plan = deco::multi_plan_create(ctxs, offs, L->n, L->grad_dtype);
+        if (!L->plan) return cudaErrorMemoryAllocation;
+        const uint32_t ring = ctxs[0]->ring;
+        std::vector<uint32_t> map;
+        L->server_host.resize(ctxs.size());
+        for (size_t q = 0; q < ctxs.size(); ++q) {
+            L->server_host[q].first_tile = static_cast<uint32_t>(map.size());
+            map.insert(map.end(), ctxs[q]->ntiles, static_cast<uint32_t>(q));
+        }
+        L->big_tiles = static_cast<uint32_t>(map.size());
+        cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&L->server_dev),
+                                     sizeof(deco::ServerLayer) * ctxs.size());
+        if (err == cudaSuccess)
+            err = cudaMalloc(reinterpret_cast<void **>(&L->big_tile_layer), sizeof(uint32_t) * map.size());
+        if (err == cudaSuccess)
+            err = cudaMemcpy(L->big_tile_layer, map.data(), sizeof(uint32_t) * map.size(), cudaMemcpyHostToDevice);
+        if (err == cudaSuccess)
+            err = cudaMalloc(reinterpret_cast<void **>(&L->big_slot_pos), sizeof(uint32_t) * ctxs.size() * ring);
+        if (err == cudaSuccess)
+            err = cudaMemset(L->big_slot_pos, 0, sizeof(uint32_t) * ctxs.size() * ring);
+        if (err != cudaSuccess) return err;
+        for (size_t q = 0; q < ctxs.size(); ++q) {
+            const deco_ctx *c = ctxs[q];
+            deco::ServerLayer &e = L->server_host[q];
+            e.msg = c->msg;
+            e.k_cap = c->k_cap;
+            e.tile_start = c->tile_start;
+            e.slots = c->slots;
+            e.params = c->params;
+            e.status = c->dev_status;
+            e.slot_pos = L->big_slot_pos + q * ring;
+            e.d = c->d;
+            e.ntiles = c->ntiles;
+        }
+        L->server_dirty = true;
+    }
+    if (L->small.empty()) return cudaSuccess;
+    const uint32_t ring = L->layers[L->small[0]]->ring;
+    cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&L->small_dev),
+                                 sizeof(deco::SmallLayer) * L->small.size());
+    if (err == cudaSuccess)
+        err = cudaMalloc(reinterpret_cast<void **>(&L->small_slot_pos),
+                         sizeof(uint32_t) * L->small.size() * ring);
+    if (err == cudaSuccess)
+        err = cudaMemset(L->small_slot_pos, 0, sizeof(uint32_t) * L->small.size() * ring);
+    if (err != cudaSuccess) return err;
+    L->small_host.resize(L->small.size());
+    for (size_t q = 0; q < L->small.size(); ++q) {
+        deco_ctx *c = L->layers[L->small[q]];
+        deco::SmallLayer &e = L->small_host[q];
+        e.e = c->e;
+        e.e_stride = c->e_stride;
+        e.g_off = L->offsets[L->small[q]];
+        e.msg = c->msg;
+        e.k_cap = c->k_cap;
+        e.slots = c->slots;
+        e.tile_start = c->tile_start;
+        e.sel = c->sel;
+        e.params = c->params;
+        e.status = c->dev_status;
+        e.slot_pos = L->small_slot_pos + q * ring;
+        e.d = static_cast<uint32_t>(c->d);
+        e.k = static_cast<uint32_t>(c->k);
+    }
+    L->small_dirty = true;
+    return cudaSuccess;
+}
+
+// One iteration of all short layers on stream s: table upload if k changed, worker side,
+// aggregation and update, and the host bookkeeping of every context.
+deco_status step_small_batch(deco_layered *L, const void *grads, cudaStream_t s)
+{
+    if (L->small.empty()) return DECO_OK;
+    const uint32_t layers = static_cast<uint32_t>(L->small.size());
+    deco_ctx *first = L->layers[L->small[0]];
+    for (uint32_t l : L->small)
+        if (L->layers[l]->phase != 0) return DECO_ERR_STATE;
+    if (L->small_dirty) {
+        for (size_t q = 0; q < L->small.size(); ++q)
+            L->small_host[q].k = static_cast<uint32_t>(L->layers[L->small[q]]->k);
+        // the host table is pageable: the copy has left it when the call returns
+        if (cudaMemcpyAsync(L->small_dev, L->small_host.data(), sizeof(deco::SmallLayer) * layers,
+                            cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        L->small_dirty = false;
+    }
+    const float alpha = first->lr_at_server ? 1.0f : first->lr;
+    const float beta = first->lr_at_server ? first->lr : 1.0f;
+    const float neg_scale = -(beta / static_cast<float>(first->n_total));
+    if (deco::launch_small_workers(L->small_dev, layers, L->n, grads, L->d, L->grad_dtype, alpha, s) !=
+        cudaSuccess)
+        return DECO_ERR_CUDA;
+    // every layer shares t, tau and the ring size, so the slots due are the same for all
+    std::vector<uint32_t> due;
+    uint32_t slot_write = 0;
+    for (size_t q = 0; q < L->small.size(); ++q)
+        slot_write = deco::advance_iteration_external(L->layers[L->small[q]], q == 0 ? &due : nullptr);
+    bool aggregate = true;
+    size_t at = 0;
+    do {
+        deco::SmallDue part;
+        part.count = 0;
+        while (at < due.size() && part.count < deco::SMALL_DUE_MAX) part.slot[part.count++] = due[at++];
+        if (deco::launch_small_server(L->small_dev, layers, L->n, aggregate, slot_write, part, neg_scale,
+                                      s) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        aggregate = false;
+    } while (at < due.size());
+    first->launches += 2;
+    return DECO_OK;
+}
+
+// Server side of all layers of `big` on stream s (their messages are complete there), and the
+// host bookkeeping of every context.
+deco_status step_big_server(deco_layered *L, cudaStream_t s)
+{
+    const uint32_t layers = static_cast<uint32_t>(L->big.size());
+    const deco_ctx *first = L->layers[L->big[0]];
+    if (L->server_dirty) {
+        uint64_t most = 1;
+        L->any_dense = L->any_sparse = false;
+        for (uint32_t q = 0; q < layers; ++q) {
+            const deco_ctx *c = L->layers[L->big[q]];
+            L->server_host[q].k = static_cast<uint32_t>(c->k);
+            L->server_host[q].dense = deco::aggregate_prefers_dense(c) ? 1u : 0u;
+            (L->server_host[q].dense ? L->any_dense : L->any_sparse) = true;
+            most = std::max<uint64_t>(most, static_cast<uint64_t>(c->n) * c->k_cap);
+        }
+        // the host table is pageable: the copy has left it when the call returns
+        if (cudaMemcpyAsync(L->server_dev, L->server_host.data(), sizeof(deco::ServerLayer) * layers,
+                            cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        const uint64_t want = (most + 255) / 256, cap = std::max<uint64_t>(1, 148ull * 16 / layers);
+        L->apply_ctas = static_cast<uint32_t>(std::min(want, cap));
+        L->server_dirty = false;
+    }
+    const float beta = first->lr_at_server ? first->lr : 1.0f;
+    const float neg_scale = -(beta / static_cast<float>(first->n_total));
+    // every layer shares t, tau and the ring size, so the slots due are the same for all
+    std::vector<uint32_t> due;
+    uint32_t slot_write = 0;
+    for (uint32_t q = 0; q < layers; ++q)
+        slot_write = deco::advance_iteration_external(L->layers[L->big[q]], q == 0 ? &due : nullptr);
+    if (deco::launch_multi_aggregate(L->server_dev, L->big_tile_layer, L->big_tiles, L->n, slot_write,
+                                     L->any_dense, L->any_sparse, s) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    for (uint32_t slot_read : due)
+        if (deco::launch_multi_apply(L->server_dev, layers, L->n, L->apply_ctas, slot_read, neg_scale, s) !=
+            cudaSuccess)
+            return DECO_ERR_CUDA;
+    L->layers[L->big[0]]->launches += 1 + due.size();
+    return DECO_OK;
 }
 
 }  // namespace
@@ -127,6 +331,11 @@ extern "C" deco_status deco_layered_init(deco_layered **out, uint64_t d, uint32_
         }
         L->layers.push_back(c);
     }
+    if (build_small_batch(L) != cudaSuccess) {
+        cudaGetLastError();
+        release(L);
+        return DECO_ERR_OOM;
+    }
     *out = L;
     return DECO_OK;
 }
@@ -150,10 +359,24 @@ extern "C" deco_status deco_layered_step(deco_layered *L, const void *grads, voi
     for (cudaStream_t q : L->streams)
         if (cudaStreamWaitEvent(q, L->ev_fork, 0) != cudaSuccess) return DECO_ERR_CUDA;
     const size_t esz = L->grad_dtype == DECO_BF16 ? 2 : 4;
-    deco_status st = DECO_OK;
-    for (size_t l = 0; l < L->layers.size() && st == DECO_OK; ++l)
-        st = deco_step(L->layers[l], static_cast<const char *>(grads) + L->offsets[l] * esz,
-                       L->streams[l % LAYER_STREAMS]);
+    // the batch of short layers first, then the others
+    deco_status st = step_small_batch(L, grads, L->streams[0]);
+    if (L->plan && st == DECO_OK) {
+        // worker side of all of them in one sequence of launches, then their server side
+        for (uint32_t l : L->big)
+            if (L->layers[l]->phase != 0) return DECO_ERR_STATE;
+        const deco_ctx *first = L->layers[L->big[0]];
+        const float alpha = first->lr_at_server ? 1.0f : first->lr;
+        cudaStream_t cs = L->streams[1 % LAYER_STREAMS];
+        if (deco::multi_compress(L->plan, grads, alpha, cs) != cudaSuccess) return DECO_ERR_CUDA;
+        st = step_big_server(L, cs);
+    } else {
+        for (size_t q = 0; q < L->big.size() && st == DECO_OK; ++q) {
+            const uint32_t l = L->big[q];
+            st = deco_step(L->layers[l], static_cast<const char *>(grads) + L->offsets[l] * esz,
+                           L->streams[(q + 1) % LAYER_STREAMS]);
+        }
+    }
     for (int q = 0; q < LAYER_STREAMS; ++q)
         if (cudaEventRecord(L->ev_done[q], L->streams[q]) != cudaSuccess ||
             cudaStreamWaitEvent(s, L->ev_done[q], 0) != cudaSuccess)
@@ -182,6 +405,9 @@ extern "C" deco_status deco_layered_set_policy(deco_layered *L, double delta, ui
         const deco_status st = deco_set_policy(c, delta, tau);
         if (st != DECO_OK) return st;
     }
+    L->small_dirty = true;
+    deco::multi_plan_mark_dirty(L->plan);
+    L->server_dirty = true;
     return DECO_OK;
 }
 

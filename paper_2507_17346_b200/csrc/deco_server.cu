@@ -208,6 +208,105 @@ __device__ __forceinline__ uint32_t warp_merge(bool valid, uint32_t idx, float v
 // whole CTA afterwards (dense_tile).
 constexpr int SPARSE_WINDOWS = 4;
 
+// One tile by one warp.  Returns true (to every lane) if the tile does not fit and has to be
+// done by the whole CTA with the dense accumulator.
+__device__ __forceinline__ bool sparse_tile_warp(const deco_pair *__restrict__ msg, uint64_t k_cap,
+                                                 const uint32_t *__restrict__ tile_start, uint32_t ntiles,
+                                                 uint32_t n, deco_pair *__restrict__ slot, uint64_t positions,
+                                                 uint32_t *__restrict__ status, uint32_t tile)
+{
+    const int lane = threadIdx.x & 31;
+    uint32_t a = 0, b = 0;
+    if (static_cast<uint32_t>(lane) < n) {
+        a = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile];
+        b = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile + 1];
+    }
+    const uint32_t len = b - a;
+    uint32_t cap = len, longest = len;
+    uint64_t out_off = a;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        cap += __shfl_xor_sync(FULL, cap, o);
+        longest = max(longest, __shfl_xor_sync(FULL, longest, o));
+        out_off += __shfl_xor_sync(FULL, out_off, o);
+    }
+    const uint32_t first = tile * static_cast<uint32_t>(TILE);
+    if (cap == 0) return false;
+    if (out_off + cap > positions) {
+        if (lane == 0) latch(status, DECO_ERR_DEVICE_CHECK, 0x400u, tile);
+        return false;
+    }
+    if (cap > 32u * SPARSE_WINDOWS || longest > 32) return true;
+    // lane i: how many of worker i's entries lie below the end of each window
+    // (every lane looks at one entry of each worker in turn: ranges are at most 32 long)
+    uint32_t below[SPARSE_WINDOWS + 1];
+    below[0] = 0;
+#pragma unroll
+    for (int q = 1; q <= SPARSE_WINDOWS; ++q) below[q] = len;
+    if (cap > 32) {
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint32_t ai = __shfl_sync(FULL, a, i), li = __shfl_sync(FULL, len, i);
+            uint32_t loc = DECO_NO_INDEX;
+            if (static_cast<uint32_t>(lane) < li)
+                loc = msg[static_cast<size_t>(i) * k_cap + ai + lane].idx - first;
+#pragma unroll
+            for (int q = 1; q < SPARSE_WINDOWS; ++q) {
+                const uint32_t cnt = __popc(__ballot_sync(FULL, loc < q * (TILE / SPARSE_WINDOWS)));
+                if (static_cast<uint32_t>(lane) == i) below[q] = cnt;
+            }
+        }
+    }
+    // per window: entries of the workers before lane's own, and in all
+    uint32_t before[SPARSE_WINDOWS], total[SPARSE_WINDOWS];
+    bool fits = true;
+#pragma unroll
+    for (int q = 0; q < SPARSE_WINDOWS; ++q) {
+        const uint32_t mine = below[q + 1] - below[q];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(FULL, incl, o);
+            if (lane >= o) incl += t;
+        }
+        before[q] = incl - mine;
+        total[q] = __shfl_sync(FULL, incl, 31);
+        fits = fits && total[q] <= 32;
+    }
+    if (!fits) return true;
+    deco_pair *out = slot + out_off;
+    uint32_t uniq = 0;
+#pragma unroll
+    for (int q = 0; q < SPARSE_WINDOWS; ++q) {
+        if (total[q] == 0) continue;
+        const uint32_t part_a = a + below[q], part_len = below[q + 1] - below[q];
+        deco_pair pr;
+        pr.idx = DECO_NO_INDEX;
+        pr.val = 0.0f;
+        bool valid = false;
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint32_t pb = __shfl_sync(FULL, before[q], i);
+            const uint32_t pl = __shfl_sync(FULL, part_len, i);
+            const uint32_t pa = __shfl_sync(FULL, part_a, i);
+            if (static_cast<uint32_t>(lane) >= pb && static_cast<uint32_t>(lane) < pb + pl) {
+                pr = msg[static_cast<size_t>(i) * k_cap + pa + (lane - pb)];
+                valid = true;
+            }
+        }
+        if (valid && pr.idx - first >= static_cast<uint32_t>(TILE)) {
+            latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pr.idx);
+            valid = false;
+        }
+        uniq += warp_merge(valid, pr.idx, pr.val, out + uniq);
+    }
+    for (uint32_t q = uniq + lane; q < cap; q += 32) {
+        deco_pair pr;
+        pr.idx = DECO_NO_INDEX;
+        pr.val = 0.0f;
+        out[q] = pr;
+    }
+    return false;
+}
+
 __global__ void __launch_bounds__(BLOCK)
 aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
                         const uint32_t *__restrict__ tile_start, uint32_t ntiles, uint32_t n,
@@ -222,100 +321,9 @@ aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     __syncthreads();
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t tile = blockIdx.x * WARPS + w;
-    if (tile < ntiles) {
-        uint32_t a = 0, b = 0;
-        if (static_cast<uint32_t>(lane) < n) {
-            a = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile];
-            b = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile + 1];
-        }
-        const uint32_t len = b - a;
-        uint32_t cap = len, longest = len;
-        uint64_t out_off = a;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            cap += __shfl_xor_sync(FULL, cap, o);
-            longest = max(longest, __shfl_xor_sync(FULL, longest, o));
-            out_off += __shfl_xor_sync(FULL, out_off, o);
-        }
-        const uint32_t first = tile * static_cast<uint32_t>(TILE);
-        if (cap == 0) {
-        } else if (out_off + cap > positions) {
-            if (lane == 0) latch(status, DECO_ERR_DEVICE_CHECK, 0x400u, tile);
-        } else if (cap > 32u * SPARSE_WINDOWS || longest > 32) {
-            if (lane == 0) atomicOr(&s_heavy, 1u << w);
-        } else {
-            // lane i: how many of worker i's entries lie below the end of each window
-            // (every lane looks at one entry of each worker in turn: ranges are at most 32 long)
-            uint32_t below[SPARSE_WINDOWS + 1];
-            below[0] = 0;
-#pragma unroll
-            for (int q = 1; q <= SPARSE_WINDOWS; ++q) below[q] = len;
-            if (cap > 32) {
-                for (uint32_t i = 0; i < n; ++i) {
-                    const uint32_t ai = __shfl_sync(FULL, a, i), li = __shfl_sync(FULL, len, i);
-                    uint32_t loc = DECO_NO_INDEX;
-                    if (static_cast<uint32_t>(lane) < li)
-                        loc = msg[static_cast<size_t>(i) * k_cap + ai + lane].idx - first;
-#pragma unroll
-                    for (int q = 1; q < SPARSE_WINDOWS; ++q) {
-                        const uint32_t cnt = __popc(__ballot_sync(FULL, loc < q * (TILE / SPARSE_WINDOWS)));
-                        if (static_cast<uint32_t>(lane) == i) below[q] = cnt;
-                    }
-                }
-            }
-            // per window: entries of the workers before lane's own, and in all
-            uint32_t before[SPARSE_WINDOWS], total[SPARSE_WINDOWS];
-            bool fits = true;
-#pragma unroll
-            for (int q = 0; q < SPARSE_WINDOWS; ++q) {
-                const uint32_t mine = below[q + 1] - below[q];
-                uint32_t incl = mine;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t t = __shfl_up_sync(FULL, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                before[q] = incl - mine;
-                total[q] = __shfl_sync(FULL, incl, 31);
-                fits = fits && total[q] <= 32;
-            }
-            if (!fits) {
-                if (lane == 0) atomicOr(&s_heavy, 1u << w);
-            } else {
-                deco_pair *out = slot + out_off;
-                uint32_t uniq = 0;
-#pragma unroll
-                for (int q = 0; q < SPARSE_WINDOWS; ++q) {
-                    if (total[q] == 0) continue;
-                    const uint32_t part_a = a + below[q], part_len = below[q + 1] - below[q];
-                    deco_pair pr;
-                    pr.idx = DECO_NO_INDEX;
-                    pr.val = 0.0f;
-                    bool valid = false;
-                    for (uint32_t i = 0; i < n; ++i) {
-                        const uint32_t pb = __shfl_sync(FULL, before[q], i);
-                        const uint32_t pl = __shfl_sync(FULL, part_len, i);
-                        const uint32_t pa = __shfl_sync(FULL, part_a, i);
-                        if (static_cast<uint32_t>(lane) >= pb && static_cast<uint32_t>(lane) < pb + pl) {
-                            pr = msg[static_cast<size_t>(i) * k_cap + pa + (lane - pb)];
-                            valid = true;
-                        }
-                    }
-                    if (valid && pr.idx - first >= static_cast<uint32_t>(TILE)) {
-                        latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pr.idx);
-                        valid = false;
-                    }
-                    uniq += warp_merge(valid, pr.idx, pr.val, out + uniq);
-                }
-                for (uint32_t q = uniq + lane; q < cap; q += 32) {
-                    deco_pair pr;
-                    pr.idx = DECO_NO_INDEX;
-                    pr.val = 0.0f;
-                    out[q] = pr;
-                }
-            }
-        }
-    }
+    if (tile < ntiles && sparse_tile_warp(msg, k_cap, tile_start, ntiles, n, slot, positions, status, tile) &&
+        lane == 0)
+        atomicOr(&s_heavy, 1u << w);
     __syncthreads();
     uint32_t heavy = s_heavy;
     if (heavy == 0) return;
@@ -325,6 +333,90 @@ aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     for (; heavy; heavy &= heavy - 1)
         dense_tile(msg, k_cap, tile_start, ntiles, n, slot, positions, status,
                    blockIdx.x * WARPS + __ffs(heavy) - 1, acc, mask, s_w);
+}
+
+// ---- the server side of many contexts (layers of the per-layer variant) in one launch each.
+// Tiles of all layers are numbered in a row; tile_layer gives the layer of each.
+__global__ void __launch_bounds__(BLOCK)
+aggregate_multi_kernel(const ServerLayer *__restrict__ table, const uint32_t *__restrict__ tile_layer,
+                       uint32_t total_tiles, uint32_t n, uint32_t slot_write)
+{
+    __shared__ float acc[TILE];
+    __shared__ uint32_t mask[TILE / 32];
+    __shared__ uint32_t s_w[WARPS];
+    for (int q = threadIdx.x; q < TILE; q += BLOCK) acc[q] = 0.0f;
+    mask[threadIdx.x] = 0;
+    __syncthreads();
+    for (uint32_t g = blockIdx.x; g < total_tiles; g += gridDim.x) {
+        const ServerLayer &L = table[tile_layer[g]];
+        if (!L.dense) continue;
+        const uint32_t tile = g - L.first_tile;
+        const uint64_t positions = static_cast<uint64_t>(n) * L.k;
+        if (tile == 0 && threadIdx.x == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
+        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles, n, L.slots + slot_write * (n * L.k_cap), positions,
+                   L.status, tile, acc, mask, s_w);
+    }
+}
+
+__global__ void __launch_bounds__(BLOCK)
+aggregate_sparse_multi_kernel(const ServerLayer *__restrict__ table, const uint32_t *__restrict__ tile_layer,
+                              uint32_t total_tiles, uint32_t n, uint32_t slot_write)
+{
+    __shared__ float acc[TILE];
+    __shared__ uint32_t mask[TILE / 32];
+    __shared__ uint32_t s_w[WARPS];
+    __shared__ uint32_t s_heavy;
+    if (threadIdx.x == 0) s_heavy = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t g = blockIdx.x * WARPS + w;
+    if (g < total_tiles) {
+        const ServerLayer &L = table[tile_layer[g]];
+        if (!L.dense) {
+            const uint32_t tile = g - L.first_tile;
+            const uint64_t positions = static_cast<uint64_t>(n) * L.k;
+            if (tile == 0 && lane == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
+            if (sparse_tile_warp(L.msg, L.k_cap, L.tile_start, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
+                                 positions, L.status, tile) && lane == 0)
+                atomicOr(&s_heavy, 1u << w);
+        }
+    }
+    __syncthreads();
+    uint32_t heavy = s_heavy;
+    if (heavy == 0) return;
+    for (int q = threadIdx.x; q < TILE; q += BLOCK) acc[q] = 0.0f;
+    mask[threadIdx.x] = 0;
+    __syncthreads();
+    for (; heavy; heavy &= heavy - 1) {
+        const uint32_t gh = blockIdx.x * WARPS + __ffs(heavy) - 1;
+        const ServerLayer &L = table[tile_layer[gh]];
+        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
+                   static_cast<uint64_t>(n) * L.k, L.status, gh - L.first_tile, acc, mask, s_w);
+    }
+}
+
+// Row y of the grid applies cache slot `slot_read` of layer y to the layer's parameters.
+__global__ void __launch_bounds__(256)
+apply_multi_kernel(const ServerLayer *__restrict__ table, uint32_t n, uint32_t slot_read, float neg_scale)
+{
+    const ServerLayer &L = table[blockIdx.y];
+    const deco_pair *slot = L.slots + slot_read * (static_cast<uint64_t>(n) * L.k_cap);
+    const uint64_t positions = L.slot_pos[slot_read];
+    if (positions > static_cast<uint64_t>(n) * L.k_cap) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) latch(L.status, DECO_ERR_DEVICE_CHECK, 0x520u, slot_read);
+        return;
+    }
+    float *params = L.params;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    for (uint64_t p = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < positions; p += stride) {
+        const deco_pair pr = slot[p];
+        if (pr.idx == DECO_NO_INDEX) continue;
+        if (pr.idx >= L.d) {
+            latch(L.status, DECO_ERR_DEVICE_CHECK, 0x500u, pr.idx);
+            continue;
+        }
+        params[pr.idx] = __fmaf_rn(neg_scale, pr.val, params[pr.idx]);
+    }
 }
 
 __global__ void __launch_bounds__(256)
@@ -344,7 +436,85 @@ apply_kernel(const deco_pair *__restrict__ slot, uint64_t positions, float neg_s
     }
 }
 
+// Short layers of the per-layer variant, one CTA per layer: the n messages are merged into the
+// layer's cache slot (the layer is one tile), then the listed slots are applied to the layer's
+// slice of the parameters, oldest first, one fused multiply-add per stored entry.
+__global__ void __launch_bounds__(BLOCK)
+small_server_kernel(const SmallLayer *__restrict__ table, uint32_t n, uint32_t aggregate,
+                    uint32_t slot_write, SmallDue due, float neg_scale)
+{
+    __shared__ float acc[TILE];
+    __shared__ uint32_t mask[TILE / 32];
+    __shared__ uint32_t s_w[WARPS];
+    const SmallLayer L = table[blockIdx.x];
+    const uint64_t slot_len = static_cast<uint64_t>(n) * L.k_cap;
+    if (aggregate) {
+        for (int q = threadIdx.x; q < TILE; q += BLOCK) acc[q] = 0.0f;
+        mask[threadIdx.x] = 0;
+        __syncthreads();
+        const uint64_t positions = static_cast<uint64_t>(n) * L.k;
+        dense_tile(L.msg, L.k_cap, L.tile_start, 1, n, L.slots + slot_write * slot_len, positions,
+                   L.status, 0, acc, mask, s_w);
+        if (threadIdx.x == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
+        __syncthreads();
+    }
+    for (uint32_t q = 0; q < due.count; ++q) {
+        const deco_pair *slot = L.slots + due.slot[q] * slot_len;
+        const uint32_t positions = L.slot_pos[due.slot[q]];
+        if (positions > slot_len) {
+            if (threadIdx.x == 0) latch(L.status, DECO_ERR_DEVICE_CHECK, 0x520u, positions);
+            return;
+        }
+        for (uint32_t p = threadIdx.x; p < positions; p += BLOCK) {
+            const deco_pair pr = slot[p];
+            if (pr.idx == DECO_NO_INDEX) continue;
+            if (pr.idx >= L.d) {
+                latch(L.status, DECO_ERR_DEVICE_CHECK, 0x500u, pr.idx);
+                continue;
+            }
+            L.params[pr.idx] = __fmaf_rn(neg_scale, pr.val, L.params[pr.idx]);
+        }
+        __syncthreads();          // an entry may be held by several slots: one pass after the other
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_small_server(const SmallLayer *table, uint32_t layers, uint32_t n, bool aggregate,
+                                uint32_t slot_write, const SmallDue &due, float neg_scale, cudaStream_t s)
+{
+    if (layers == 0) return cudaSuccess;
+    small_server_kernel<<<layers, BLOCK, 0, s>>>(table, n, aggregate ? 1u : 0u, slot_write, due, neg_scale);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_multi_aggregate(const ServerLayer *table, const uint32_t *tile_layer, uint32_t total_tiles,
+                                   uint32_t n, uint32_t slot_write, bool any_dense, bool any_sparse,
+                                   cudaStream_t s)
+{
+    if (any_sparse)
+        aggregate_sparse_multi_kernel<<<(total_tiles + WARPS - 1) / WARPS, BLOCK, 0, s>>>(table, tile_layer,
+                                                                                       total_tiles, n, slot_write);
+    if (any_dense) {
+        const uint32_t blocks = total_tiles < 148u * 6 ? total_tiles : 148u * 6;
+        aggregate_multi_kernel<<<blocks, BLOCK, 0, s>>>(table, tile_layer, total_tiles, n, slot_write);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_multi_apply(const ServerLayer *table, uint32_t layers, uint32_t n, uint32_t ctas_per_layer,
+                               uint32_t slot_read, float neg_scale, cudaStream_t s)
+{
+    apply_multi_kernel<<<dim3(ctas_per_layer, layers), 256, 0, s>>>(table, n, slot_read, neg_scale);
+    return cudaGetLastError();
+}
+
+// the rule of launch_aggregate: a warp per tile up to 80 entries per tile on average
+bool aggregate_prefers_dense(const deco_ctx *c)
+{
+    const uint64_t positions = static_cast<uint64_t>(c->n_total) * c->k;
+    return !(c->n_total <= 32 && positions <= 80ull * c->ntiles);
+}
 
 cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s)
 {

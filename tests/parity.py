@@ -143,10 +143,12 @@ def run_layered_parity(layer_offsets, n, delta, tau, lr, grad_fn, steps, grad_dt
         info = B.deco_layered_info(ctx)
         assert info["n_layers"] == len(layer_offsets) - 1 and info["k_total"] == orc.k
         layers = [B.deco_layered_layer(ctx, l) for l in range(info["n_layers"])]
+        tau_now = tau
         for t in range(steps):
             if policy_plan and t in policy_plan:
                 B.deco_layered_set_policy(ctx, *policy_plan[t])
                 orc.set_policy(*policy_plan[t])
+                tau_now = policy_plan[t][1]
                 assert B.deco_layered_info(ctx)["k_total"] == orc.k
             g = grad_fn(t)
             ref = orc.step(W.to_numpy_bits(g))
@@ -164,19 +166,21 @@ def run_layered_parity(layer_offsets, n, delta, tau, lr, grad_fn, steps, grad_dt
                 e = read_e(sub, n, ln, device)
                 assert np.array_equal(bits(e), bits(orc.e[:, off:off + ln])), \
                     "step %d layer at %d: residual" % (t, off)
-                aidx, aval = read_aggregate(sub, t, device)
-                agg_idx.append(aidx.astype(np.uint64) + off)
-                agg_val.append(aval)
+                if tau_now > 0:        # with tau = 0 the aggregate is consumed inside the step
+                    aidx, aval = read_aggregate(sub, t, device)
+                    agg_idx.append(aidx.astype(np.uint64) + off)
+                    agg_val.append(aval)
             for i, (sel, vals) in enumerate(ref["msgs"]):
                 assert np.array_equal(np.concatenate(idx_parts[i]), sel.astype(np.uint64)), \
                     "step %d worker %d: index set" % (t, i)
                 assert np.array_equal(bits(np.concatenate(val_parts[i])), bits(vals)), \
                     "step %d worker %d: message values" % (t, i)
-            touched = np.unique(np.concatenate([s for s, _ in ref["msgs"]]))
-            assert np.array_equal(np.concatenate(agg_idx), touched.astype(np.uint64)), \
-                "step %d: aggregate index set" % t
-            assert np.array_equal(bits(np.concatenate(agg_val)), bits(ref["S"][touched])), \
-                "step %d: aggregate" % t
+            if tau_now > 0:
+                touched = np.unique(np.concatenate([s for s, _ in ref["msgs"]]))
+                assert np.array_equal(np.concatenate(agg_idx), touched.astype(np.uint64)), \
+                    "step %d: aggregate index set" % t
+                assert np.array_equal(bits(np.concatenate(agg_val)), bits(ref["S"][touched])), \
+                    "step %d: aggregate" % t
             x = B.view_f32(info["params"], (d,), device).cpu().numpy()
             assert np.array_equal(bits(x), bits(orc.x)), "step %d: parameters" % t
         for sub, _, _ in layers:

@@ -237,6 +237,25 @@ def test_per_layer_topk_variant():
         run_layered_parity(odd, 4, 0.02, 1, 0.1, grads, steps=4, grad_dtype=name)
 
 
+@pytest.mark.parametrize("kind", ["normal", "coarse", "all_equal", "signed_zero"])
+def test_per_layer_topk_short_layers_batch(kind):
+    """Layers of at most 8192 entries are stepped as one batch (a CTA per layer and worker, a
+    CTA per layer on the server side): lengths 1, 31, 8191, 8192 next to one of 8193 that takes
+    the ordinary route, heavy ties (few distinct magnitudes, all equal, signed zeros), delta
+    up to 1, and a staleness that goes 3 -> 0 -> 2 so that one update drains several cached
+    aggregates and another applies its own iteration's."""
+    lengths = [1, 31, 8191, 8192, 8193, 2, 4097, 640]
+    offsets = [0]
+    for ln in lengths:
+        offsets.append(offsets[-1] + ln)
+    n = 5
+    for dtype, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        run_layered_parity(offsets, n, 0.05, 3, 0.1,
+                           lambda t: _values(kind, n, offsets[-1], t, dtype), steps=9,
+                           grad_dtype=name, policy_plan={4: (1.0, 0), 6: (0.3, 2)},
+                           tau_max=3, delta_max=1.0)
+
+
 @pytest.mark.parametrize("compressor", ["topk", "randk"])
 def test_worker_sharded_contexts_equal_the_single_job(compressor):
     """Five workers split 2 + 3 over two contexts on one GPU.  Each compresses its own workers;
