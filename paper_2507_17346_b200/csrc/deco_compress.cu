@@ -463,7 +463,7 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         // how far the sampled rank sits above k/d decides how far above the bound the
         // threshold may lie (in value: that ratio to the power 1/tail-index)
         const double rho = static_cast<double>(R) / (mean > 1e-9 ? mean : 1e-9);
-        rel_shift = rho <= 1.5 ? 10u : (rho <= 1.75 ? 11u : 12u);
+        rel_shift = rho <= 1.7 ? 10u : 12u;
         if (p.rk.on) rel_shift = 10u;          // uniform 23-bit priorities: 4095 << 10 is half the range
     }
     uint32_t *gh = p.sample_hist + i * SAMPLE_HIST_BINS;
@@ -1718,12 +1718,14 @@ struct AccLayer {
     SelectState *sel;
     uint32_t *tile_off, *tile_cnt, *tile_rej, *tile_eq;
     uint64_t e_stride, stage_cap, d, g_off;
-    uint32_t ntiles, first_tile;     // first_tile: relative to the table's first layer
-    uint32_t rows_aligned, pad;
+    uint32_t ntiles, rows_aligned;
 };
 struct AccTable {
-    AccLayer L[ACC_LAYERS_MAX];
+    // first tile of every layer, relative to the table's first layer: one kilobyte that the
+    // bisection of every CTA walks, so it stays in the constant cache
+    uint32_t first_tile[ACC_LAYERS_MAX];
     uint32_t count, pad;
+    AccLayer L[ACC_LAYERS_MAX];
 };
 static_assert(sizeof(AccTable) < 32000, "kernel parameters are limited to 32764 bytes");
 
@@ -1735,16 +1737,17 @@ ef_accumulate_multi_kernel(const __grid_constant__ AccTable tab, const void *__r
     uint32_t lo = 0, hi = tab.count;                         // the layer lies in [lo, hi)
     while (hi - lo > 1) {
         const uint32_t mid = (lo + hi) >> 1;
-        if (tab.L[mid].first_tile <= blockIdx.x) lo = mid;
+        if (tab.first_tile[mid] <= blockIdx.x) lo = mid;
         else hi = mid;
     }
     const AccLayer &m = tab.L[lo];
+    const uint32_t tile = blockIdx.x - tab.first_tile[lo];
     if ((m.rows_aligned != 0) != ALIGNED) return;
     const char *g = static_cast<const char *>(grads) + m.g_off * (GT ? 2 : 4);
     RandParams rk;
     rk.on = 0;
     rk.seed_lo = rk.seed_hi = rk.step_lo = rk.step_hi = rk.worker_base = 0;
-    ef_accumulate_body<GT, ALIGNED, true, false>(blockIdx.x - m.first_tile, blockIdx.y, true, m.e, m.e_stride, g,
+    ef_accumulate_body<GT, ALIGNED, true, false>(tile, blockIdx.y, true, m.e, m.e_stride, g,
                                                  m.d, g_stride, alpha, rk, m.sel, m.stage, m.stage_cap,
                                                  m.tile_off, m.tile_cnt, m.tile_rej, m.tile_eq, m.ntiles);
 }
@@ -2101,9 +2104,8 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
         a.d = m.p.d;
         a.g_off = m.g_off;
         a.ntiles = m.p.ntiles;
-        a.first_tile = grp.tiles;
+        grp.tab.first_tile[l % ACC_LAYERS_MAX] = grp.tiles;
         a.rows_aligned = m.rows_aligned;
-        a.pad = 0;
         grp.tiles += m.p.ntiles;
         grp.tab.count = l % ACC_LAYERS_MAX + 1;
         grp.tab.pad = 0;
