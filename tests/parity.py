@@ -130,14 +130,15 @@ def run_parity(d, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32", select_mo
 
 
 def run_layered_parity(layer_offsets, n, delta, tau, lr, grad_fn, steps, grad_dtype="f32",
-                       policy_plan=None, tau_max=0, delta_max=0.0, device=0):
+                       policy_plan=None, tau_max=0, delta_max=0.0, device=0, select_mode=None):
     """Per-layer Top-k: the layered context (one library context per layer, stepped together)
     against the oracle's per-layer variant, which keeps one flat state and only selects per
     range.  Messages, residuals, aggregates and parameters must agree bit for bit."""
     d = int(layer_offsets[-1])
     ctx = B.deco_layered_init(d, n, layer_offsets, delta, tau, lr,
                               grad_dtype=B.DECO_F32 if grad_dtype == "f32" else B.DECO_BF16,
-                              tau_max=tau_max, delta_max=delta_max, device=device)
+                              tau_max=tau_max, delta_max=delta_max, device=device,
+                              select_mode=B.DECO_SELECT_AUTO if select_mode is None else select_mode)
     try:
         orc = O.DDEFSGD(d, n, delta, tau, lr, layer_offsets=layer_offsets)
         info = B.deco_layered_info(ctx)

@@ -235,6 +235,9 @@ def test_per_layer_topk_variant():
             x[:, 4:1001] *= 40.0
             return x.to(dtype).contiguous()
         run_layered_parity(odd, 4, 0.02, 1, 0.1, grads, steps=4, grad_dtype=name)
+    # the multi-pass selection keeps the route that steps every layer's context on its own
+    run_layered_parity(offsets, 3, 0.01, 1, 0.1, lambda t: W.gradients(wl, t, "cuda")[:3].contiguous(),
+                       steps=3, select_mode=B.DECO_SELECT_EXACT_PASSES)
 
 
 @pytest.mark.parametrize("kind", ["normal", "coarse", "all_equal", "signed_zero"])
