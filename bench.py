@@ -149,14 +149,15 @@ def grad_bytes(wl):
     return wl.n * wl.d * (4 if wl.grad_dtype == "f32" else 2)
 
 
-# DRAM read + write bytes of one ef_accumulate_kernel launch from the ncu capture summarised in
-# profiles/ef_accumulate_kernel_resnet18.md (taken on this kernel version); other workloads
-# were not captured.
+# DRAM read + write bytes of one ef_accumulate_kernel launch from the ncu captures summarised in
+# profiles/ef_accumulate_kernel_dram_traffic.md (taken on this kernel version).  resnet18 was
+# captured at full size; the others at reduced size (--scale) and are scaled by the entry count:
+# the kernel streams every entry once, so its traffic grows in proportion.
 NCU_TRAFFIC_BYTES = {
-    "resnet18": 1076.4e6,        # captured at full size
-    # captured at --scale 0.5 (163.9 M entries, 1589.2 MB) and scaled by the entry count:
-    # the kernel streams every entry once, so its traffic grows in proportion
-    "gpt2_small": 1589.2e6 * (995518464 / 163946496),
+    "resnet18": 1075.3e6,
+    "gpt2_small": 1585.7e6 * (995518464 / 163946496),
+    "decoder_1b": 2110.6e6 * (4400193536 / 216158400),
+    "sweep_100m": 1155.0e6 * (400000000 / 100000000),
 }
 
 
