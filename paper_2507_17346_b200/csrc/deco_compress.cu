@@ -1222,31 +1222,32 @@ __device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, 
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t T = p.sel[i].threshold;
     if (blockIdx.x < dir_ctas) {
-        const uint32_t chunk = blockIdx.x * WARPS + w;
-        if (chunk >= p.nchunks) return;
-        const TileInfo t = chunk_header<true>(p, i, chunk);
-        const uint32_t tile = chunk * CHUNK_TILES + lane;
-        if (t.cnt == 0 || t.cnt > EMIT_LANE_MAX) return;
-        const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
-        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
-        deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
-        float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
-        uint32_t written = 0, ties_seen = 0;
-        for (uint32_t q = 0; q < t.cnt; ++q) {
-            const deco_pair pr = src[q];
-            const uint32_t key = key_of(p, i, pr);
-            const bool eq = key == T;
-            const bool pick = key > T || (eq && ties_seen < t.take);
-            ties_seen += eq ? 1u : 0u;
-            if (pick) {
-                const uint32_t pos = t.start + written++;
-                if (pos < p.k && pr.idx < p.d) out[pos] = pr;
-                else latch(p.status, DECO_ERR_DEVICE_CHECK, 0x312u, tile);
-            } else if (eq && pr.idx < p.d) {
-                erow[pr.idx] = pr.val;                       // tie not taken: undo the guess
+        // the directory CTAs stride over the chunks (one trip when there is a warp per chunk)
+        for (uint32_t chunk = blockIdx.x * WARPS + w; chunk < p.nchunks; chunk += dir_ctas * WARPS) {
+            const TileInfo t = chunk_header<true>(p, i, chunk);
+            const uint32_t tile = chunk * CHUNK_TILES + lane;
+            if (t.cnt == 0 || t.cnt > EMIT_LANE_MAX) continue;
+            const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
+            const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
+            deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
+            float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+            uint32_t written = 0, ties_seen = 0;
+            for (uint32_t q = 0; q < t.cnt; ++q) {
+                const deco_pair pr = src[q];
+                const uint32_t key = key_of(p, i, pr);
+                const bool eq = key == T;
+                const bool pick = key > T || (eq && ties_seen < t.take);
+                ties_seen += eq ? 1u : 0u;
+                if (pick) {
+                    const uint32_t pos = t.start + written++;
+                    if (pos < p.k && pr.idx < p.d) out[pos] = pr;
+                    else latch(p.status, DECO_ERR_DEVICE_CHECK, 0x312u, tile);
+                } else if (eq && pr.idx < p.d) {
+                    erow[pr.idx] = pr.val;                       // tie not taken: undo the guess
+                }
             }
+            if (written != t.sel) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x313u, tile);
         }
-        if (written != t.sel) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x313u, tile);
         return;
     }
     const uint32_t n_items = min(p.done[i * DONE_SLOTS + 5], static_cast<uint32_t>(p.work_cap));
@@ -2069,7 +2070,7 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
 {
     const uint32_t L = static_cast<uint32_t>(mp->layers.size());
     const uint64_t esz = mp->grad_dtype == DECO_BF16 ? 2 : 4;
-    uint64_t begin_max = 1, stage_max = 1, chunk_max = 0, dir_max = 1, item_max = 1;
+    uint64_t begin_max = 1, stage_max = 1, chunk_max = 0, dir_max = 1, item_max = 1, dir_sum = 0;
     for (uint32_t l = 0; l < L; ++l) {
         const deco_ctx *c = mp->layers[l];
         MultiLayer &m = mp->host[l];
@@ -2083,6 +2084,7 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
         stage_max = std::max<uint64_t>(stage_max, (2 * c->k + 65536 + BLOCK * 4 - 1) / (BLOCK * 4));
         if (!m.walk_here) chunk_max = std::max<uint64_t>(chunk_max, (c->nchunks + WARPS - 1) / WARPS);
         dir_max = std::max<uint64_t>(dir_max, (c->nchunks + WARPS - 1) / WARPS);
+        dir_sum += (c->nchunks + WARPS - 1) / WARPS;
         const uint64_t staged = 13 * c->k / 10, many = staged / (EMIT_LANE_MAX + 1);
         const uint64_t est_items = staged / EMIT_SLICE + (many < c->ntiles ? many : c->ntiles);
         item_max = std::max<uint64_t>(item_max, (est_items + WARPS - 1) / WARPS + 1);
@@ -2117,7 +2119,9 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
     mp->begin_ctas = static_cast<uint32_t>(begin_max);
     mp->stage_ctas = static_cast<uint32_t>(std::min(stage_max, cap));
     mp->chunk_ctas = static_cast<uint32_t>(chunk_max);
-    mp->dir_ctas = static_cast<uint32_t>(dir_max);
+    // directory CTAs stride over the chunks: the longest layer may take four trips, so that the
+    // many short layers do not each bring a grid row full of idle CTAs
+    mp->dir_ctas = static_cast<uint32_t>(std::max<uint64_t>({1, (dir_max + 3) / 4, (dir_sum + L - 1) / L}));
     mp->item_ctas = static_cast<uint32_t>(std::min(item_max, std::max<uint64_t>(1, 2 * cap)));
     (void)grads;
     // the host table is pageable: the copy has left it when the call returns

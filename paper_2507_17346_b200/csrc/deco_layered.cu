@@ -239,7 +239,7 @@ deco_status step_big_server(deco_layered *L, cudaStream_t s)
         if (cudaMemcpyAsync(L->server_dev, L->server_host.data(), sizeof(deco::ServerLayer) * layers,
                             cudaMemcpyHostToDevice, s) != cudaSuccess)
             return DECO_ERR_CUDA;
-        const uint64_t want = (most + 255) / 256, cap = std::max<uint64_t>(1, 148ull * 16 / layers);
+        const uint64_t want = (most + 1023) / 1024, cap = std::max<uint64_t>(1, 148ull * 64 / layers);
         L->apply_ctas = static_cast<uint32_t>(std::min(want, cap));
         L->server_dirty = false;
     }

@@ -408,14 +408,32 @@ apply_multi_kernel(const ServerLayer *__restrict__ table, uint32_t n, uint32_t s
     }
     float *params = L.params;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
-    for (uint64_t p = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < positions; p += stride) {
-        const deco_pair pr = slot[p];
-        if (pr.idx == DECO_NO_INDEX) continue;
-        if (pr.idx >= L.d) {
-            latch(L.status, DECO_ERR_DEVICE_CHECK, 0x500u, pr.idx);
-            continue;
+    // four independent entries per thread and trip (entries of a slot are distinct)
+    for (uint64_t p0 = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p0 < positions;
+         p0 += 4 * stride) {
+        deco_pair pr[4];
+        float x[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint64_t p = p0 + r * stride;
+            pr[r].idx = DECO_NO_INDEX;
+            pr[r].val = 0.0f;
+            if (p < positions) pr[r] = slot[p];
         }
-        params[pr.idx] = __fmaf_rn(neg_scale, pr.val, params[pr.idx]);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            x[r] = 0.0f;
+            if (pr[r].idx == DECO_NO_INDEX) continue;
+            if (pr[r].idx >= L.d) {
+                latch(L.status, DECO_ERR_DEVICE_CHECK, 0x500u, pr[r].idx);
+                pr[r].idx = DECO_NO_INDEX;
+                continue;
+            }
+            x[r] = params[pr[r].idx];
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+            if (pr[r].idx != DECO_NO_INDEX) params[pr[r].idx] = __fmaf_rn(neg_scale, pr[r].val, x[r]);
     }
 }
 
