@@ -36,7 +36,7 @@ def _host_bits(g_row, idx):
     return v.numpy()
 
 
-def _check_step(ctx, wl, g, e_prev, k, lr, rng):
+def _check_step(ctx, wl, g, e_prev, k, lr, rng, samples=SAMPLES):
     n, d = wl.n, wl.d
     buf = B.deco_get_buffers(ctx)
     e_new = B.view_f32(buf["e"], (n, buf["e_stride"]))
@@ -61,7 +61,7 @@ def _check_step(ctx, wl, g, e_prev, k, lr, rng):
             taken = idx[kv == t_key]
             assert int(taken.max()) < int(left.min())
         # --- arithmetic on sampled positions, through the oracle's accumulate
-        pos = torch.from_numpy(rng.integers(0, d, SAMPLES)).cuda()
+        pos = torch.from_numpy(rng.integers(0, d, samples)).cuda()
         pos = torch.cat([pos, idx[:: max(1, k // 50_000)]])
         a = O.accumulate(np.float32(lr), _host_bits(g[i], pos),
                          e_prev[i, :d][pos].cpu().numpy())
@@ -159,4 +159,68 @@ def test_full_size_workload(name):
         assert st["device_status"] == 0 and st["exact_pass_workers"] == 0
     finally:
         B.deco_destroy(ctx)
+        torch.cuda.empty_cache()
+
+
+class _Layer:
+    """What _check_step reads of a workload, for one layer of the per-layer variant."""
+    def __init__(self, n, d):
+        self.n, self.d = n, d
+
+
+def test_full_size_per_layer_variant():
+    """GPT-2-small shape, Top-k per tensor (148 layers: 50 through the table-driven kernels, 98
+    through the batch kernels for short layers), two iterations with tau = 1.  On a spread of
+    layers — the two embeddings, every seventh tensor, the last one — each layer's message is
+    pinned as the unique Top-k set of that layer by the properties above, the arithmetic is
+    compared with the oracle on sampled positions, and the update of iteration 1 with the
+    worker-order sum of iteration 0's messages."""
+    wl = W.make_workload("gpt2_small")
+    n = wl.n
+    offsets = [0]
+    for t in wl.tensors:
+        offsets.append(offsets[-1] + int(t.numel))
+    rng = np.random.default_rng(wl.seed + 1)
+    ctx = B.deco_layered_init(wl.d, n, offsets, wl.delta, 1, wl.lr, grad_dtype=B.DECO_BF16)
+    try:
+        info = B.deco_layered_info(ctx)
+        nl = info["n_layers"]
+        chosen = sorted(set([0, 1, nl - 1] + list(range(2, nl, 7))))
+        x_all = B.view_f32(info["params"], (wl.d,))
+        S_prev = {}
+        g = None
+        for t in range(2):
+            g = W.gradients(wl, t, "cuda", out=g)
+            subs, e_prev, x_prev = {}, {}, {}
+            for l in chosen:
+                sub, off, ln = B.deco_layered_layer(ctx, l)
+                buf = B.deco_get_buffers(sub)
+                subs[l] = (sub, off, ln, buf)
+                e_prev[l] = B.view_f32(buf["e"], (n, buf["e_stride"])).clone()
+                x_prev[l] = x_all[off:off + ln].clone()
+            B.deco_layered_step(ctx, g)
+            B.deco_layered_join(ctx)
+            torch.cuda.synchronize()
+            for l in chosen:
+                sub, off, ln, buf = subs[l]
+                k_l = B.deco_get_k(sub)
+                assert k_l == O.k_from_delta(wl.delta, ln)
+                _check_step(sub, _Layer(n, ln), g[:, off:off + ln], e_prev[l], k_l, wl.lr, rng,
+                            samples=min(SAMPLES, 4 * ln))
+                msg = B.view_i32(buf["msg"], (n, buf["k_cap"], 2))
+                S = _dense_from_messages(msg, n, k_l, ln)
+                x_new = x_all[off:off + ln]
+                if t == 0:
+                    assert bool((x_new == 0).all())
+                else:
+                    want = x_prev[l].cpu().numpy().copy()
+                    O.apply_update(want, S_prev[l].cpu().numpy().copy(), np.float32(1.0) / np.float32(n))
+                    assert np.array_equal(x_new.cpu().numpy().view(np.uint32), want.view(np.uint32)), l
+                S_prev[l] = S
+            del e_prev, x_prev
+        for l in range(nl):
+            st = B.deco_get_stats(B.deco_layered_layer(ctx, l)[0])
+            assert st["device_status"] == 0 and st["step"] == 2
+    finally:
+        B.deco_layered_destroy(ctx)
         torch.cuda.empty_cache()
