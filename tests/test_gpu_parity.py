@@ -259,6 +259,30 @@ def test_per_layer_topk_short_layers_batch(kind):
                            tau_max=3, delta_max=1.0)
 
 
+@pytest.mark.parametrize("seed", [31, 32])
+def test_per_layer_seeded_random_partitions(seed):
+    """Layer lengths (1 … 200 K, on both sides of the 8192-entry limit of the batched route),
+    worker counts, densities, staleness, dtypes and value structure drawn from a seeded
+    generator, with a policy change in the middle: bit for bit against the oracle."""
+    rng = np.random.default_rng(seed)
+    for _ in range(6):
+        nl = int(rng.integers(1, 25))
+        lens = [int(rng.choice([rng.integers(1, 200), rng.integers(200, 8193),
+                                rng.integers(8193, 200_000)])) for _ in range(nl)]
+        offsets = [0]
+        for ln in lens:
+            offsets.append(offsets[-1] + ln)
+        d, n = offsets[-1], int(rng.integers(1, 12))
+        delta = float(min(1.0, 10.0 ** rng.uniform(-3.5, 0.1)))
+        delta2 = float(min(1.0, 10.0 ** rng.uniform(-3.5, 0.1)))
+        tau, tau2 = int(rng.integers(0, 4)), int(rng.integers(0, 4))
+        dtype, name = ((torch.float32, "f32"), (torch.bfloat16, "bf16"))[int(rng.integers(0, 2))]
+        kind = str(rng.choice(["normal", "coarse", "all_equal", "two_valued"]))
+        run_layered_parity(offsets, n, delta, tau, 0.1, lambda t: _values(kind, n, d, t, dtype),
+                           steps=5, grad_dtype=name, policy_plan={2: (delta2, tau2)}, tau_max=3,
+                           delta_max=max(delta, delta2))
+
+
 @pytest.mark.parametrize("compressor", ["topk", "randk"])
 def test_worker_sharded_contexts_equal_the_single_job(compressor):
     """Five workers split 2 + 3 over two contexts on one GPU.  Each compresses its own workers;
