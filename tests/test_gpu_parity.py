@@ -259,6 +259,44 @@ def test_per_layer_topk_short_layers_batch(kind):
                            tau_max=3, delta_max=1.0)
 
 
+def test_per_layer_random_k_equals_one_context_per_layer():
+    """Random-k per layer (layer l draws from the stream seeded seed + l) keeps the route that
+    steps every layer's context on its own; it must give what separate ordinary contexts give
+    on the layers' slices (those are checked against the oracle elsewhere)."""
+    lengths = [5000, 8192, 30_001, 70_000]
+    offsets = [0]
+    for ln in lengths:
+        offsets.append(offsets[-1] + ln)
+    d, n, seed = offsets[-1], 3, 4242
+    lay = B.deco_layered_init(d, n, offsets, 0.02, 1, 0.1, compressor=B.DECO_COMPRESSOR_RANDK, seed=seed)
+    flat = [B.deco_init(ln, n, 0.02, 1, 0.1, compressor=B.DECO_COMPRESSOR_RANDK, seed=seed + l)
+            for l, ln in enumerate(lengths)]
+    try:
+        info = B.deco_layered_info(lay)
+        for t in range(4):
+            g = _values("normal", n, d, t, torch.float32)
+            B.deco_layered_step(lay, g)
+            for l, ln in enumerate(lengths):
+                B.deco_step(flat[l], g[:, offsets[l]:offsets[l + 1]].contiguous())
+            B.deco_layered_join(lay)
+            torch.cuda.synchronize()
+            for l, ln in enumerate(lengths):
+                sub, off, _ = B.deco_layered_layer(lay, l)
+                ba, bb = B.deco_get_buffers(sub), B.deco_get_buffers(flat[l])
+                k = B.deco_get_k(sub)
+                assert k == B.deco_get_k(flat[l])
+                assert torch.equal(B.view_i32(ba["msg"], (n, ba["k_cap"], 2))[:, :k],
+                                   B.view_i32(bb["msg"], (n, bb["k_cap"], 2))[:, :k]), (t, l)
+                assert torch.equal(B.view_i32(ba["e"], (n, ba["e_stride"])),
+                                   B.view_i32(bb["e"], (n, bb["e_stride"]))), (t, l)
+                assert torch.equal(B.view_i32(info["params"], (d,))[off:off + ln],
+                                   B.view_i32(bb["params"], (ln,))), (t, l)
+    finally:
+        B.deco_layered_destroy(lay)
+        for c in flat:
+            B.deco_destroy(c)
+
+
 @pytest.mark.parametrize("seed", [31, 32])
 def test_per_layer_seeded_random_partitions(seed):
     """Layer lengths (1 … 200 K, on both sides of the 8192-entry limit of the batched route),
