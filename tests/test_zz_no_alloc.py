@@ -7,6 +7,8 @@ array inside the library.  This file is collected last on purpose, so that a run
 at the first failure has already run every other test; it also passes on its own in a fresh
 process.  Two calls in a row check that nothing of the first call's scratch contents leaks
 into the second."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -51,11 +53,15 @@ def test_static_entry_point_matches_context_path_twice_in_a_row():
     cases.append((coarse, k2))
     want = [_reference_message(a, k) for a, k in cases]
     outs = [torch.full((k, 2), -1, dtype=torch.int32, device="cuda") for _, k in cases]
+    # Tensors left over from earlier tests may be released by Python's collector at any moment,
+    # which lowers the counter: collect them first, and accept only "no growth" afterwards.
+    gc.collect()
+    torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
     for (a, k), out in zip(cases, outs):                         # two calls back to back
         B.deco_topk_compress_static(a, a.numel(), k, out)
     torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before
+    assert torch.cuda.memory_allocated() <= before               # nothing was allocated through torch
     for (a, k), out, ref in zip(cases, outs, want):
         # integer indices and copied values: the tolerance of the parity tests is bit-exact
         assert torch.equal(out, ref)
