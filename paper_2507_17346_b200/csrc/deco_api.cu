@@ -760,6 +760,10 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
         h.compressor != static_cast<uint32_t>(c->compressor) || h.seed != c->seed ||
         h.sharding != ((c->n_total << 16) | c->worker_base))
         return DECO_ERR_INVALID_ARG;
+    // a blob that was cut, edited or damaged: the policy must be one deco_set_policy accepts
+    if (!(h.delta > 0.0) || !(h.delta <= 1.0) || h.k < 1 || h.k != deco_k_from_delta(h.delta, c->d) ||
+        !(h.lr == h.lr))
+        return DECO_ERR_INVALID_ARG;
     if (bytes < sizeof(StateHeader) + sizeof(SlotRecord) * c->ring) return DECO_ERR_INVALID_ARG;
     std::vector<Slot> slots(c->ring);
     uint64_t need = sizeof(StateHeader) + sizeof(SlotRecord) * c->ring +
@@ -768,7 +772,11 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
         SlotRecord r;
         std::memcpy(&r, in, sizeof r);
         in += sizeof r;
-        if (r.valid && (r.positions > static_cast<uint64_t>(c->n_total) * c->k_cap || r.step % c->ring != q))
+        // a cached aggregate was sent in one of the last `ring` iterations before t and holds
+        // the same number of positions for every worker
+        if (r.valid && (r.positions > static_cast<uint64_t>(c->n_total) * c->k_cap ||
+                        r.positions < c->n_total || r.positions % c->n_total != 0 ||
+                        r.step % c->ring != q || r.step >= h.t || r.step + c->ring < h.t))
             return DECO_ERR_INVALID_ARG;
         slots[q].step = r.step;
         slots[q].positions = r.positions;

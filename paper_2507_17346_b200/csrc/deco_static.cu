@@ -293,6 +293,8 @@ extern "C" deco_status deco_topk_compress_static(const float *a, uint64_t d, uin
     const uint32_t k32 = static_cast<uint32_t>(k);
     uint32_t hblocks = static_cast<uint32_t>((d + ST_BLOCK * 16 - 1) / (ST_BLOCK * 16));
     if (hblocks > 148 * 8) hblocks = 148 * 8;
+    // an error some earlier, unrelated launch of this thread left behind is not this call's
+    (void)cudaGetLastError();
     st_clear_kernel<<<32, 256, 0, s>>>(scratch, k32, ntiles);
     st_hist_kernel<0><<<hblocks, ST_BLOCK, 0, s>>>(a, d, scratch);
     st_pick_kernel<0><<<1, ST_BLOCK, 0, s>>>(scratch);

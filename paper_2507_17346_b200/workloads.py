@@ -250,6 +250,44 @@ def gradients(wl, step, device="cpu", out=None):
     return out
 
 
+def entry_scales(wl, device="cpu"):
+    """Per-entry multiplier [d] float32 that turns unit draws into the workload's values:
+    1/sqrt(fan_in) of the entry's tensor (Student-t recipe), sigma times the layer's scale,
+    sigma times 50 on the outlier rows, or sigma."""
+    parts = []
+    scales = layer_scales(wl) if wl.dist == "normal_layer_scale" else None
+    for ti, spec in enumerate(wl.tensors):
+        if wl.dist == "student_t":
+            parts.append(torch.full((spec.numel,), 1.0 / float(spec.fan_in) ** 0.5))
+        elif wl.dist == "normal_layer_scale":
+            parts.append(torch.full((spec.numel,), wl.sigma * scales[ti]))
+        elif wl.dist == "normal_outlier_rows":
+            cols = spec.fan_in if len(spec.shape) > 1 else 1
+            rows = outlier_rows(wl, ti).repeat_interleave(cols)
+            parts.append(torch.where(rows, 50.0 * wl.sigma, wl.sigma).to(torch.float32))
+        else:
+            parts.append(torch.full((spec.numel,), float(wl.sigma)))
+    return torch.cat(parts).to(torch.float32).to(device)
+
+
+def gradients_batched(wl, step, scales, out=None):
+    """The workload's distribution drawn for all workers at once (a handful of device launches
+    per step instead of several per tensor and worker): unit draws [n, d] times `scales` =
+    entry_scales(wl, device).  Another stream than gradients(), the same recipe."""
+    device = scales.device
+    gen = _gen(device, _mix(wl.seed, step, 0x6261))
+    z = torch.randn((wl.n, wl.d), generator=gen, device=device, dtype=torch.float32)
+    if wl.dist == "student_t":
+        w = torch.randn((3, wl.n, wl.d), generator=gen, device=device, dtype=torch.float32)
+        z = z / torch.sqrt((w * w).sum(0) / 3.0)
+    z = z * scales
+    dtype = torch.float32 if wl.grad_dtype == "f32" else torch.bfloat16
+    if out is None:
+        return z.to(dtype)
+    out.copy_(z)
+    return out
+
+
 def to_numpy_bits(g):
     """Host copy for the oracle: float32 array, or uint16 bit patterns for bfloat16."""
     g = g.detach().cpu().contiguous()

@@ -1,8 +1,15 @@
-"""Full-size parity in the launch configuration the benchmark times: the three workloads with
-d >= 100 M.  The oracle cannot sort 10^9 entries in seconds, so the unique Top-k set is pinned
-by properties that hold at any size (count, strict index order, threshold domination, tie cut
-by index — together they admit exactly one set), and every arithmetic result is compared with
-the oracle's own functions on sampled positions, bit for bit."""
+"""Full-size parity in the launch configuration the benchmark times (`deco_step`, with the
+stale update and the aggregation on the library's internal streams), at each workload's own
+(delta, tau) and step count: the three workloads with d >= 100 M.
+
+The oracle cannot sort 10^9 entries for every worker and step in seconds, so at every step the
+unique Top-k set is pinned by properties that hold at any size (count, strict index order,
+threshold domination, tie cut by index: together they admit exactly one set) and every
+arithmetic result is compared bit for bit with the oracle's own functions on sampled
+positions; on the first two and the last step one worker's whole residual, message and the
+whole parameter vector go through the oracle's arithmetic on the host, and at step 0 one
+worker's index set is compared with the oracle's full sort where d allows it.  Which cached
+aggregates an update applies is modelled here by a plain FIFO (exactly-once drain)."""
 import numpy as np
 import pytest
 import torch
@@ -15,6 +22,7 @@ pytestmark = pytest.mark.gpu
 
 ABS = 0x7FFFFFFF
 SAMPLES = 200_000
+SORT_LIMIT = 130_000_000          # the oracle's full sort is run up to this length
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -28,9 +36,9 @@ def _keys(t):
     return t.view(torch.int32) & ABS
 
 
-def _host_bits(g_row, idx):
-    """Gradient entries at idx as the oracle wants them (float32 or bfloat16 bit patterns)."""
-    v = g_row[idx].cpu()
+def _host_bits(v):
+    """A gradient tensor as the oracle wants it (float32, or bfloat16 bit patterns)."""
+    v = v.cpu()
     if v.dtype == torch.bfloat16:
         return v.view(torch.int16).numpy().view(np.uint16)
     return v.numpy()
@@ -63,8 +71,7 @@ def _check_step(ctx, wl, g, e_prev, k, lr, rng, samples=SAMPLES):
         # --- arithmetic on sampled positions, through the oracle's accumulate
         pos = torch.from_numpy(rng.integers(0, d, samples)).cuda()
         pos = torch.cat([pos, idx[:: max(1, k // 50_000)]])
-        a = O.accumulate(np.float32(lr), _host_bits(g[i], pos),
-                         e_prev[i, :d][pos].cpu().numpy())
+        a = O.accumulate(np.float32(lr), _host_bits(g[i][pos]), e_prev[i, :d][pos].cpu().numpy())
         sent = torch.zeros(d, dtype=torch.bool, device="cuda")
         sent[idx] = True
         is_sent = sent[pos].cpu().numpy()
@@ -78,6 +85,23 @@ def _check_step(ctx, wl, g, e_prev, k, lr, rng, samples=SAMPLES):
         del sent
 
 
+def _check_worker_in_full(ctx, wl, g, e_prev, k, lr, i, with_sort):
+    """Worker i's whole residual and message through the oracle's arithmetic on the host."""
+    n, d = wl.n, wl.d
+    buf = B.deco_get_buffers(ctx)
+    e_new = B.view_f32(buf["e"], (n, buf["e_stride"]))
+    msg = B.view_i32(buf["msg"], (n, buf["k_cap"], 2))
+    a = O.accumulate(np.float32(lr), _host_bits(g[i]), e_prev[i, :d].cpu().numpy())
+    idx = msg[i, :k, 0].cpu().numpy().view(np.uint32)
+    val = np.ascontiguousarray(msg[i, :k, 1].cpu().numpy()).view(np.uint32)
+    assert np.array_equal(val, a[idx].view(np.uint32))                # values are a verbatim
+    if with_sort:
+        assert np.array_equal(idx, O.topk_select(a, k))               # the oracle's own selection
+    a[idx] = np.float32(0.0)
+    got = e_new[i, :d].cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), a.view(np.uint32))     # e = a - Delta, every entry
+
+
 def _dense_from_messages(msg, n, k, d):
     """Worker-order fp32 sum from +0 with torch index_put (one worker at a time)."""
     S = torch.zeros(d, dtype=torch.float32, device="cuda")
@@ -87,79 +111,162 @@ def _dense_from_messages(msg, n, k, d):
     return S
 
 
-@pytest.mark.parametrize("name", ["gpt2_small", "sweep_100m", "decoder_1b"])
-def test_full_size_workload(name):
-    wl = W.make_workload(name)
+def _check_aggregate(ctx, t, msg, S, n, k, d, rng):
+    """The cached aggregate of step t: every touched index once, increasing, with the
+    worker-order fp32 sum; and the oracle's aggregate on a sample of the touched indices."""
+    addr, positions = B.deco_get_aggregate(ctx, t)
+    assert positions == n * k
+    slot = B.view_i32(addr, (positions, 2))
+    keep = slot[:, 0] != -1
+    sidx = slot[keep, 0].long()
+    sval = slot[keep, 1].contiguous().view(torch.float32)
+    touched = torch.zeros(d, dtype=torch.bool, device="cuda")
+    for i in range(n):
+        touched[msg[i, :k, 0].long()] = True
+    assert int(sidx.numel()) == int(touched.sum())
+    assert bool((sidx[1:] > sidx[:-1]).all()) and bool(touched[sidx].all())
+    assert bool((sval.view(torch.int32) == S[sidx].view(torch.int32)).all())
+    del touched
+    pick = sidx[torch.from_numpy(rng.integers(0, sidx.numel(), 100_000)).cuda()].unique()
+    small = []
+    for i in range(n):
+        idx_i = msg[i, :k, 0].long()
+        m = torch.isin(idx_i, pick)
+        small.append((torch.searchsorted(pick, idx_i[m]).cpu().numpy().astype(np.uint32),
+                      msg[i, :k, 1][m].contiguous().view(torch.float32).cpu().numpy()))
+    S_orc, _ = O.aggregate(small, int(pick.numel()))
+    got = sval[torch.searchsorted(sidx, pick)].cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), S_orc.view(np.uint32))
+
+
+def _run_as_configured(wl, delta, tau, steps, fused, plan=None, tau_max=0, delta_max=0.0,
+                       full_steps=None, expect_no_multipass=True):
+    """`steps` iterations at full size.  fused: deco_step (what the benchmark times), else the
+    three calls.  plan: {step: (delta, tau)} applied before that step (Algorithm 2)."""
     n, d = wl.n, wl.d
-    tau = 1                                   # apply from the second step on (ring logic is
-    steps = 3                                 # covered at small sizes); delta and the rest as configured
+    if full_steps is None:
+        full_steps = {0, 1, steps - 1}
     rng = np.random.default_rng(wl.seed)
-    ctx = B.deco_init(d, n, wl.delta, tau, wl.lr,
-                      grad_dtype=B.DECO_F32 if wl.grad_dtype == "f32" else B.DECO_BF16)
+    scale = np.float32(1.0) / np.float32(n)
+    ctx = B.deco_init(d, n, delta, tau, wl.lr,
+                      grad_dtype=B.DECO_F32 if wl.grad_dtype == "f32" else B.DECO_BF16,
+                      tau_max=tau_max, delta_max=delta_max)
     try:
         k = B.deco_get_k(ctx)
-        assert k == O.k_from_delta(wl.delta, d)
+        assert k == O.k_from_delta(delta, d)
         buf = B.deco_get_buffers(ctx)
         e_view = B.view_f32(buf["e"], (n, buf["e_stride"]))
         x_view = B.view_f32(buf["params"], (d,))
         msg = B.view_i32(buf["msg"], (n, buf["k_cap"], 2))
-        S_prev = None
+        cache = []                                   # server cache model: (step, dense S), FIFO
         g = None
+        applied_total = 0
         for t in range(steps):
+            if plan and t in plan:
+                delta, tau = plan[t]
+                B.deco_set_policy(ctx, delta, tau)
+                k = B.deco_get_k(ctx)
+                assert k == O.k_from_delta(delta, d)
             g = W.gradients(wl, t, "cuda", out=g)
             e_prev = e_view.clone()
             x_prev = x_view.clone()
-            B.deco_ef_compress(ctx, g)
+            if fused:
+                B.deco_step(ctx, g)
+                B.deco_join(ctx)
+            else:
+                B.deco_ef_compress(ctx, g)
+                B.deco_aggregate_stale(ctx)
+                B.deco_apply_update(ctx)
+            torch.cuda.synchronize()
             _check_step(ctx, wl, g, e_prev, k, wl.lr, rng)
+            if t in full_steps:
+                _check_worker_in_full(ctx, wl, g, e_prev, k, wl.lr, t % n,
+                                      with_sort=(t == 0 and d <= SORT_LIMIT))
             del e_prev
-            B.deco_aggregate_stale(ctx)
-            # aggregate: every touched index once, with the worker-order fp32 sum
             S = _dense_from_messages(msg, n, k, d)
-            addr, positions = B.deco_get_aggregate(ctx, t)
-            slot = B.view_i32(addr, (positions, 2))
-            keep = slot[:, 0] != -1
-            sidx = slot[keep, 0].long()
-            sval = slot[keep, 1].contiguous().view(torch.float32)
-            touched = torch.zeros(d, dtype=torch.bool, device="cuda")
-            for i in range(n):
-                touched[msg[i, :k, 0].long()] = True
-            assert int(sidx.numel()) == int(touched.sum())
-            assert bool((sidx[1:] > sidx[:-1]).all()) and bool(touched[sidx].all())
-            assert bool((sval.view(torch.int32) == S[sidx].view(torch.int32)).all())
-            del touched
-            # the same through the oracle's aggregate, on a sample of the touched indices
-            pick = sidx[torch.from_numpy(rng.integers(0, sidx.numel(), 100_000)).cuda()].unique()
-            small = []
-            for i in range(n):
-                idx_i = msg[i, :k, 0].long()
-                m = torch.isin(idx_i, pick)
-                small.append((torch.searchsorted(pick, idx_i[m]).cpu().numpy().astype(np.uint32),
-                              msg[i, :k, 1][m].contiguous().view(torch.float32).cpu().numpy()))
-            S_orc, _ = O.aggregate(small, int(pick.numel()))
-            got = sval[torch.searchsorted(sidx, pick)].cpu().numpy()
-            assert np.array_equal(got.view(np.uint32), S_orc.view(np.uint32))
-            B.deco_apply_update(ctx)
-            if t >= tau:
-                # x_new = fma(-1/n, S_{t-tau}, x_old) through the oracle on sampled positions
+            if tau > 0:                              # with tau = 0 the slot is consumed at once
+                _check_aggregate(ctx, t, msg, S, n, k, d, rng)
+            cache.append((t, S))
+            due = [(s, Ss) for (s, Ss) in cache if s <= t - tau]     # oldest first
+            cache = [(s, Ss) for (s, Ss) in cache if s > t - tau]
+            applied_total += len(due)
+            if not due:
+                assert bool((x_view.view(torch.int32) == x_prev.view(torch.int32)).all())
+            else:
+                # x = fma(-1/n, S_s, x) for every due aggregate in turn, through the oracle
                 pos = torch.from_numpy(rng.integers(0, d, SAMPLES)).cuda()
-                pos = torch.cat([pos, torch.nonzero(S_prev).flatten()[::97][:SAMPLES]])
+                pos = torch.cat([pos] + [torch.nonzero(Ss).flatten()[::97][:SAMPLES] for _, Ss in due])
                 xs = x_prev[pos].cpu().numpy().copy()
-                O.apply_update(xs, S_prev[pos].cpu().numpy().copy(), np.float32(1.0) / np.float32(n))
+                for _, Ss in due:
+                    O.apply_update(xs, Ss[pos].cpu().numpy().copy(), scale)
                 got = x_view[pos].cpu().numpy()
                 assert np.array_equal(got.view(np.uint32), xs.view(np.uint32))
-                untouched = (S_prev == 0)
+                untouched = due[0][1] == 0
+                for _, Ss in due[1:]:
+                    untouched &= Ss == 0
                 assert bool((x_view.view(torch.int32)[untouched] ==
                              x_prev.view(torch.int32)[untouched]).all())
                 del untouched
-            else:
-                assert bool((x_view == 0).all())
-            S_prev = S
-            del x_prev
+                if t in full_steps:                  # the whole parameter vector
+                    xh = x_prev.cpu().numpy().copy()
+                    for _, Ss in due:
+                        O.apply_update(xh, Ss.cpu().numpy(), scale)
+                    assert np.array_equal(x_view.cpu().numpy().view(np.uint32), xh.view(np.uint32))
+                    del xh
+            del x_prev, due
         st = B.deco_get_stats(ctx)
-        assert st["device_status"] == 0 and st["exact_pass_workers"] == 0
+        assert st["device_status"] == 0 and st["step"] == steps
+        assert st["cached_aggregates"] == len(cache)
+        if expect_no_multipass:
+            assert st["exact_pass_workers"] == 0
+        return applied_total
     finally:
         B.deco_destroy(ctx)
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["gpt2_small", "decoder_1b"])
+def test_full_size_workload_as_configured(name):
+    """Configurations 3 and 5: own delta, tau (8 / 4) and step count (20 / 10), so that the
+    cache fills, wraps and 12 / 6 stale updates are applied."""
+    wl = W.make_workload(name)
+    applied = _run_as_configured(wl, wl.delta, wl.tau, wl.steps, fused=True)
+    assert applied == wl.steps - wl.tau
+
+
+@pytest.mark.parametrize("delta,tau,fused", [(0.1, 0, False), (0.1, 16, True),
+                                             (0.0001, 0, True), (0.0001, 16, False)])
+def test_full_size_sweep_corners(delta, tau, fused):
+    """Configuration 4 at d = 10^8: the four corners of the delta x tau grid (10^7 and 10^4
+    entries per message; no staleness and a 17-slot cache that wraps)."""
+    wl = W.make_workload("sweep_100m")
+    steps = tau + 4
+    applied = _run_as_configured(wl, delta, tau, steps, fused=fused,
+                                 full_steps={0, steps - 1})
+    assert applied == steps - tau
+
+
+def test_full_size_adaptive_run():
+    """Configuration 4, second half: 200 iterations at d = 10^8 in which DeCo (Algorithm 3)
+    re-selects (delta, tau) every E = 10 iterations from the synthetic trace (Algorithm 2); the
+    library's decision must equal the oracle's, and every iteration is checked as above."""
+    from oracle import deco_policy as P
+    wl = W.make_workload("sweep_100m")
+    d, steps, E = wl.d, 200, 10
+    V_g, T_comp, tau_max, delta_max = 32.0 * d, 0.05, 16, 0.2
+    lat, bw = W.network_trace(wl.seed, steps)
+    plan = {}
+    for t in range(E, steps, E):                      # decided after iteration t-1
+        a_bar, b = float(np.mean(bw[t - E:t])), float(lat[t - 1])
+        tau, delta = B.deco_policy_select(V_g, a_bar, b, T_comp, tau_max, False)
+        otau, odelta = P.deco_select(V_g, a_bar, b, T_comp)
+        if otau > tau_max:
+            otau, odelta = tau_max, P.delta_star(tau_max, V_g, a_bar, b, T_comp)
+        assert (tau, delta) == (otau, pytest.approx(odelta, rel=1e-12))
+        plan[t] = (min(delta_max, max(delta, 1.0 / d)), tau)
+    assert len(set(plan.values())) >= 3               # the trace does move the decision
+    _run_as_configured(wl, 0.01, 2, steps, fused=True, plan=plan, tau_max=tau_max,
+                       delta_max=delta_max, full_steps={0, 1, steps - 1})
 
 
 class _Layer:

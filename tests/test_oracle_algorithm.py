@@ -154,3 +154,68 @@ def test_quadratic_converges_to_known_minimiser():
     mixed = rng.standard_normal((n, d)).astype(np.float32)
     coarse, fine = run(mixed, 1.0 / (4 * tau), 800), run(mixed, 1.0 / (16 * tau), 3000)
     assert fine < 0.5 * coarse
+
+
+def test_apply_update_is_one_fused_rounding():
+    """Server update of Algorithm 1, x <- x - scale*S, pinned bit for bit against exact
+    rational arithmetic with a single rounding (no fmaf is called on the checking side).  The
+    triples include ones where rounding the product scale*S first gives different bits."""
+    from tests import exact_arith as X
+    rng = np.random.default_rng(7)
+    m = 300
+    S = (rng.standard_normal(m) * 10.0 ** rng.integers(-5, 5, m)).astype(np.float32)
+    x = (rng.standard_normal(m) * 10.0 ** rng.integers(-5, 5, m)).astype(np.float32)
+    # crafted: scale*S needs more than 24 bits and nearly cancels x
+    S[0], x[0] = np.float32(1.0 + 2 ** -12), np.float32(1.0 / 3.0)
+    S[1], x[1] = np.float32(3.0 + 2 ** -20), np.float32(1.0)
+    S[2], x[2] = np.float32(0.0), np.float32(-0.0)
+    S[3], x[3] = np.float32(1e-42), np.float32(-1e-43)           # subnormals
+    differs = 0
+    for scale in (np.float32(1.0) / np.float32(3.0), np.float32(0.1) / np.float32(4.0),
+                  np.float32(0.25), np.float32(1.0 + 2 ** -12)):
+        got = x.copy()
+        O.apply_update(got, S.copy(), scale)
+        neg = X.f32_bits(float(-np.float32(scale)))
+        for j in range(m):
+            want = X.fma_f32_bits(neg, X.f32_bits(float(S[j])), X.f32_bits(float(x[j])))
+            assert int(got[j:j + 1].view(np.uint32)[0]) == want, (float(scale), j, S[j], x[j])
+        two_step = x - (np.float32(scale) * S).astype(np.float32)
+        differs += int(np.sum(got.view(np.uint32) != two_step.view(np.uint32)))
+    assert differs > 0          # the pin can tell one rounding from two
+
+
+def _sequential_f32_sum_bits(terms):
+    """Bits of ((0 + t0) + t1) + ... with one rounding per addition, by exact arithmetic."""
+    from tests import exact_arith as X
+    one = X.f32_bits(1.0)
+    acc = 0                                                  # +0
+    for t in terms:
+        acc = X.fma_f32_bits(one, X.f32_bits(float(t)), acc)   # 1*t + acc, rounded once
+    return acc
+
+
+def test_aggregate_sums_in_worker_order_from_plus_zero():
+    """S = sum_i Delta^i is taken in fp32 in worker order 0..n-1 starting from +0 (fp32 addition
+    is not associative, so the order is part of the result).  Three workers send the same index
+    with values whose sum depends on the order; the expected bits come from exact arithmetic
+    with one rounding per addition in the order 0, 1, 2, and differ from the reversed order."""
+    d = 6
+    big, small = np.float32(2.0 ** 24), np.float32(1.0)
+    cases = [
+        (np.array([big, small, small], np.float32)),           # (2^24 + 1) + 1 = 2^24 ; reversed: 2^24 + 2
+        (np.array([small, small, big], np.float32)),
+        (np.array([np.float32(1e8), np.float32(-1e8), np.float32(3.25)], np.float32)),
+        (np.array([np.float32(0.1), np.float32(0.2), np.float32(-0.3)], np.float32)),
+    ]
+    order_matters = 0
+    for vals in cases:
+        msgs = [(np.array([4], np.uint32), vals[i:i + 1].copy()) for i in range(3)]
+        # a second index sent only by worker 1: must come out as 0 + v, i.e. v itself
+        msgs[1] = (np.array([2, 4], np.uint32), np.array([np.float32(-0.0), vals[1]], np.float32))
+        S, S64 = O.aggregate(msgs, d)
+        assert int(S[4:5].view(np.uint32)[0]) == _sequential_f32_sum_bits(vals)
+        assert int(S[2:3].view(np.uint32)[0]) == 0              # +0 + -0 = +0
+        assert S64[4] == float(vals[0]) + float(vals[1]) + float(vals[2])     # float64 shadow
+        assert np.all(S[[0, 1, 3, 5]].view(np.uint32) == 0)
+        order_matters += _sequential_f32_sum_bits(vals) != _sequential_f32_sum_bits(vals[::-1])
+    assert order_matters >= 2   # the pin can tell the order 0..n-1 from its reverse

@@ -57,6 +57,14 @@ def _aggregate_drops_last_worker(msgs, d):
     return ORIG_AGGREGATE(msgs[:-1], d)
 
 
+def _aggregate_reversed_order(msgs, d):               # workers summed n-1..0
+    return ORIG_AGGREGATE(msgs[::-1], d)
+
+
+def _apply_two_roundings(x, S, scale):                # product rounded before the subtraction
+    x -= (np.float32(scale) * S).astype(np.float32)
+
+
 ORIG_AGGREGATE = O.aggregate
 ORIG_STEP = O.DDEFSGD.step
 
@@ -71,7 +79,9 @@ ALGO_PINS = [TA.test_delta1_tau0_is_dsgd, TA.test_delta1_is_delayed_aggregation,
              TA.test_update_t_uses_exactly_aggregate_t_minus_tau,
              TA.test_tau0_is_compression_with_error_feedback,
              TA.test_error_conservation_per_worker_and_global,
-             TA.test_quadratic_converges_to_known_minimiser]
+             TA.test_quadratic_converges_to_known_minimiser,
+             TA.test_apply_update_is_one_fused_rounding,
+             TA.test_aggregate_sums_in_worker_order_from_plus_zero]
 POLICY_PINS = [TP.test_phi_degradation_conditions,
                TP.test_delta_star_is_the_largest_ratio_with_no_pipeline_bubble,
                TP.test_deco_select_matches_brute_force_and_hand_cases,
@@ -93,6 +103,10 @@ def test_pins_pass_unmutated():
      lambda delta, d: max(1, min(int(d), int(math.floor(delta * d)))), COMPRESS_PINS),
     ("update added instead of subtracted", O, "apply_update", _apply_wrong_sign, ALGO_PINS),
     ("last worker not aggregated", O, "aggregate", _aggregate_drops_last_worker, ALGO_PINS),
+    ("workers summed in reverse order", O, "aggregate", _aggregate_reversed_order,
+     [TA.test_aggregate_sums_in_worker_order_from_plus_zero]),
+    ("update with two roundings", O, "apply_update", _apply_two_roundings,
+     [TA.test_apply_update_is_one_fused_rounding]),
     ("phi without the staleness power", P, "phi",
      lambda delta, tau: (1 - delta) / delta, POLICY_PINS),
     ("phi with (1 - delta)^tau", P, "phi",
