@@ -98,7 +98,7 @@ typedef struct {
     int32_t  compressor;     /* deco_compressor; default Top-k */
     uint32_t seed_lo;        /* Random-k: 64-bit seed of the priority stream, low word */
     uint32_t seed_hi;        /*           high word */
-    uint32_t n_total;        /* worker-sharded context: workers of the whole job (0: n) */
+    uint32_t n_total;        /* worker-sharded context: workers of the whole job (0: n, no exchange buffer) */
     uint32_t worker_base;    /* ... and the global id of this context's first worker */
     uint32_t reserved[3];    /* must be zero */
 } deco_options;
@@ -150,8 +150,10 @@ deco_status deco_ef_compress(deco_ctx *ctx, const void *grads, void *stream);
 /*
  * Server side, arrival of iteration t's messages (Algorithm 1: the sum inside
  * "x = x - (1/n) sum_i Delta_{t-tau}^i", kept in the server's cache of stale updates):
- * S_t[j] = sum over workers, in worker order, of the values sent for index j, stored sparsely
- * in cache slot t mod (tau_max + 1).  Must follow deco_ef_compress of the same iteration.
+ * S_t[j] = sum over workers, in worker order, of the values sent for index j, stored in cache
+ * slot t mod (tau_max + 1): as (index, sum) pairs, or, when the n messages together hold at
+ * least d / 4 entries, as the plain vector S_t[0 .. d) (see deco_get_aggregate_vector).  Must
+ * follow deco_ef_compress of the same iteration.
  */
 deco_status deco_aggregate_stale(deco_ctx *ctx, void *stream);
 
@@ -251,19 +253,28 @@ deco_status deco_get_k(const deco_ctx *ctx, uint64_t *k /* HOST */);
 /*
  * Device pointers of the library-owned state (any out-pointer may be NULL):
  *   e       [n][e_stride] fp32, error terms; columns >= d are padding
- *   msg     [n][k_cap] pairs, the messages of the last deco_ef_compress (first k valid)
+ *   msg     [n][k_cap] pairs, the messages of the last deco_ef_compress (first k valid); *k_cap is
+ *           the distance between rows in pairs: k(delta_max), or, in a context created with
+ *           n_total, half the current exchange row (see deco_get_exchange)
  *   params  [d] fp32
  */
 deco_status deco_get_buffers(deco_ctx *ctx, float **e, uint64_t *e_stride, deco_pair **msg,
                              uint64_t *k_cap, float **params);
 
 /*
- * The cached aggregate of iteration `step` (must still be in the cache): DEVICE pointer to
- * `positions` pairs; positions with idx == DECO_NO_INDEX are unused, the others hold each
- * touched index once (increasing) with its fp32 sum.
+ * The cached aggregate of iteration `step` (must still be in the cache), in the layout the
+ * library chose when it was formed (Algorithm 1 only fixes its value, S_step = sum_i Delta^i):
+ *   deco_get_aggregate         pair layout: DEVICE pointer to `positions` pairs; positions with
+ *                              idx == DECO_NO_INDEX are unused, the others hold each touched
+ *                              index once (increasing) with its fp32 sum
+ *   deco_get_aggregate_vector  vector layout (messages of at least d / 4 entries in all):
+ *                              DEVICE pointer to d fp32 values, S_step[j] at j, +0 where no
+ *                              worker sent j
+ * Each returns DECO_ERR_STATE when the aggregate is kept in the other layout (or is not cached).
  */
 deco_status deco_get_aggregate(deco_ctx *ctx, uint64_t step, const deco_pair **entries,
                                uint64_t *positions);
+deco_status deco_get_aggregate_vector(deco_ctx *ctx, uint64_t step, const float **values);
 
 /*
  * Per-worker facts about the last deco_ef_compress (waits for `stream`); each HOST array has
@@ -314,26 +325,28 @@ uint64_t deco_launch_count(const deco_ctx *ctx);
 
 /*
  * Algorithm 1's workers are separate machines that exchange only the sparse messages.  A
- * context created with opt->n_total > n holds n of the job's n_total workers (global ids
+ * context created with opt->n_total >= n holds n of the job's n_total workers (global ids
  * worker_base ... worker_base + n - 1: e, gradients and the worker side are local) and a full
- * replica of the server side: its message buffer and tile directory have n_total rows,
- * deco_ef_compress fills the context's own rows, the CALLER brings the other rows in (one
- * all-gather of the two buffers among the contexts of the job: NCCL over NVLink between GPUs,
- * plain copies between contexts on one GPU), then deco_aggregate_stale sums all n_total
- * messages in global worker order and deco_apply_update scales by 1/n_total, so every replica
- * of x stays bit-identical to the single-context run.  Random-k draws with the global id.
- * deco_step is not available on such a context (the exchange sits between its parts):
- * DECO_ERR_STATE.
+ * replica of the server side.  Its messages live in one exchange buffer of n_total rows:
  *
- * Buffers to exchange, valid for the context's lifetime (all DEVICE):
- *   msg_all   [n_total][msg_row_pairs] pairs; row w = message of global worker w, the first
- *             k pairs of a row are meaningful
- *   dir_all   [n_total][dir_row_words] u32; row w = message position of every tile of worker w
- *             (dir_row_words = tiles + 1)
- * row0 / rows_local: the rows this context writes.  Every out pointer may be NULL.
+ *   row w = | k pairs: the message of global worker w | tiles + 1 words: message position of
+ *           | every 8192-entry index block of worker w | padding to an even number of words |
+ *
+ * with k the current number of kept entries (not the capacity k(delta_max)), rows back to back.
+ * deco_ef_compress fills the context's own rows; the CALLER brings the other rows in with ONE
+ * all-gather of rows_total * row_words 32-bit words among the contexts of the job (NCCL over
+ * NVLink between GPUs: the rows land in local memory; plain copies between contexts on one
+ * GPU); then deco_aggregate_stale sums all n_total messages in global worker order and
+ * deco_apply_update scales by 1/n_total, so every replica of x stays bit-identical to the
+ * single-context run.  Random-k draws with the global id.  deco_step is not available while
+ * n_total > n (the exchange sits between its parts): DECO_ERR_STATE.
+ *
+ *   rows        DEVICE, the exchange buffer, valid for the context's lifetime
+ *   row_words   words per row for the current k; changes when deco_set_policy changes k
+ *   row0 / rows_local   the rows this context writes;  rows_total = n_total
+ * Every out pointer may be NULL.  DECO_ERR_STATE for a context created without n_total.
  */
-deco_status deco_get_exchange(deco_ctx *ctx, deco_pair **msg_all, uint64_t *msg_row_pairs,
-                              uint32_t **dir_all, uint64_t *dir_row_words, uint32_t *row0,
+deco_status deco_get_exchange(deco_ctx *ctx, uint32_t **rows, uint64_t *row_words, uint32_t *row0,
                               uint32_t *rows_local, uint32_t *rows_total);
 
 /* ------------------------------------------------------------- per-layer Top-k (variant) */

@@ -101,6 +101,7 @@ SIGNATURES = {
     "deco_get_k": (_i32, [_vp, _P(_u64)]),
     "deco_get_buffers": (_i32, [_vp, _P(_vp), _P(_u64), _P(_vp), _P(_u64), _P(_vp)]),
     "deco_get_aggregate": (_i32, [_vp, _u64, _P(_vp), _P(_u64)]),
+    "deco_get_aggregate_vector": (_i32, [_vp, _u64, _P(_vp)]),
     "deco_get_select_info": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "deco_get_stats": (_i32, [_vp, _vp, _P(deco_stats)]),
     "deco_set_kernel_timing": (_i32, [_vp, _i32]),
@@ -109,8 +110,7 @@ SIGNATURES = {
     "deco_export_state": (_i32, [_vp, _vp, _u64, _vp]),
     "deco_import_state": (_i32, [_vp, _vp, _u64, _vp]),
     "deco_launch_count": (_u64, [_vp]),
-    "deco_get_exchange": (_i32, [_vp, _P(_vp), _P(_u64), _P(_vp), _P(_u64), _P(_u32), _P(_u32),
-                                 _P(_u32)]),
+    "deco_get_exchange": (_i32, [_vp, _P(_vp), _P(_u64), _P(_u32), _P(_u32), _P(_u32)]),
     "deco_topk_compress_static": (_i32, [_vp, _u64, _u64, _vp, _vp]),
     "deco_layered_init": (_i32, [_P(_vp), _u64, _u32, _P(_u64), _u32, _f64, _u32, _f32, _vp]),
     "deco_layered_destroy": (None, [_vp]),
@@ -352,6 +352,14 @@ def deco_get_aggregate(ctx, step):
     return entries.value, positions.value
 
 
+def deco_get_aggregate_vector(ctx, step):
+    """-> device address of the d fp32 values of a cached aggregate kept as a plain vector."""
+    values = _vp()
+    _check(load().deco_get_aggregate_vector(ctx, step, ctypes.byref(values)),
+           "deco_get_aggregate_vector")
+    return values.value
+
+
 def deco_get_select_info(ctx, n, stream=None):
     """-> (threshold_key[n], n_greater[n], exact_passes[n]) as Python lists."""
     thr, gt, ex = (_u32 * n)(), (_u32 * n)(), (_u32 * n)()
@@ -402,29 +410,27 @@ def deco_launch_count(ctx):
 
 
 def deco_get_exchange(ctx):
-    """Buffers a worker-sharded job all-gathers between compress and aggregate."""
-    m, mr, dd, dr = _vp(), _u64(), _vp(), _u64()
+    """The exchange buffer of a worker-sharded context: what the job all-gathers between
+    compress and aggregate."""
+    rows, rw = _vp(), _u64()
     r0, rl, rt = _u32(), _u32(), _u32()
-    _check(load().deco_get_exchange(ctx, ctypes.byref(m), ctypes.byref(mr), ctypes.byref(dd),
-                                    ctypes.byref(dr), ctypes.byref(r0), ctypes.byref(rl),
-                                    ctypes.byref(rt)), "deco_get_exchange")
-    return {"msg_all": m.value, "msg_row_pairs": mr.value, "dir_all": dd.value,
-            "dir_row_words": dr.value, "row0": r0.value, "rows_local": rl.value,
+    _check(load().deco_get_exchange(ctx, ctypes.byref(rows), ctypes.byref(rw), ctypes.byref(r0),
+                                    ctypes.byref(rl), ctypes.byref(rt)), "deco_get_exchange")
+    return {"rows": rows.value, "row_words": rw.value, "row0": r0.value, "rows_local": rl.value,
             "rows_total": rt.value}
 
 
-def exchange_views(ctx, device=0):
-    """torch views of the two exchange buffers: ([n_total, k_cap, 2] int32, [n_total, tiles+1]
-    int32), for torch.distributed collectives or plain copies."""
+def exchange_view(ctx, device=0):
+    """torch view [rows_total, row_words] int32 of the exchange buffer at the current k (rows
+    back to back: contiguous), for one torch.distributed collective or plain copies."""
     x = deco_get_exchange(ctx)
-    msg = view_i32(x["msg_all"], (x["rows_total"], x["msg_row_pairs"], 2), device)
-    dirs = view_i32(x["dir_all"], (x["rows_total"], x["dir_row_words"]), device)
-    return msg, dirs, x
+    return view_i32(x["rows"], (x["rows_total"], x["row_words"]), device), x
 
 
 def all_gather_rows(full, row0, rows_local, group=None):
-    """In-place all-gather of a row-sharded tensor: this rank owns rows [row0, row0+rows_local)
-    of `full`, every rank the same number, in rank order.  Plumbing (torch.distributed)."""
+    """In-place all-gather of a row-sharded contiguous tensor: this rank owns rows
+    [row0, row0 + rows_local) of `full`, every rank the same number, in rank order.  One
+    collective.  Plumbing (torch.distributed)."""
     import torch.distributed as dist
     mine = full[row0:row0 + rows_local]
     dist.all_gather_into_tensor(full, mine, group=group)
@@ -432,14 +438,14 @@ def all_gather_rows(full, row0, rows_local, group=None):
 
 def deco_step_sharded(ctx, grads, group=None, stream=None, device=0):
     """One iteration of a worker-sharded context: compress the local workers, all-gather the
-    sparse messages and their tile directories among the ranks of `group` (NCCL on GPUs: the
-    collectives run on torch's current stream, which must be `stream`), aggregate, update."""
+    exchange rows (k pairs and the tile directory of every worker) among the ranks of `group`
+    with one collective (NCCL on GPUs: it runs on torch's current stream, which must be
+    `stream`), aggregate, update."""
     deco_ef_compress(ctx, grads, stream)
-    msg, dirs, x = exchange_views(ctx, device)
+    rows, x = exchange_view(ctx, device)
     import torch.distributed as dist
     if dist.is_available() and dist.is_initialized():
-        all_gather_rows(msg, x["row0"], x["rows_local"], group)
-        all_gather_rows(dirs, x["row0"], x["rows_local"], group)
+        all_gather_rows(rows, x["row0"], x["rows_local"], group)
     elif x["rows_total"] != x["rows_local"]:
         raise RuntimeError("a worker-sharded context needs an initialised process group")
     deco_aggregate_stale(ctx, stream)

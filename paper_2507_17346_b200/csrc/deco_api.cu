@@ -43,8 +43,10 @@ void free_all(deco_ctx *c)
     cudaFree(c->e);
     if (c->own_params) cudaFree(c->params);
     cudaFree(c->msg);
+    cudaFree(c->xchg);
     cudaFree(c->slots);
     cudaFree(c->stage);
+    cudaFree(c->band);
     cudaFree(c->work);
     cudaFree(c->hist);
     cudaFree(c->sel);
@@ -87,7 +89,8 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
     if (err == cudaSuccess)
         err = cudaMemsetAsync(c->sample_hist, 0, sizeof(uint32_t) * c->n * SAMPLE_BINS, s);
     if (err == cudaSuccess)
-        err = cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n_total * (c->ntiles + 1), s);
+        err = c->packed ? cudaMemsetAsync(c->xchg, 0, sizeof(uint32_t) * c->n_total * c->xrow_cap, s)
+                        : cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n * (c->ntiles + 1), s);
     c->launches += 5;
     c->t = 0;
     c->phase = 0;
@@ -223,9 +226,25 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
         need(dev_alloc(c, &c->params, d));
         c->own_params = (st == DECO_OK);
     }
-    need(dev_alloc(c, &c->msg, static_cast<uint64_t>(c->n_total) * c->k_cap));
-    need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * c->n_total * c->k_cap));
+    c->packed = o.n_total != 0;
+    if (c->packed) {
+        c->xrow_cap = exchange_row_words(c, c->k_cap);
+        need(dev_alloc(c, &c->xchg, static_cast<uint64_t>(c->n_total) * c->xrow_cap));
+    } else {
+        need(dev_alloc(c, &c->msg, static_cast<uint64_t>(n) * c->k_cap));
+    }
+    // a cache slot holds the n_total * k_cap pairs of a merged aggregate; where the messages can
+    // be dense enough for the plain vector S[e_stride] to be the better layout, it has room for
+    // that too (a context that is one layer of a layered one keeps the pair layout only)
+    c->slot_pairs = static_cast<uint64_t>(c->n_total) * c->k_cap;
+    c->dense_capable = g_stride == 0 && c->slot_pairs * 4 >= d;
+    if (c->dense_capable) {
+        if (c->slot_pairs < c->e_stride / 2) c->slot_pairs = c->e_stride / 2;
+        c->slot_pairs = (c->slot_pairs + 31) & ~31ull;  // vectors start on 256-byte boundaries
+    }
+    need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * c->slot_pairs));
     need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
+    need(dev_alloc(c, &c->band, static_cast<uint64_t>(n) * c->stage_cap));
     // slices of 256 staged entries, plus one partial slice for every tile that has any
     c->work_cap = c->stage_cap / 256 + (c->stage_cap / 17 < c->ntiles ? c->stage_cap / 17 : c->ntiles) + 32;
     need(dev_alloc(c, &c->work, static_cast<uint64_t>(n) * c->work_cap));
@@ -237,7 +256,8 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     need(dev_alloc(c, &c->tile_gt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_eq, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_take, static_cast<uint64_t>(n) * c->ntiles));
-    need(dev_alloc(c, &c->tile_start, static_cast<uint64_t>(c->n_total) * (c->ntiles + 1)));
+    if (!c->packed) need(dev_alloc(c, &c->tile_start, static_cast<uint64_t>(n) * (c->ntiles + 1)));
+    set_message_layout(c, c->k);
     need(dev_alloc(c, &c->tile_off, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_cnt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_rej, static_cast<uint64_t>(n) * c->ntiles));
@@ -295,6 +315,7 @@ extern "C" deco_status deco_ef_compress(deco_ctx *c, const void *grads, void *st
     if (!guard.ok) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);
     c->k_of_msg = c->k;
+    set_message_layout(c, c->k);
     cudaError_t err = launch_begin_step(c, grads, s);
     mark(c, 0, s);
     if (err == cudaSuccess) err = launch_accumulate(c, grads, s);
@@ -315,13 +336,17 @@ extern "C" deco_status deco_aggregate_stale(deco_ctx *c, void *stream)
     const uint32_t si = static_cast<uint32_t>(c->t % c->ring);
     Slot &sl = c->slot_info[si];
     if (sl.valid) return DECO_ERR_STATE;    // cannot happen while tau <= tau_max
-    deco_pair *slot = c->slots + static_cast<uint64_t>(si) * c->n_total * c->k_cap;
+    deco_pair *slot = c->slots + static_cast<uint64_t>(si) * c->slot_pairs;
+    const bool dense = aggregate_as_vector(c, c->k_of_msg);
     if (wait_for_aggregate(c, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
     mark(c, 3, as_stream(stream));
-    if (launch_aggregate(c, slot, as_stream(stream)) != cudaSuccess) return DECO_ERR_CUDA;
+    const cudaError_t err = dense ? launch_aggregate_dense(c, reinterpret_cast<float *>(slot), as_stream(stream))
+                                  : launch_aggregate(c, slot, as_stream(stream));
+    if (err != cudaSuccess) return DECO_ERR_CUDA;
     mark(c, 4, as_stream(stream));
     sl.step = c->t;
-    sl.positions = static_cast<uint64_t>(c->n_total) * c->k_of_msg;
+    sl.positions = dense ? c->d : static_cast<uint64_t>(c->n_total) * c->k_of_msg;
+    sl.dense = dense;
     sl.valid = true;
     c->phase = 2;
     return DECO_OK;
@@ -342,8 +367,10 @@ deco_status apply_due(deco_ctx *c, cudaStream_t s)
     for (uint64_t step = lo; step <= due; ++step) {
         Slot &sl = c->slot_info[step % c->ring];
         if (!sl.valid || sl.step != step) continue;
-        const deco_pair *slot = c->slots + (step % c->ring) * c->n_total * c->k_cap;
-        if (launch_apply(c, slot, sl.positions, neg_scale, s) != cudaSuccess) return DECO_ERR_CUDA;
+        const deco_pair *slot = c->slots + (step % c->ring) * c->slot_pairs;
+        const cudaError_t err = sl.dense ? launch_apply_dense(c, reinterpret_cast<const float *>(slot), neg_scale, s)
+                                         : launch_apply(c, slot, sl.positions, neg_scale, s);
+        if (err != cudaSuccess) return DECO_ERR_CUDA;
         sl.valid = false;
     }
     return DECO_OK;
@@ -373,6 +400,7 @@ uint32_t deco::advance_iteration_external(deco_ctx *c, std::vector<uint32_t> *du
     Slot &now = c->slot_info[si];
     now.step = c->t;
     now.positions = static_cast<uint64_t>(c->n_total) * c->k;
+    now.dense = false;
     now.valid = true;
     if (c->t >= c->tau) {
         const uint64_t last = c->t - c->tau;
@@ -520,8 +548,8 @@ extern "C" deco_status deco_step_host(deco_ctx *c, const void *grads_host, deco_
     if (msg_out) {
         // rows of k pairs, packed: [n][k]
         if (cudaMemcpy2DAsync(msg_out, c->k_of_msg * sizeof(deco_pair),
-                              c->msg + static_cast<uint64_t>(c->worker_base) * c->k_cap,
-                              c->k_cap * sizeof(deco_pair), c->k_of_msg * sizeof(deco_pair), c->n,
+                              c->msg_rows + static_cast<uint64_t>(c->worker_base) * c->msg_stride,
+                              c->msg_stride * sizeof(deco_pair), c->k_of_msg * sizeof(deco_pair), c->n,
                               cudaMemcpyDeviceToHost, s) != cudaSuccess)
             return DECO_ERR_CUDA;
         c->launches += 1;
@@ -568,8 +596,8 @@ extern "C" deco_status deco_get_buffers(deco_ctx *c, float **e, uint64_t *e_stri
     if (!c) return DECO_ERR_INVALID_ARG;
     if (e) *e = c->e;
     if (e_stride) *e_stride = c->e_stride;
-    if (msg) *msg = c->msg + static_cast<uint64_t>(c->worker_base) * c->k_cap;   // the local rows
-    if (k_cap) *k_cap = c->k_cap;
+    if (msg) *msg = c->msg_rows + static_cast<uint64_t>(c->worker_base) * c->msg_stride;   // the local rows
+    if (k_cap) *k_cap = c->msg_stride;
     if (params) *params = c->params;
     return DECO_OK;
 }
@@ -579,13 +607,26 @@ extern "C" deco_status deco_get_aggregate(deco_ctx *c, uint64_t step, const deco
 {
     if (!c || !entries || !positions) return DECO_ERR_INVALID_ARG;
     const Slot &sl = c->slot_info[step % c->ring];
-    if (!sl.valid || sl.step != step) return DECO_ERR_STATE;
+    if (!sl.valid || sl.step != step || sl.dense) return DECO_ERR_STATE;
     {
         DeviceGuard guard(c->device);
         if (!guard.ok || drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
     }
-    *entries = c->slots + (step % c->ring) * c->n_total * c->k_cap;
+    *entries = c->slots + (step % c->ring) * c->slot_pairs;
     *positions = sl.positions;
+    return DECO_OK;
+}
+
+extern "C" deco_status deco_get_aggregate_vector(deco_ctx *c, uint64_t step, const float **values)
+{
+    if (!c || !values) return DECO_ERR_INVALID_ARG;
+    const Slot &sl = c->slot_info[step % c->ring];
+    if (!sl.valid || sl.step != step || !sl.dense) return DECO_ERR_STATE;
+    {
+        DeviceGuard guard(c->device);
+        if (!guard.ok || drain_internal(c) != cudaSuccess) return DECO_ERR_CUDA;
+    }
+    *values = reinterpret_cast<const float *>(c->slots + (step % c->ring) * c->slot_pairs);
     return DECO_OK;
 }
 
@@ -646,15 +687,13 @@ extern "C" deco_status deco_get_stats(deco_ctx *c, void *stream, deco_stats *out
     return DECO_OK;
 }
 
-extern "C" deco_status deco_get_exchange(deco_ctx *c, deco_pair **msg_all, uint64_t *msg_row_pairs,
-                                         uint32_t **dir_all, uint64_t *dir_row_words,
-                                         uint32_t *row0, uint32_t *rows_local, uint32_t *rows_total)
+extern "C" deco_status deco_get_exchange(deco_ctx *c, uint32_t **rows, uint64_t *row_words, uint32_t *row0,
+                                         uint32_t *rows_local, uint32_t *rows_total)
 {
     if (!c) return DECO_ERR_INVALID_ARG;
-    if (msg_all) *msg_all = c->msg;
-    if (msg_row_pairs) *msg_row_pairs = c->k_cap;
-    if (dir_all) *dir_all = c->tile_start;
-    if (dir_row_words) *dir_row_words = static_cast<uint64_t>(c->ntiles) + 1;
+    if (!c->packed) return DECO_ERR_STATE;
+    if (rows) *rows = c->xchg;
+    if (row_words) *row_words = exchange_row_words(c, c->phase == 0 ? c->k : c->k_of_msg);
     if (row0) *row0 = c->worker_base;
     if (rows_local) *rows_local = c->n;
     if (rows_total) *rows_total = c->n_total;
@@ -681,12 +720,18 @@ struct SlotRecord {
     uint64_t step, positions, valid;
 };
 
+// bytes a cached aggregate takes in the blob: its pairs, or the d values of a dense one
+uint64_t slot_bytes(const Slot &sl)
+{
+    return sl.dense ? sizeof(float) * sl.positions : sizeof(deco_pair) * sl.positions;
+}
+
 uint64_t state_size(const deco_ctx *c)
 {
     uint64_t bytes = sizeof(StateHeader) + sizeof(SlotRecord) * c->ring;
     bytes += sizeof(float) * c->n * c->d + sizeof(float) * c->d;
     for (const Slot &sl : c->slot_info)
-        if (sl.valid) bytes += sizeof(deco_pair) * sl.positions;
+        if (sl.valid) bytes += slot_bytes(sl);
     return bytes;
 }
 
@@ -722,7 +767,7 @@ extern "C" deco_status deco_export_state(deco_ctx *c, void *buf, uint64_t bytes,
     std::memcpy(out, &h, sizeof h);
     out += sizeof h;
     for (const Slot &sl : c->slot_info) {
-        SlotRecord r = {sl.step, sl.positions, sl.valid ? 1ull : 0ull};
+        SlotRecord r = {sl.step, sl.positions, sl.valid ? (sl.dense ? 2ull : 1ull) : 0ull};
         std::memcpy(out, &r, sizeof r);
         out += sizeof r;
     }
@@ -737,10 +782,10 @@ extern "C" deco_status deco_export_state(deco_ctx *c, void *buf, uint64_t bytes,
     for (uint32_t q = 0; q < c->ring; ++q) {
         const Slot &sl = c->slot_info[q];
         if (!sl.valid) continue;
-        if (cudaMemcpyAsync(out, c->slots + static_cast<uint64_t>(q) * c->n_total * c->k_cap,
-                            sizeof(deco_pair) * sl.positions, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        if (cudaMemcpyAsync(out, c->slots + static_cast<uint64_t>(q) * c->slot_pairs, slot_bytes(sl),
+                            cudaMemcpyDeviceToHost, s) != cudaSuccess)
             return DECO_ERR_CUDA;
-        out += sizeof(deco_pair) * sl.positions;
+        out += slot_bytes(sl);
     }
     c->launches += 2 + c->ring;
     return cudaStreamSynchronize(s) == cudaSuccess ? DECO_OK : DECO_ERR_CUDA;
@@ -774,14 +819,18 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
         in += sizeof r;
         // a cached aggregate was sent in one of the last `ring` iterations before t and holds
         // the same number of positions for every worker
-        if (r.valid && (r.positions > static_cast<uint64_t>(c->n_total) * c->k_cap ||
-                        r.positions < c->n_total || r.positions % c->n_total != 0 ||
-                        r.step % c->ring != q || r.step >= h.t || r.step + c->ring < h.t))
+        if (r.valid > 2) return DECO_ERR_INVALID_ARG;
+        if (r.valid && (r.step % c->ring != q || r.step >= h.t || r.step + c->ring < h.t))
             return DECO_ERR_INVALID_ARG;
+        if (r.valid == 1 && (r.positions > static_cast<uint64_t>(c->n_total) * c->k_cap ||
+                             r.positions < c->n_total || r.positions % c->n_total != 0))
+            return DECO_ERR_INVALID_ARG;
+        if (r.valid == 2 && (!c->dense_capable || r.positions != c->d)) return DECO_ERR_INVALID_ARG;
         slots[q].step = r.step;
         slots[q].positions = r.positions;
         slots[q].valid = r.valid != 0;
-        if (slots[q].valid) need += sizeof(deco_pair) * r.positions;
+        slots[q].dense = r.valid == 2;
+        if (slots[q].valid) need += slot_bytes(slots[q]);
     }
     if (bytes < need) return DECO_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
@@ -799,14 +848,16 @@ extern "C" deco_status deco_import_state(deco_ctx *c, const void *buf, uint64_t 
     in += sizeof(float) * c->d;
     for (uint32_t q = 0; q < c->ring; ++q) {
         if (!slots[q].valid) continue;
-        if (cudaMemcpyAsync(c->slots + static_cast<uint64_t>(q) * c->n_total * c->k_cap, in,
-                            sizeof(deco_pair) * slots[q].positions, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        if (cudaMemcpyAsync(c->slots + static_cast<uint64_t>(q) * c->slot_pairs, in, slot_bytes(slots[q]),
+                            cudaMemcpyHostToDevice, s) != cudaSuccess)
             return DECO_ERR_CUDA;
-        in += sizeof(deco_pair) * slots[q].positions;
+        in += slot_bytes(slots[q]);
+        // the padding of a dense vector (entries d .. e_stride) is never read
     }
     c->slot_info = slots;
     c->t = h.t;
     c->k = h.k;
+    set_message_layout(c, c->k);
     c->delta = h.delta;
     c->tau = h.tau;
     c->lr = h.lr;

@@ -99,14 +99,17 @@ struct Sel {
     uint32_t *chunk_cnt, *chunk_rej, *chunk_eq;   // [n][nchunks] staged / rejected / ties
     uint32_t *chunk_eqb;     // [n][nchunks] ties in earlier chunks
     uint32_t *chunk_start;   // [n][nchunks + 1] message position of each chunk
-    deco_pair *msg;
+    deco_pair *msg;          // first local worker's message; rows k_cap pairs apart
     uint64_t k_cap;
-    deco_pair *stage;
+    uint64_t dir_stride;     // words between the workers' rows of tile_start
+    deco_pair *stage;        // [n][stage_cap] candidates, each tile's in index order
+    deco_pair *band;         // [n][stage_cap] the candidates below cert_key, unordered
     uint64_t stage_cap;
     uint2 *work;             // [n][work_cap] (tile, slice) entries of the emit work list
     uint64_t work_cap;
     uint32_t *status;        // [0] latched status, [1..2] detail, [3] "some worker needs the multi-pass route"
     RandParams rk;
+    uint32_t use_band;       // the streaming pass writes the band list (dense messages only)
     uint32_t sample_shift;   // sample histogram bin = key >> sample_shift
     uint32_t bound_low_bit;  // lowest key bit the bound is refined to
 };
@@ -124,6 +127,24 @@ __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t 
         status[1] = a;
         status[2] = b;
     }
+}
+
+// What the streaming pass staged for a worker, read through L2 (another CTA of the same launch
+// may have written the record): candidates in all, and those inside the band.
+__device__ __forceinline__ void staged_counts(const SelectState &s, uint32_t &n_staged, uint32_t &n_band)
+{
+    const unsigned long long v = __ldcg(&s.staged_band);
+    n_staged = static_cast<uint32_t>(v);
+    n_band = static_cast<uint32_t>(v >> 32);
+}
+
+// The list the selection kernels read for worker i and its length: the band list, or (when the
+// streaming pass does not write one) all staged candidates.
+__device__ __forceinline__ const deco_pair *select_list(const Sel &p, uint32_t i, uint32_t n_staged,
+                                                        uint32_t &n_band)
+{
+    if (!p.use_band) n_band = n_staged;
+    return (p.use_band ? p.band : p.stage) + static_cast<size_t>(i) * p.stage_cap;
 }
 
 __device__ __forceinline__ uint32_t *hist_of(const Sel &p, uint32_t i, int route, int level)
@@ -168,6 +189,44 @@ __device__ __forceinline__ void ordered_prefix(const uint32_t (&cnt)[U], uint32_
 #pragma unroll
     for (int u = 0; u < U; ++u) pos[u] += before;
     block_total = total;
+    __syncthreads();
+}
+
+// ordered_prefix plus, for a second per-thread count nb, positions that are unique inside the
+// CTA (in thread order) and the CTA's total.  s_w and s_b are WARPS words each.
+template <int U>
+__device__ __forceinline__ void ordered_prefix2(const uint32_t (&m)[U], uint32_t (&pos)[U], uint32_t nb,
+                                                uint32_t &bpos, uint32_t *s_w, uint32_t *s_b,
+                                                uint32_t &block_total, uint32_t &band_total)
+{
+    // m[u]: the low byte marks the thread's entries of round u that count
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint32_t run = 0;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t c = __popc(m[u] & 0xFFu);
+        const uint32_t incl = warp_incl_scan(c);
+        pos[u] = run + incl - c;
+        run += __shfl_sync(FULL, incl, 31);
+    }
+    const uint32_t bincl = warp_incl_scan(nb);
+    if (lane == 0) s_w[w] = run;
+    if (lane == 31) s_b[w] = bincl;
+    __syncthreads();
+    uint32_t before = 0, total = 0, bbefore = 0, btotal = 0;
+#pragma unroll
+    for (int ww = 0; ww < WARPS; ++ww) {
+        const uint32_t v = s_w[ww], vb = s_b[ww];
+        before += (ww < w) ? v : 0u;
+        total += v;
+        bbefore += (ww < w) ? vb : 0u;
+        btotal += vb;
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) pos[u] += before;
+    bpos = bbefore + bincl - nb;
+    block_total = total;
+    band_total = btotal;
     __syncthreads();
 }
 
@@ -375,7 +434,8 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
             s.ties_take = 0;
             s.exact = exact_all;
             s.spec_key = SPEC_DISABLED;
-            s.n_staged = 0;
+            s.cert_key = SPEC_DISABLED;
+            s.staged_band = 0;
             s.rel_shift = 12;
             if (exact_all) s.exact_total += 1;
         }
@@ -387,6 +447,7 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
     __shared__ uint32_t s_cnt[NW];
     __shared__ uint32_t s_w[33];
     __shared__ uint32_t s_flag;
+    __shared__ uint32_t s_hi;
     const float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     const char *grow = reinterpret_cast<const char *>(grads) +
                        static_cast<size_t>(i) * p.g_stride * (GT ? 2 : 4);
@@ -453,6 +514,7 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
     // rank inside the sample: mean + 5 sigma + 2 of a binomial with p = k/d (exact when the
     // sample is the whole vector)
     uint32_t R;
+    uint32_t R_hi = 0;          // sample rank of the certainty bound: mean - 5 sigma - 2, if there is one
     uint32_t rel_shift = 10;
     if (m_total >= p.d) {
         R = p.k;
@@ -460,6 +522,8 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         const double mean = static_cast<double>(p.k) * m_total / static_cast<double>(p.d);
         const double r = mean + 5.0 * sqrt(mean) + 2.0;
         R = r >= static_cast<double>(m_total) ? m_total + 1u : static_cast<uint32_t>(r) + 1u;
+        const double rh = mean - 5.0 * sqrt(mean) - 2.0;
+        R_hi = (p.use_band && rh >= 1.0) ? static_cast<uint32_t>(rh) : 0u;
         // how far the sampled rank sits above k/d decides how far above the bound the
         // threshold may lie (in value: that ratio to the power 1/tail-index)
         const double rho = static_cast<double>(R) / (mean > 1e-9 ? mean : 1e-9);
@@ -492,14 +556,20 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         if (t == 0) {
             s_flag = 0;
             s_cnt[0] = 0;
+            s_hi = SPEC_DISABLED;
         }
         __syncthreads();
 #pragma unroll
         for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) {
+            const uint32_t hb = SAMPLE_HIST_BINS - 1 - (t * SAMPLE_BINS_PER_THREAD + c);
             if (higher < R && higher + cnt[c] >= R) {
-                s_flag = (SAMPLE_HIST_BINS - 1 - (t * SAMPLE_BINS_PER_THREAD + c)) << p.sample_shift;
+                s_flag = hb << p.sample_shift;
                 s_cnt[0] = higher;
             }
+            // certainty bound: upper edge of the bin that holds the sample key of rank R_hi, so
+            // that fewer than R_hi sample keys reach it (the edge above the top bin is beyond
+            // every key: nothing is certain then)
+            if (R_hi && higher < R_hi && higher + cnt[c] >= R_hi) s_hi = (hb + 1u) << p.sample_shift;
             higher += cnt[c];
         }
         __syncthreads();
@@ -595,6 +665,7 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
     }
     if (t == 0) {
         s.spec_key = bound;                    // lower edge of a 2^bound_low_bit-wide key bin
+        s.cert_key = s_hi;                     // above the bound's own histogram bin
         s.rel_shift = rel_shift;
     }
 }
@@ -612,12 +683,12 @@ begin_step_kernel(Sel p, const void *__restrict__ grads, float alpha, uint32_t e
 // otherwise (and in the tile that holds the end of the vector) gradients are read entry by
 // entry.  SPEC: stage the entries whose key reaches sel[i].spec_key.
 // ------------------------------------------------------------------------------------------
-template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
+template <int GT, bool ALIGNED, bool SPEC, bool RANDK, bool BAND>
 __device__ __forceinline__ void
 ef_accumulate_body(const uint32_t tile, const uint32_t i, const bool rows_aligned,
                    float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
                    uint64_t d, uint64_t g_stride, float alpha, const RandParams &rk, SelectState *__restrict__ sel,
-                   deco_pair *__restrict__ stage, uint64_t stage_cap,
+                   deco_pair *__restrict__ stage, deco_pair *__restrict__ band, uint64_t stage_cap,
                    uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
                    uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
                    uint32_t ntiles)
@@ -705,11 +776,15 @@ ef_accumulate_body(const uint32_t tile, const uint32_t i, const bool rows_aligne
     // segment reserved with one atomic per tile.  Staged entries are written to e as +0 (the
     // guess is that they are selected); the selection kernels write the value back for the
     // few that are not.  The store is issued before any barrier; a tile whose segment turns
-    // out not to fit stores its values again.
-    __shared__ uint32_t s_w[WARPS];
-    __shared__ uint32_t s_off;
+    // out not to fit stores its values again.  With BAND the staged entries below the
+    // certainty bound (the band: only among them can the threshold lie) are written once more,
+    // in any order, to the band list, which is then all the selection kernels have to read.
+    __shared__ uint32_t s_w[WARPS], s_b[WARPS];
+    __shared__ uint32_t s_off, s_boff;
     const uint32_t bound = sel[i].spec_key;
-    uint32_t m[U], cnt[U], pos[U], any = 0;
+    const uint32_t cert = BAND ? sel[i].cert_key : SPEC_DISABLED;
+    // m[u]: bit c = entry c of round u is staged, bit 8 + c = and lies in the band
+    uint32_t m[U], pos[U], any = 0, nb = 0;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint64_t j = wbase + u * (32 * V) + lane * V;
@@ -727,32 +802,55 @@ ef_accumulate_body(const uint32_t tile, const uint32_t i, const bool rows_aligne
         }
 #pragma unroll
         for (int c = 0; c < V; ++c)
-            if (keys[c] >= bound && (full || j + c < d)) m[u] |= 1u << c;
-        cnt[u] = __popc(m[u]);
+            if (keys[c] >= bound && (full || j + c < d))
+                m[u] |= ((BAND && keys[c] < cert) ? 0x101u : 0x1u) << c;
+        if (BAND) nb += __popc(m[u] >> 8);
         any |= m[u];
     }
     store_tile(m);
-    uint32_t total = 0;
+    uint32_t total = 0, band_total = 0, bpos = 0;
     if (__syncthreads_or(any != 0)) {
-        ordered_prefix<U>(cnt, pos, s_w, total);
+        if (BAND) {
+            ordered_prefix2<U>(m, pos, nb, bpos, s_w, s_b, total, band_total);
+        } else {
+            uint32_t cnt[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) cnt[u] = __popc(m[u]);
+            ordered_prefix<U>(cnt, pos, s_w, total);
+        }
     }
     if (threadIdx.x == 0) {
-        uint32_t off = 0;
-        if (total) off = atomicAdd(&sel[i].n_staged, total);
+        uint32_t off = 0, boff = 0;
+        if (total) {
+            if (BAND) {
+                const unsigned long long old = atomicAdd(
+                    &sel[i].staged_band, static_cast<unsigned long long>(total) |
+                                             (static_cast<unsigned long long>(band_total) << 32));
+                off = static_cast<uint32_t>(old);
+                boff = static_cast<uint32_t>(old >> 32);
+            } else {
+                // the low word alone (little-endian): the candidate count
+                off = atomicAdd(reinterpret_cast<uint32_t *>(&sel[i].staged_band), total);
+            }
+        }
         tile_off[static_cast<size_t>(i) * ntiles + tile] = off;
         tile_cnt[static_cast<size_t>(i) * ntiles + tile] = total;
         tile_rej[static_cast<size_t>(i) * ntiles + tile] = 0;
         tile_eq[static_cast<size_t>(i) * ntiles + tile] = 0;
         s_off = off;
+        if (BAND) s_boff = boff;
     }
     if (total == 0) return;
     __syncthreads();
     const uint64_t off = s_off;
-    if (off + total > stage_cap) {                   // overflow: n_staged tells the selector,
+    if (off + total > stage_cap) {                   // overflow: the counts tell the selector,
         store_tile(nullptr);                         // and this tile takes its values back
         return;
     }
+    // band entries are a subset of the staged ones and both offsets grow in the same atomic,
+    // so the band segment fits whenever the staged segment does
     deco_pair *out = stage + static_cast<size_t>(i) * stage_cap + off;
+    deco_pair *bout = BAND ? band + static_cast<size_t>(i) * stage_cap + s_boff + bpos : nullptr;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint64_t j = wbase + u * (32 * V) + lane * V;
@@ -764,21 +862,22 @@ ef_accumulate_body(const uint32_t tile, const uint32_t i, const bool rows_aligne
                 pr.idx = static_cast<uint32_t>(j + c);
                 pr.val = x[u][c];
                 out[q++] = pr;
+                if (BAND && (m[u] & (0x100u << c))) *bout++ = pr;
             }
     }
 }
 
-template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
-__global__ void __launch_bounds__(BLOCK)
+template <int GT, bool ALIGNED, bool SPEC, bool RANDK, bool BAND>
+__global__ void __launch_bounds__(BLOCK, 3)
 ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
                      uint64_t d, uint64_t g_stride, float alpha, RandParams rk, SelectState *__restrict__ sel,
-                     deco_pair *__restrict__ stage, uint64_t stage_cap,
+                     deco_pair *__restrict__ stage, deco_pair *__restrict__ band, uint64_t stage_cap,
                      uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
                      uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
                      uint32_t ntiles)
 {
-    ef_accumulate_body<GT, ALIGNED, SPEC, RANDK>(blockIdx.x, blockIdx.y, true, e, e_stride, grads, d, g_stride,
-                                                 alpha, rk, sel, stage, stage_cap, tile_off, tile_cnt,
+    ef_accumulate_body<GT, ALIGNED, SPEC, RANDK, BAND>(blockIdx.x, blockIdx.y, true, e, e_stride, grads, d, g_stride,
+                                                 alpha, rk, sel, stage, band, stage_cap, tile_off, tile_cnt,
                                                  tile_rej, tile_eq, ntiles);
 }
 
@@ -842,25 +941,36 @@ __device__ __forceinline__ void build_emit_work(const Sel &p, uint32_t i)
 }
 
 
-// Level A: histogram of the coarse bins of all staged keys.  The last CTA of a worker to
-// arrive takes the decision: is the staged set usable (at least k entries, so it contains the
-// k largest, and no overflow of the staging area), and which coarse bin holds the k-th
-// largest.  If the set is not usable, or the threshold falls into the shared top bin, the
-// worker is handed to the multi-pass route.
-__device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i)
+// Shared memory of the selection bodies: one radix histogram and a few words.
+struct SelectShared {
+    uint32_t h[RADIX_BINS];
+    uint32_t scan[33];
+    uint32_t misc[3];
+    uint32_t warp[WARPS];
+    uint32_t out[2];
+};
+
+// Level A: histogram of the coarse bins of the band keys.  The last CTA of a worker to
+// arrive takes the decision: is the staged set usable (at least k candidates, so it contains
+// the k largest; no overflow of the staging area; fewer than k of them at or above the
+// certainty bound, so the threshold lies in the band), and which coarse bin holds the entry of
+// rank k - (candidates above the band).  If the set is not usable, or the threshold falls into
+// the shared top bin, the worker is handed to the multi-pass route.
+__device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i, SelectShared &sm)
 {
     SelectState &s = p.sel[i];
-    if (s.exact) return;
-    const uint32_t n_staged = s.n_staged, spec = s.spec_key, shift = s.rel_shift;
-    const bool valid = n_staged >= p.k && n_staged <= p.stage_cap;
-    __shared__ uint32_t h[RADIX_BINS];
-    __shared__ uint32_t s_scan[33];
-    __shared__ uint32_t s_misc[3];
+    if (__ldcg(&s.exact)) return;
+    uint32_t n_staged, n_band;
+    staged_counts(s, n_staged, n_band);
+    const deco_pair *src = select_list(p, i, n_staged, n_band);
+    const uint32_t n_cert = n_staged - n_band;
+    const uint32_t spec = __ldcg(&s.spec_key), shift = __ldcg(&s.rel_shift);
+    const bool valid = n_staged >= p.k && n_staged <= p.stage_cap && n_cert < p.k;
+    uint32_t *h = sm.h;
     if (valid) {
         for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
         __syncthreads();
-        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
-        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
              base += gridDim.x * (4 * BLOCK)) {
             deco_pair v[4];
 #pragma unroll
@@ -868,11 +978,11 @@ __device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i
                 const uint32_t q = base + r * BLOCK + threadIdx.x;
                 v[r].idx = 0;
                 v[r].val = 0.0f;
-                if (q < n_staged) v[r] = src[q];
+                if (q < n_band) v[r] = src[q];
             }
 #pragma unroll
             for (int r = 0; r < 4; ++r)
-                if (base + r * BLOCK + threadIdx.x < n_staged)
+                if (base + r * BLOCK + threadIdx.x < n_band)
                     atomicAdd(&h[rel_bin_a(key_of(p, i, v[r]), spec, shift)], 1u);
         }
         __syncthreads();
@@ -880,9 +990,9 @@ __device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i
         for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
             if (h[b]) atomicAdd(&out[b], h[b]);
     }
-    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 0], &s_misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 0], &sm.misc[2])) return;
     uint32_t a_sel = REL_TOP, above_a = 0;
-    if (valid) pick_bin(hist_of(p, i, 0, 0), p.k, s_scan, s_misc, a_sel, above_a);
+    if (valid) pick_bin(hist_of(p, i, 0, 0), p.k - n_cert, sm.scan, sm.misc, a_sel, above_a);
     if (threadIdx.x == 0) {
         if (!valid || a_sel >= REL_TOP) {
             s.exact = 1;
@@ -890,31 +1000,35 @@ __device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i
             p.status[3] = 1;
         } else {
             s.prefix = a_sel;
-            s.n_greater = above_a;
-            s.k_rem = p.k - above_a;
+            s.n_greater = n_cert + above_a;
+            s.k_rem = p.k - n_cert - above_a;
         }
     }
 }
 
-// Level B: histogram of the low bits of the staged keys that fell into the chosen A bin; the
-// last CTA of a worker to arrive fixes the threshold key and the number of ties to take.
-__global__ void __launch_bounds__(BLOCK) stage_hist_a_kernel(Sel p) { stage_hist_a_body(p, blockIdx.y); }
+__global__ void __launch_bounds__(BLOCK) stage_hist_a_kernel(Sel p)
+{
+    __shared__ SelectShared sm;
+    stage_hist_a_body(p, blockIdx.y, sm);
+}
 
-__device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i)
+// Level B: histogram of the low bits of the band keys that fell into the chosen A bin; the
+// last CTA of a worker to arrive fixes the threshold key and the number of ties to take.
+__device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i, SelectShared &sm)
 {
     SelectState &s = p.sel[i];
-    if (s.exact) return;
-    __shared__ uint32_t h[RADIX_BINS];
-    __shared__ uint32_t s_scan[33];
-    __shared__ uint32_t s_misc[3];
-    const uint32_t n_staged = s.n_staged, spec = s.spec_key, shift = s.rel_shift;
-    const uint32_t a_sel = s.prefix, above_a = s.n_greater, k_rem = s.k_rem;   // from level A
+    if (__ldcg(&s.exact)) return;
+    uint32_t *h = sm.h;
+    uint32_t n_staged, n_band;
+    staged_counts(s, n_staged, n_band);
+    const uint32_t spec = __ldcg(&s.spec_key), shift = __ldcg(&s.rel_shift);
+    const uint32_t a_sel = __ldcg(&s.prefix), above_a = __ldcg(&s.n_greater), k_rem = __ldcg(&s.k_rem);   // from level A
     const uint32_t low_mask = (1u << shift) - 1u;
-    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
+    const deco_pair *src = select_list(p, i, n_staged, n_band);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
     build_emit_work(p, i);                              // independent of the histogram
     __syncthreads();
-    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
          base += gridDim.x * (4 * BLOCK)) {
         deco_pair v[4];
 #pragma unroll
@@ -922,11 +1036,11 @@ __device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i
             const uint32_t q = base + r * BLOCK + threadIdx.x;
             v[r].idx = 0;
             v[r].val = 0.0f;
-            if (q < n_staged) v[r] = src[q];
+            if (q < n_band) v[r] = src[q];
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            if (base + r * BLOCK + threadIdx.x >= n_staged) continue;
+            if (base + r * BLOCK + threadIdx.x >= n_band) continue;
             const uint32_t key = key_of(p, i, v[r]);
             if (rel_bin_a(key, spec, shift) == a_sel) atomicAdd(&h[(key - spec) & low_mask], 1u);
         }
@@ -935,9 +1049,9 @@ __device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i
     uint32_t *out = hist_of(p, i, 0, 1);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
         if (h[b]) atomicAdd(&out[b], h[b]);
-    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 1], &s_misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 1], &sm.misc[2])) return;
     uint32_t bin, above;
-    pick_bin(hist_of(p, i, 0, 1), k_rem, s_scan, s_misc, bin, above);
+    pick_bin(hist_of(p, i, 0, 1), k_rem, sm.scan, sm.misc, bin, above);
     if (threadIdx.x == 0) {
         if (bin == 0xFFFFFFFFu) {                   // counts do not add up: report, stay safe
             latch(p.status, DECO_ERR_DEVICE_CHECK, 0x120u, i);
@@ -953,7 +1067,11 @@ __device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i
     }
 }
 
-__global__ void __launch_bounds__(BLOCK) stage_hist_b_kernel(Sel p) { stage_hist_b_body(p, blockIdx.y); }
+__global__ void __launch_bounds__(BLOCK) stage_hist_b_kernel(Sel p)
+{
+    __shared__ SelectShared sm;
+    stage_hist_b_body(p, blockIdx.y, sm);
+}
 
 // One CTA: ties are granted to chunks in index order until ties_take are used up, then every
 // chunk gets its position in the message.  Per thread a contiguous range of chunks.  With
@@ -969,7 +1087,7 @@ __device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, 
     const uint32_t *tcnt = p.tile_cnt + static_cast<size_t>(i) * p.ntiles;
     const uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     const uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
-    const uint32_t ties = p.sel[i].ties_take;
+    const uint32_t ties = __ldcg(&p.sel[i].ties_take);
     const uint32_t per = (p.nchunks + blockDim.x - 1) / blockDim.x;
     const uint32_t lo = min(p.nchunks, threadIdx.x * per), hi = min(p.nchunks, lo + per);
     uint32_t eq_sum = 0;
@@ -1019,22 +1137,20 @@ __device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, 
 }
 
 // Many chunks: their sums are taken in parallel, one warp per chunk (three coalesced loads
-// and a warp reduction), and the last CTA of a worker to arrive walks the chunks.
-__device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i)
+// and a warp reduction; the CTAs stride over the chunks), and the last CTA of a worker to
+// arrive walks the chunks.
+__device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i, SelectShared &sm)
 {
-    if (p.sel[i].exact) return;
-    __shared__ uint32_t s_scan[33];
-    __shared__ uint32_t s_flag;
+    if (__ldcg(&p.sel[i].exact)) return;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t chunk = blockIdx.x * WARPS + w;
-    if (chunk < p.nchunks) {
+    for (uint32_t chunk = blockIdx.x * WARPS + w; chunk < p.nchunks; chunk += gridDim.x * WARPS) {
         const uint32_t tile = chunk * CHUNK_TILES + lane;
         const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
         uint32_t a = 0, b = 0, q = 0;
         if (tile < p.ntiles) {
-            a = p.tile_cnt[ti];
-            b = p.tile_rej[ti];
-            q = p.tile_eq[ti];
+            a = __ldcg(&p.tile_cnt[ti]);
+            b = __ldcg(&p.tile_rej[ti]);
+            q = __ldcg(&p.tile_eq[ti]);
         }
         for (int o = 16; o > 0; o >>= 1) {
             a += __shfl_down_sync(FULL, a, o);
@@ -1047,30 +1163,36 @@ __device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i)
             p.chunk_eq[static_cast<size_t>(i) * p.nchunks + chunk] = q;
         }
     }
-    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 4], &s_flag)) return;
-    chunk_walk(p, i, s_scan, true);
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 4], &sm.misc[2])) return;
+    chunk_walk(p, i, sm.scan, true);
 }
 
-__global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p) { chunk_sums_body(p, blockIdx.y); }
+__global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p)
+{
+    __shared__ SelectShared sm;
+    chunk_sums_body(p, blockIdx.y, sm);
+}
 
-// Classification.  With the threshold known every staged entry below it is rejected: counted
-// for its tile and its chunk (CHUNK_TILES consecutive tiles) and given its value back in e;
-// entries equal to it are counted as ties.  With few chunks (walk_here) the last CTA of a worker
-// to arrive then walks the chunks once; with many, chunk_sums_kernel follows.  (The per-tile positions follow from these inside the
-// emit kernel, so nothing here is serial in the number of tiles.)
-__device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t i, uint32_t walk_here)
+// Classification.  With the threshold known every band entry below it is rejected: counted
+// for its tile and given its value back in e; entries equal to it are counted as ties.  (The
+// candidates above the band are above the threshold.)  With few chunks (walk_here) the last
+// CTA of a worker to arrive then walks the chunks once; with many, the chunk sums follow.
+// (The per-tile positions follow from these inside the emit step, so nothing here is serial
+// in the number of tiles.)
+__device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t i, uint32_t walk_here,
+                                                    SelectShared &sm)
 {
     const SelectState &s = p.sel[i];
-    if (s.exact) return;
-    __shared__ uint32_t s_scan[33];
-    __shared__ uint32_t s_flag;
-    const uint32_t n_staged = s.n_staged, T = s.threshold;
-    const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap;
+    if (__ldcg(&s.exact)) return;
+    uint32_t n_staged, n_band;
+    staged_counts(s, n_staged, n_band);
+    const uint32_t T = __ldcg(&s.threshold);
+    const deco_pair *src = select_list(p, i, n_staged, n_band);
     uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
     float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     const int lane = threadIdx.x & 31;
-    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
          base += gridDim.x * (4 * BLOCK)) {
         deco_pair prs[4];
 #pragma unroll
@@ -1078,13 +1200,13 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
             const uint32_t q = base + r * BLOCK + threadIdx.x;
             prs[r].idx = 0;
             prs[r].val = __uint_as_float(0x7FFFFFFFu);       // above any threshold: no action
-            if (q < n_staged) prs[r] = src[q];
+            if (q < n_band) prs[r] = src[q];
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            // neighbours in the staging area mostly belong to the same tile: lanes with the
+            // neighbours in the band list mostly belong to the same tile: lanes with the
             // same (tile, class) elect one of them to add the group's size
-            const bool in = base + r * BLOCK + threadIdx.x < n_staged;
+            const bool in = base + r * BLOCK + threadIdx.x < n_band;
             const uint32_t key = in ? key_of(p, i, prs[r]) : 0x7FFFFFFFu;
             const uint32_t tile = prs[r].idx / TILE;
             const uint32_t cls = !in ? 0u : (key < T ? 1u : (key == T ? 2u : 0u));
@@ -1093,17 +1215,17 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
                 atomicAdd(cls == 1 ? &rej[tile] : &eqc[tile], static_cast<uint32_t>(__popc(grp)));
         }
     }
-    const bool last = last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &s_flag);
+    const bool last = last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &sm.misc[2]);
     // after the arrival, off the critical path: undo the +0 guess for the rejected entries
     auto write_back_rejected = [&]() {
-        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_staged;
+        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
              base += gridDim.x * (4 * BLOCK)) {
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const uint32_t q = base + r * BLOCK + threadIdx.x;
-                if (q < n_staged) {
+                if (q < n_band) {
                     const deco_pair pr = src[q];
-                    if (key_of(p, i, pr) < T) erow[pr.idx] = pr.val;
+                    if (key_of(p, i, pr) < T && pr.idx < p.d) erow[pr.idx] = pr.val;
                 }
             }
         }
@@ -1112,13 +1234,14 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
         write_back_rejected();
         return;
     }
-    if (walk_here) chunk_walk(p, i, s_scan, false);
+    if (walk_here) chunk_walk(p, i, sm.scan, false);
     write_back_rejected();
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_classify_kernel(Sel p, uint32_t walk_here)
 {
-    stage_classify_body(p, blockIdx.y, walk_here);
+    __shared__ SelectShared sm;
+    stage_classify_body(p, blockIdx.y, walk_here, sm);
 }
 
 // What a warp learns about the CHUNK_TILES tiles of one chunk from three coalesced loads and
@@ -1139,12 +1262,12 @@ __device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint3
     uint32_t cnt = 0, rej = 0, eq = 0;
     if (tile < p.ntiles) {
         cnt = p.tile_cnt[ti];
-        rej = p.tile_rej[ti];
-        eq = p.tile_eq[ti];
+        rej = __ldcg(&p.tile_rej[ti]);
+        eq = __ldcg(&p.tile_eq[ti]);
     }
-    const uint32_t ties = p.sel[i].ties_take;
-    const uint32_t eqb0 = p.chunk_eqb[static_cast<size_t>(i) * p.nchunks + chunk];
-    const uint32_t start0 = p.chunk_start[static_cast<size_t>(i) * (p.nchunks + 1) + chunk];
+    const uint32_t ties = __ldcg(&p.sel[i].ties_take);
+    const uint32_t eqb0 = __ldcg(&p.chunk_eqb[static_cast<size_t>(i) * p.nchunks + chunk]);
+    const uint32_t start0 = __ldcg(&p.chunk_start[static_cast<size_t>(i) * (p.nchunks + 1) + chunk]);
     const uint32_t eq_before = eqb0 + warp_incl_scan(eq) - eq;
     const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
     TileInfo t;
@@ -1154,9 +1277,9 @@ __device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint3
     t.start = start0 + warp_incl_scan(t.sel) - t.sel;
     if (WRITE_DIR) {
         // the directory the aggregation reads: message position of every tile
-        if (tile < p.ntiles) p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile] = t.start;
+        if (tile < p.ntiles) p.tile_start[static_cast<size_t>(i) * p.dir_stride + tile] = t.start;
         if (tile == p.ntiles - 1)
-            p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + p.ntiles] = t.start + t.sel;
+            p.tile_start[static_cast<size_t>(i) * p.dir_stride + p.ntiles] = t.start + t.sel;
     }
     return t;
 }
@@ -1212,48 +1335,51 @@ __device__ __forceinline__ uint32_t emit_segment_warp(const Sel &p, uint32_t i, 
     return written;
 }
 
-// Emit.  CTAs [0, dir_ctas) of a worker: one warp per chunk of CHUNK_TILES tiles writes the
-// directory and each lane walks its own tile if that holds at most EMIT_LANE_MAX staged
-// entries.  The remaining CTAs: their warps stride over the work list; a warp that gets slice
-// j > 0 of a tile first counts, with independent loads, what the slices before it emit.
-__device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, uint32_t dir_ctas)
+// Emit, directory part: CTA `cta` of `nctas`; a warp per chunk of CHUNK_TILES tiles (the CTAs
+// stride over the chunks) writes the directory and each lane walks its own tile if that holds
+// at most EMIT_LANE_MAX staged entries.
+__device__ __forceinline__ void emit_directory_part(const Sel &p, const uint32_t i, uint32_t cta, uint32_t nctas)
 {
-    if (p.sel[i].exact) return;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t T = p.sel[i].threshold;
-    if (blockIdx.x < dir_ctas) {
-        // the directory CTAs stride over the chunks (one trip when there is a warp per chunk)
-        for (uint32_t chunk = blockIdx.x * WARPS + w; chunk < p.nchunks; chunk += dir_ctas * WARPS) {
-            const TileInfo t = chunk_header<true>(p, i, chunk);
-            const uint32_t tile = chunk * CHUNK_TILES + lane;
-            if (t.cnt == 0 || t.cnt > EMIT_LANE_MAX) continue;
-            const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
-            const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
-            deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
-            float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
-            uint32_t written = 0, ties_seen = 0;
-            for (uint32_t q = 0; q < t.cnt; ++q) {
-                const deco_pair pr = src[q];
-                const uint32_t key = key_of(p, i, pr);
-                const bool eq = key == T;
-                const bool pick = key > T || (eq && ties_seen < t.take);
-                ties_seen += eq ? 1u : 0u;
-                if (pick) {
-                    const uint32_t pos = t.start + written++;
-                    if (pos < p.k && pr.idx < p.d) out[pos] = pr;
-                    else latch(p.status, DECO_ERR_DEVICE_CHECK, 0x312u, tile);
-                } else if (eq && pr.idx < p.d) {
-                    erow[pr.idx] = pr.val;                       // tie not taken: undo the guess
-                }
+    const uint32_t T = __ldcg(&p.sel[i].threshold);
+    for (uint32_t chunk = cta * WARPS + w; chunk < p.nchunks; chunk += nctas * WARPS) {
+        const TileInfo t = chunk_header<true>(p, i, chunk);
+        const uint32_t tile = chunk * CHUNK_TILES + lane;
+        if (t.cnt == 0 || t.cnt > EMIT_LANE_MAX) continue;
+        const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
+        const deco_pair *src = p.stage + static_cast<size_t>(i) * p.stage_cap + off;
+        deco_pair *out = p.msg + static_cast<size_t>(i) * p.k_cap;
+        float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
+        uint32_t written = 0, ties_seen = 0;
+        for (uint32_t q = 0; q < t.cnt; ++q) {
+            const deco_pair pr = src[q];
+            const uint32_t key = key_of(p, i, pr);
+            const bool eq = key == T;
+            const bool pick = key > T || (eq && ties_seen < t.take);
+            ties_seen += eq ? 1u : 0u;
+            if (pick) {
+                const uint32_t pos = t.start + written++;
+                if (pos < p.k && pr.idx < p.d) out[pos] = pr;
+                else latch(p.status, DECO_ERR_DEVICE_CHECK, 0x312u, tile);
+            } else if (eq && pr.idx < p.d) {
+                erow[pr.idx] = pr.val;                       // tie not taken: undo the guess
             }
-            if (written != t.sel) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x313u, tile);
         }
-        return;
+        if (written != t.sel) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x313u, tile);
     }
-    const uint32_t n_items = min(p.done[i * DONE_SLOTS + 5], static_cast<uint32_t>(p.work_cap));
+}
+
+// Emit, work-list part: the warps of CTA `cta` of `nctas` stride over the work list; a warp
+// that gets slice j > 0 of a tile first counts, with independent loads, what the slices before
+// it emit.
+__device__ __forceinline__ void emit_items_part(const Sel &p, const uint32_t i, uint32_t cta, uint32_t nctas)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t T = __ldcg(&p.sel[i].threshold);
+    const uint32_t n_items = min(__ldcg(&p.done[i * DONE_SLOTS + 5]), static_cast<uint32_t>(p.work_cap));
     const uint2 *work = p.work + static_cast<size_t>(i) * p.work_cap;
-    const uint32_t warps = (gridDim.x - dir_ctas) * WARPS;
-    for (uint32_t q = (blockIdx.x - dir_ctas) * WARPS + w; q < n_items; q += warps) {
+    const uint32_t warps = nctas * WARPS;
+    for (uint32_t q = cta * WARPS + w; q < n_items; q += warps) {
         const uint2 item = work[q];
         const uint32_t tile = item.x, slice = item.y;
         if (tile >= p.ntiles) {
@@ -1299,6 +1425,15 @@ __device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, 
         if (end == cnt && lane == 0 && written != want)
             latch(p.status, DECO_ERR_DEVICE_CHECK, 0x311u, tile);
     }
+}
+
+// Emit as a launch of its own: CTAs [0, dir_ctas) of a worker do the directory part, the
+// remaining CTAs the work list.
+__device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, uint32_t dir_ctas)
+{
+    if (__ldcg(&p.sel[i].exact)) return;
+    if (blockIdx.x < dir_ctas) emit_directory_part(p, i, blockIdx.x, dir_ctas);
+    else emit_items_part(p, i, blockIdx.x - dir_ctas, gridDim.x - dir_ctas);
 }
 
 __global__ void __launch_bounds__(BLOCK) emit_stage_kernel(Sel p, uint32_t dir_ctas)
@@ -1401,7 +1536,7 @@ __device__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w /*[33]*/
     const uint32_t *eq = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
     auto gt = [&](uint32_t t) { return streaming ? cnt[t] - rej[t] - eq[t] : gtp[t]; };
     uint32_t *take = p.tile_take + static_cast<size_t>(i) * p.ntiles;
-    uint32_t *start = p.tile_start + static_cast<size_t>(i) * (p.ntiles + 1);
+    uint32_t *start = p.tile_start + static_cast<size_t>(i) * p.dir_stride;
     const uint32_t ties = p.sel[i].ties_take;
     const uint32_t per = (p.ntiles + nt - 1) / nt;
     const uint32_t lo = min(p.ntiles, threadIdx.x * per), hi = min(p.ntiles, lo + per);
@@ -1474,8 +1609,8 @@ __device__ __forceinline__ void emit_e_tile(const Sel &p, uint32_t i, uint32_t t
                                             uint32_t *s_w /*[WARPS]*/)
 {
     constexpr int V = 4, U = WARP_ELEMS / (32 * V);
-    const uint32_t start = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile];
-    const uint32_t count = p.tile_start[static_cast<size_t>(i) * (p.ntiles + 1) + tile + 1] - start;
+    const uint32_t start = p.tile_start[static_cast<size_t>(i) * p.dir_stride + tile];
+    const uint32_t count = p.tile_start[static_cast<size_t>(i) * p.dir_stride + tile + 1] - start;
     if (count == 0) return;
     const uint32_t T = p.sel[i].threshold;
     const uint32_t take = p.tile_take[static_cast<size_t>(i) * p.ntiles + tile];
@@ -1605,7 +1740,8 @@ __global__ void __launch_bounds__(BLOCK) emit_e_kernel(Sel p)
 __device__ __forceinline__ void exact_fallback_body(const Sel &p, cg::grid_group &grid, uint32_t *h,
                                                     uint32_t *s_a, uint32_t *s_b, uint32_t *s_out)
 {
-    const uint32_t cta = blockIdx.x, ncta = gridDim.x;
+    // CTAs numbered in a row, whatever the shape of the grid
+    const uint32_t cta = blockIdx.y * gridDim.x + blockIdx.x, ncta = gridDim.x * gridDim.y;
     // The streaming pass wrote +0 over the staged entries of every tile whose segment fitted;
     // the passes below need the values back.
     for (uint32_t i = 0; i < p.n; ++i) {
@@ -1673,6 +1809,37 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
     exact_fallback_body(p, grid, h, s_a, s_b, s_out);
 }
 
+// ---- the whole selection of the streaming route in one cooperative launch: level A, level B,
+// classification, chunk sums and walk, emit, each separated from the next by a grid-wide
+// barrier (where the separate kernels have a launch boundary), then the multi-pass route for
+// the workers whose staged set was rejected, if there are any.  Grid: x = CTAs of a worker,
+// y = worker; every body strides over its work by gridDim.x.  Which barriers a CTA takes depends
+// only on kernel arguments and on a flag that is final after the first barrier, so the whole
+// grid takes the same ones.
+__global__ void __launch_bounds__(BLOCK, 3) select_chain_kernel(Sel p, uint32_t walk_here)
+{
+    cg::grid_group grid = cg::this_grid();
+    __shared__ SelectShared sm;
+    const uint32_t i = blockIdx.y;
+    stage_hist_a_body(p, i, sm);
+    grid.sync();
+    stage_hist_b_body(p, i, sm);
+    grid.sync();
+    stage_classify_body(p, i, walk_here, sm);
+    grid.sync();
+    if (!walk_here) {
+        chunk_sums_body(p, i, sm);
+        grid.sync();
+    }
+    if (!__ldcg(&p.sel[i].exact)) {
+        emit_directory_part(p, i, blockIdx.x, gridDim.x);
+        emit_items_part(p, i, blockIdx.x, gridDim.x);
+    }
+    if (__ldcg(&p.status[3]) == 0) return;
+    __syncthreads();
+    exact_fallback_body(p, grid, sm.h, sm.scan, sm.warp, sm.out);
+}
+
 // ------------------------------------------------------------------------------------------
 // Many contexts in one launch (per-layer Top-k: one context per layer, all with n workers).
 // Row y of the grid is worker y % n of layer y / n; the layer's parameters come from a table
@@ -1715,7 +1882,7 @@ begin_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, const 
 constexpr int ACC_LAYERS_MAX = 256;
 struct AccLayer {
     float *e;
-    deco_pair *stage;
+    deco_pair *stage, *band;
     SelectState *sel;
     uint32_t *tile_off, *tile_cnt, *tile_rej, *tile_eq;
     uint64_t e_stride, stage_cap, d, g_off;
@@ -1748,28 +1915,31 @@ ef_accumulate_multi_kernel(const __grid_constant__ AccTable tab, const void *__r
     RandParams rk;
     rk.on = 0;
     rk.seed_lo = rk.seed_hi = rk.step_lo = rk.step_hi = rk.worker_base = 0;
-    ef_accumulate_body<GT, ALIGNED, true, false>(tile, blockIdx.y, true, m.e, m.e_stride, g,
-                                                 m.d, g_stride, alpha, rk, m.sel, m.stage, m.stage_cap,
+    ef_accumulate_body<GT, ALIGNED, true, false, false>(tile, blockIdx.y, true, m.e, m.e_stride, g,
+                                                 m.d, g_stride, alpha, rk, m.sel, m.stage, m.band, m.stage_cap,
                                                  m.tile_off, m.tile_cnt, m.tile_rej, m.tile_eq, m.ntiles);
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_hist_a_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
 {
     const Sel p = table[blockIdx.y / n].p;
-    stage_hist_a_body(p, blockIdx.y % n);
+    __shared__ SelectShared sm;
+    stage_hist_a_body(p, blockIdx.y % n, sm);
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_hist_b_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
 {
     const Sel p = table[blockIdx.y / n].p;
-    stage_hist_b_body(p, blockIdx.y % n);
+    __shared__ SelectShared sm;
+    stage_hist_b_body(p, blockIdx.y % n, sm);
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_classify_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
 {
     const MultiLayer &m = table[blockIdx.y / n];
     const Sel p = m.p;
-    stage_classify_body(p, blockIdx.y % n, m.walk_here);
+    __shared__ SelectShared sm;
+    stage_classify_body(p, blockIdx.y % n, m.walk_here, sm);
 }
 
 __global__ void __launch_bounds__(BLOCK) chunk_sums_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
@@ -1777,7 +1947,8 @@ __global__ void __launch_bounds__(BLOCK) chunk_sums_multi_kernel(const MultiLaye
     const MultiLayer &m = table[blockIdx.y / n];
     if (m.walk_here) return;                                 // the classification did the walk
     const Sel p = m.p;
-    chunk_sums_body(p, blockIdx.y % n);
+    __shared__ SelectShared sm;
+    chunk_sums_body(p, blockIdx.y % n, sm);
 }
 
 __global__ void __launch_bounds__(BLOCK)
@@ -1806,6 +1977,11 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_multi_kernel(const Multi
         __syncthreads();
     }
 }
+
+// The band list costs the streaming pass a second, unordered write of some candidates and a
+// few instructions per entry, and saves the selection kernels the candidates that are certain to
+// be selected.  That pays when the messages are dense (many candidates, most of them certain).
+bool band_route(const deco_ctx *c) { return c->k * 32 >= c->d; }
 
 RandParams make_rand(const deco_ctx *c)
 {
@@ -1838,7 +2014,8 @@ Sel make_sel(const deco_ctx *c)
     p.tile_eq = c->tile_eq;
     p.tile_take = c->tile_take;
     // the context's own rows of the job-wide directory and message buffer
-    p.tile_start = c->tile_start + static_cast<size_t>(c->worker_base) * (c->ntiles + 1);
+    p.tile_start = c->dir_rows + static_cast<size_t>(c->worker_base) * c->dir_stride;
+    p.dir_stride = c->dir_stride;
     p.tile_off = c->tile_off;
     p.tile_cnt = c->tile_cnt;
     p.tile_rej = c->tile_rej;
@@ -1848,14 +2025,16 @@ Sel make_sel(const deco_ctx *c)
     p.chunk_eq = c->chunk_eq;
     p.chunk_eqb = c->chunk_eqb;
     p.chunk_start = c->chunk_start;
-    p.msg = c->msg + static_cast<size_t>(c->worker_base) * c->k_cap;
-    p.k_cap = c->k_cap;
+    p.msg = c->msg_rows + static_cast<size_t>(c->worker_base) * c->msg_stride;
+    p.k_cap = c->msg_stride;
     p.stage = c->stage;
+    p.band = c->band;
     p.stage_cap = c->stage_cap;
     p.work = c->work;
     p.work_cap = c->work_cap;
     p.status = c->dev_status;
     p.rk = make_rand(c);
+    p.use_band = band_route(c) ? 1u : 0u;
     // Top-k keys have 31 bits, Random-k priorities 23
     p.sample_shift = (p.rk.on ? 23u : 31u) - SAMPLE_HIST_BITS;
     p.bound_low_bit = p.rk.on ? 0u : 7u;
@@ -1877,6 +2056,10 @@ uint32_t part_blocks(const deco_ctx *c, uint64_t items_per_worker, uint32_t item
 // ------------------------------------------------------------------------------------------
 bool streaming_route(const deco_ctx *c) { return c->select_mode == DECO_SELECT_AUTO; }
 
+// Up to this many staged pairs (estimated, all workers) the selection runs as one cooperative
+// launch; above it the separate kernels' higher occupancy outweighs their launch boundaries.
+constexpr uint64_t FUSED_CHAIN_MAX_PAIRS = 4ull << 20;
+
 cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s)
 {
     const float alpha = c->lr_at_server ? 1.0f : c->lr;
@@ -1892,12 +2075,12 @@ cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s)
     return cudaGetLastError();
 }
 
-template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
+template <int GT, bool ALIGNED, bool SPEC, bool RANDK, bool BAND>
 static void launch_acc_variant(deco_ctx *c, const void *grads, float alpha, cudaStream_t s)
 {
     dim3 grid(c->ntiles, c->n);
-    ef_accumulate_kernel<GT, ALIGNED, SPEC, RANDK><<<grid, BLOCK, 0, s>>>(
-        c->e, c->e_stride, grads, c->d, c->g_stride, alpha, make_rand(c), c->sel, c->stage, c->stage_cap,
+    ef_accumulate_kernel<GT, ALIGNED, SPEC, RANDK, BAND><<<grid, BLOCK, 0, s>>>(
+        c->e, c->e_stride, grads, c->d, c->g_stride, alpha, make_rand(c), c->sel, c->stage, c->band, c->stage_cap,
         c->tile_off, c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
 }
 
@@ -1906,11 +2089,16 @@ static void launch_acc(deco_ctx *c, const void *grads, float alpha, cudaStream_t
 {
     const bool randk = c->compressor == DECO_COMPRESSOR_RANDK;
     if (streaming_route(c)) {
-        if (randk) launch_acc_variant<GT, ALIGNED, true, true>(c, grads, alpha, s);
-        else launch_acc_variant<GT, ALIGNED, true, false>(c, grads, alpha, s);
+        if (band_route(c)) {
+            if (randk) launch_acc_variant<GT, ALIGNED, true, true, true>(c, grads, alpha, s);
+            else launch_acc_variant<GT, ALIGNED, true, false, true>(c, grads, alpha, s);
+        } else {
+            if (randk) launch_acc_variant<GT, ALIGNED, true, true, false>(c, grads, alpha, s);
+            else launch_acc_variant<GT, ALIGNED, true, false, false>(c, grads, alpha, s);
+        }
     } else {
         // the multi-pass route derives the keys itself: nothing is staged here
-        launch_acc_variant<GT, ALIGNED, false, false>(c, grads, alpha, s);
+        launch_acc_variant<GT, ALIGNED, false, false, false>(c, grads, alpha, s);
     }
 }
 
@@ -1942,6 +2130,9 @@ cudaError_t query_fallback_grid(deco_ctx *c)
     if (per_sm < 1) return cudaErrorLaunchOutOfResources;
     if (per_sm > 4) per_sm = 4;
     c->fallback_grid = static_cast<uint32_t>(per_sm * sms);
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_chain_kernel, BLOCK, 0);
+    if (err != cudaSuccess) return err;
+    c->chain_grid = per_sm < 1 ? 0u : static_cast<uint32_t>((per_sm > 8 ? 8 : per_sm) * sms);
     return cudaSuccess;
 }
 
@@ -1966,17 +2157,30 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     }
     // staged pairs per worker are a few times k: size the grids for that
     dim3 sgrid(part_blocks(c, 2 * c->k + 65536, BLOCK * 4), c->n);
-    stage_hist_a_kernel<<<sgrid, BLOCK, 0, s>>>(p);
-    stage_hist_b_kernel<<<sgrid, BLOCK, 0, s>>>(p);
     // the chunk walk is done by one CTA: with many chunks their sums are taken in parallel first
     const bool walk_here = c->nchunks <= 256;
+    // the kernels from here on rewrite the messages and their directory, which the previous
+    // iteration's aggregation may still be reading on the internal stream
+    if (c->chain_grid >= c->n && static_cast<uint64_t>(c->n) * (2 * c->k + 65536) <= FUSED_CHAIN_MAX_PAIRS) {
+        // one cooperative launch for the whole chain: as many CTAs per worker as the separate
+        // kernels would use, as far as they can all be resident at once
+        if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();
+        uint32_t gx = sgrid.x;
+        if (gx > c->chain_grid / c->n) gx = c->chain_grid / c->n;
+        uint32_t walk = walk_here ? 1u : 0u;
+        void *args[] = {&p, &walk};
+        c->launches += 1;
+        return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(select_chain_kernel), dim3(gx, c->n),
+                                           dim3(BLOCK), args, 0, s);
+    }
+    // more workers than CTAs that can be resident together: one launch per step of the chain
+    stage_hist_a_kernel<<<sgrid, BLOCK, 0, s>>>(p);
+    stage_hist_b_kernel<<<sgrid, BLOCK, 0, s>>>(p);
     stage_classify_kernel<<<sgrid, BLOCK, 0, s>>>(p, walk_here ? 1u : 0u);
     if (!walk_here) {
         chunk_sums_kernel<<<dim3((c->nchunks + WARPS - 1) / WARPS, c->n), BLOCK, 0, s>>>(p);
         c->launches += 1;
     }
-    // the kernels from here on rewrite the messages and their directory, which the previous
-    // iteration's aggregation may still be reading on the internal stream
     if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();
     // directory CTAs (a warp per chunk), then the CTAs whose warps stride over the work list:
     // enough of them for one slice per warp at about 1.3 k staged entries, capped at a few
@@ -2075,6 +2279,7 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
         const deco_ctx *c = mp->layers[l];
         MultiLayer &m = mp->host[l];
         m.p = make_sel(c);
+        m.p.use_band = 0;                // the streaming pass of many layers writes no band list
         m.g_off = mp->g_off[l];
         m.S = sample_groups(c->d, c->k);
         m.walk_here = c->nchunks <= 256 ? 1u : 0u;
@@ -2096,6 +2301,7 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
         AccLayer &a = grp.tab.L[l % ACC_LAYERS_MAX];
         a.e = m.p.e;
         a.stage = m.p.stage;
+        a.band = m.p.band;
         a.sel = m.p.sel;
         a.tile_off = m.p.tile_off;
         a.tile_cnt = m.p.tile_cnt;

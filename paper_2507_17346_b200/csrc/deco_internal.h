@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include <vector>
@@ -37,13 +38,17 @@ struct SelectState {
     uint32_t ties_take;     // final: how many entries equal to `threshold` are taken (by index)
     uint32_t exact;         // 1: this worker runs the multi-pass selection over e this step
     uint32_t spec_key;      // speculative lower bound used by the streaming pass (or DISABLED)
-    uint32_t n_staged;      // candidates staged by the streaming pass
+    uint32_t cert_key;      // staged entries with key >= cert_key are taken to be above the
+                            // threshold (checked by count); the others form the band
+    // what the streaming pass staged, updated with one 64-bit atomic per tile: low word =
+    // candidates (key >= spec_key), high word = those of them inside the band (key < cert_key)
+    unsigned long long staged_band;
     uint32_t exact_total;   // cumulative count of steps that took the multi-pass path
-    uint32_t unused0;
-    uint32_t rel_shift;     // log2 width of a coarse bin of the staged-key histogram (10..12)
-    uint32_t pad[5];
+    uint32_t rel_shift;     // log2 width of a coarse bin of the band-key histogram (10..12)
+    uint32_t pad[4];
 };
 static_assert(sizeof(SelectState) == 64, "one line per worker");
+static_assert(offsetof(SelectState, staged_band) % 8 == 0, "64-bit atomic target");
 
 constexpr uint32_t SPEC_DISABLED = 0x80000000u;   // above every 31-bit key
 
@@ -57,8 +62,9 @@ constexpr uint32_t SAMPLE_BINS = 4096;                  // bins of the sample hi
 
 struct Slot {
     uint64_t step = 0;
-    uint64_t positions = 0;
+    uint64_t positions = 0;     // pairs of a sparse aggregate; d for a dense one
     bool valid = false;
+    bool dense = false;         // the slot holds the plain vector S[d] instead of pairs
 };
 
 }  // namespace deco
@@ -92,9 +98,24 @@ struct deco_ctx {
     float *e = nullptr;
     float *params = nullptr;
     bool own_params = false;
-    deco_pair *msg = nullptr;           // [n_total][k_cap]
-    deco_pair *slots = nullptr;         // [ring][n_total * k_cap]
-    deco_pair *stage = nullptr;         // [n][stage_cap]
+    deco_pair *msg = nullptr;           // [n][k_cap] (not allocated with the exchange layout)
+    // Exchange layout (context created with n_total): one buffer of n_total rows, row w = the k
+    // pairs of global worker w's message followed by its tile directory (ntiles + 1 words),
+    // padded to an even number of words, so that what the ranks of a job all-gather is one
+    // contiguous range that holds k, not k_cap, pairs per worker.
+    bool packed = false;
+    uint32_t *xchg = nullptr;           // [n_total][xrow_cap] words
+    uint64_t xrow_cap = 0;              // words of a row at k = k_cap
+    // where the messages and their directory lie for the k of the current iteration
+    deco_pair *msg_rows = nullptr;      // row of global worker 0
+    uint64_t msg_stride = 0;            // pairs between rows
+    uint32_t *dir_rows = nullptr;
+    uint64_t dir_stride = 0;            // words between rows
+    deco_pair *slots = nullptr;         // [ring][slot_pairs]
+    uint64_t slot_pairs = 0;            // pairs per cache slot: n_total * k_cap, or room for a dense vector
+    bool dense_capable = false;         // a slot can hold S as a plain fp32 vector of e_stride entries
+    deco_pair *stage = nullptr;         // [n][stage_cap] candidates, tile by tile in index order
+    deco_pair *band = nullptr;          // [n][stage_cap] the candidates below cert_key once more, unordered
     uint2 *work = nullptr;              // [n][work_cap] emit work list: (tile, slice)
     uint64_t work_cap = 0;
     uint32_t *hist = nullptr;           // [n][2 routes][RADIX_LEVELS][RADIX_BINS]
@@ -102,11 +123,12 @@ struct deco_ctx {
     uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
     uint32_t *sample_hist = nullptr;    // [n][SAMPLE_BINS] sample keys per bin of their top bits (self-clearing)
     uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
+    uint32_t chain_grid = 0;            // most CTAs the cooperative selection launch may have
     deco::SelectState *sel = nullptr;   // [n]
     uint32_t *tile_gt = nullptr;        // [n][ntiles]  entries above the threshold per tile
     uint32_t *tile_eq = nullptr;        // [n][ntiles]  entries equal to it per tile
     uint32_t *tile_take = nullptr;      // [n][ntiles]  ties taken per tile
-    uint32_t *tile_start = nullptr;     // [n_total][ntiles + 1] message position of each tile
+    uint32_t *tile_start = nullptr;     // [n][ntiles + 1] message position of each tile (not with the exchange layout)
     uint32_t *tile_off = nullptr;       // [n][ntiles]  staging offset of each tile's candidates
     uint32_t *tile_cnt = nullptr;       // [n][ntiles]  staged candidates per tile
     uint32_t *tile_rej = nullptr;       // [n][ntiles]  staged candidates below the threshold
@@ -151,6 +173,29 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s);
 // deco_init with the distance between gradient rows given (0: d)
 deco_status init_context(deco_ctx **out, uint64_t d, uint32_t n, double delta, uint32_t tau, float lr,
                          const deco_options *opt, uint64_t g_stride);
+
+// Words of an exchange row at k pairs per message.
+inline uint64_t exchange_row_words(const deco_ctx *c, uint64_t k)
+{
+    return (2 * k + c->ntiles + 1 + 1) & ~1ull;
+}
+
+// Point msg_rows / dir_rows at the layout for messages of k pairs.
+inline void set_message_layout(deco_ctx *c, uint64_t k)
+{
+    if (c->packed) {
+        const uint64_t rw = exchange_row_words(c, k);
+        c->msg_rows = reinterpret_cast<deco_pair *>(c->xchg);
+        c->msg_stride = rw / 2;
+        c->dir_rows = c->xchg + 2 * k;
+        c->dir_stride = rw;
+    } else {
+        c->msg_rows = c->msg;
+        c->msg_stride = c->k_cap;
+        c->dir_rows = c->tile_start;
+        c->dir_stride = static_cast<uint64_t>(c->ntiles) + 1;
+    }
+}
 
 // Order stream s after the aggregation that deco_step left running on the internal stream.
 inline cudaError_t wait_for_aggregate(deco_ctx *c, cudaStream_t s)
@@ -235,6 +280,14 @@ uint32_t advance_iteration_external(deco_ctx *c, std::vector<uint32_t> *due);
 
 // --- kernel launchers (deco_server.cu) ---------------------------------------------------
 cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s);
+// the same with the aggregate kept as a plain vector of ntiles * TILE entries (dense messages)
+cudaError_t launch_aggregate_dense(deco_ctx *c, float *slot, cudaStream_t s);
+cudaError_t launch_apply_dense(deco_ctx *c, const float *slot, float neg_scale, cudaStream_t s);
+// dense when the messages of an iteration hold at least d / 4 entries in all
+inline bool aggregate_as_vector(const deco_ctx *c, uint64_t k)
+{
+    return c->dense_capable && static_cast<uint64_t>(c->n_total) * k * 4 >= c->d;
+}
 cudaError_t launch_apply(deco_ctx *c, const deco_pair *slot, uint64_t positions, float neg_scale,
                          cudaStream_t s);
 

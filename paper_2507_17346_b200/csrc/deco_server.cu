@@ -30,7 +30,8 @@ __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t 
 // One tile by the whole CTA: dense fp32 accumulator and touched-bit mask in shared memory (both
 // all-zero on entry and on exit), workers added in order, output in index order.
 __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, uint64_t k_cap,
-                                           const uint32_t *__restrict__ tile_start, uint32_t ntiles,
+                                           const uint32_t *__restrict__ tile_start, uint64_t dir_stride,
+                                           uint32_t ntiles,
                                            uint32_t n, deco_pair *__restrict__ slot,
                                            uint64_t positions, uint32_t *__restrict__ status,
                                            uint32_t tile, float *acc, uint32_t *mask, uint32_t *s_w)
@@ -39,8 +40,8 @@ __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, ui
     uint64_t out_off = 0;
     uint32_t cap = 0, longest = 0;
     for (uint32_t i = 0; i < n; ++i) {
-        const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-        const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+        const uint32_t a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
+        const uint32_t b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
         out_off += a;
         cap += b - a;
         longest = max(longest, b - a);
@@ -60,8 +61,8 @@ __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, ui
             pre[i].idx = DECO_NO_INDEX;
             pre[i].val = 0.0f;
             if (i < n) {
-                const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-                const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+                const uint32_t a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
+                const uint32_t b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
                 if (a + threadIdx.x < b) pre[i] = msg[static_cast<size_t>(i) * k_cap + a + threadIdx.x];
             }
         }
@@ -81,8 +82,8 @@ __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, ui
         }
     } else {
         for (uint32_t i = 0; i < n; ++i) {                 // worker order 0..n-1
-            const uint32_t a = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile];
-            const uint32_t b = tile_start[static_cast<size_t>(i) * (ntiles + 1) + tile + 1];
+            const uint32_t a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
+            const uint32_t b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
             if (b == a) continue;
             const deco_pair *src = msg + static_cast<size_t>(i) * k_cap;
             for (uint32_t p0 = a; p0 < b; p0 += 4 * BLOCK) {   // four loads in flight
@@ -151,7 +152,7 @@ __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, ui
 // Persistent CTAs, every tile by the whole CTA: for messages with many entries per tile.
 __global__ void __launch_bounds__(BLOCK)
 aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
-                 const uint32_t *__restrict__ tile_start, uint32_t ntiles, uint32_t n,
+                 const uint32_t *__restrict__ tile_start, uint64_t dir_stride, uint32_t ntiles, uint32_t n,
                  deco_pair *__restrict__ slot, uint64_t positions, uint32_t *__restrict__ status)
 {
     static_assert(TILE / 32 == BLOCK, "one mask word per thread");
@@ -162,7 +163,96 @@ aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     mask[threadIdx.x] = 0;
     __syncthreads();
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        dense_tile(msg, k_cap, tile_start, ntiles, n, slot, positions, status, tile, acc, mask, s_w);
+        dense_tile(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status, tile, acc, mask, s_w);
+}
+
+// Dense messages (n k entries in all comparable with d): the aggregate is kept as the plain
+// vector S[0 .. tiles * TILE) with +0 where no worker sent the index.  Same accumulator, same
+// worker order; the tile is then written out whole, with no mask and no compaction.
+__global__ void __launch_bounds__(BLOCK)
+aggregate_dense_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
+                       const uint32_t *__restrict__ tile_start, uint64_t dir_stride, uint32_t ntiles, uint32_t n,
+                       float *__restrict__ slot, uint32_t *__restrict__ status)
+{
+    __shared__ __align__(16) float acc[TILE];
+    for (int q = threadIdx.x; q < TILE; q += BLOCK) acc[q] = 0.0f;
+    __syncthreads();
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const uint32_t first = tile * static_cast<uint32_t>(TILE);
+        for (uint32_t i = 0; i < n; ++i) {                 // worker order 0..n-1
+            const uint32_t a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
+            const uint32_t b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
+            if (b <= a) continue;                          // the same for the whole CTA
+            const deco_pair *src = msg + static_cast<size_t>(i) * k_cap;
+            for (uint32_t p0 = a; p0 < b; p0 += 4 * BLOCK) {   // four loads in flight
+                deco_pair prs[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const uint32_t p = p0 + r * BLOCK + threadIdx.x;
+                    prs[r].idx = DECO_NO_INDEX;
+                    prs[r].val = 0.0f;
+                    if (p < b) prs[r] = src[p];
+                }
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if (prs[r].idx == DECO_NO_INDEX) continue;
+                    const uint32_t loc = prs[r].idx - first;
+                    if (loc >= static_cast<uint32_t>(TILE)) {
+                        latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, prs[r].idx);
+                        continue;
+                    }
+                    acc[loc] = acc[loc] + prs[r].val;      // indices are unique per worker
+                }
+            }
+            __syncthreads();
+        }
+        float4 *out = reinterpret_cast<float4 *>(slot + static_cast<size_t>(tile) * TILE);
+        float4 *acc4 = reinterpret_cast<float4 *>(acc);
+#pragma unroll
+        for (int q = threadIdx.x; q < TILE / 4; q += BLOCK) {
+            out[q] = acc4[q];
+            acc4[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+        __syncthreads();
+    }
+}
+
+// x[j] = fma(neg_scale, S[j], x[j]) for every j < d, S being a dense aggregate.  Where S is +0
+// the result is x[j] itself, bit for bit (also for x = -0), so groups of four untouched entries
+// are not written back.
+__global__ void __launch_bounds__(256)
+apply_dense_kernel(const float *__restrict__ S, float neg_scale, float *__restrict__ params, uint64_t d)
+{
+    const uint64_t nvec = d >> 2;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    const float4 *S4 = reinterpret_cast<const float4 *>(S);
+    float4 *x4 = reinterpret_cast<float4 *>(params);
+    for (uint64_t v0 = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; v0 < nvec; v0 += 4 * stride) {
+        float4 sv[4], xv[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint64_t v = v0 + r * stride;
+            sv[r] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            xv[r] = sv[r];
+            if (v < nvec) {
+                sv[r] = __ldcs(S4 + v);
+                xv[r] = x4[v];
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint64_t v = v0 + r * stride;
+            if (v >= nvec) continue;
+            if (sv[r].x == 0.0f && sv[r].y == 0.0f && sv[r].z == 0.0f && sv[r].w == 0.0f) continue;
+            x4[v] = make_float4(__fmaf_rn(neg_scale, sv[r].x, xv[r].x), __fmaf_rn(neg_scale, sv[r].y, xv[r].y),
+                                __fmaf_rn(neg_scale, sv[r].z, xv[r].z), __fmaf_rn(neg_scale, sv[r].w, xv[r].w));
+        }
+    }
+    // the last d % 4 entries
+    if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
+        const uint64_t j = (nvec << 2) + threadIdx.x;
+        params[j] = __fmaf_rn(neg_scale, S[j], params[j]);
+    }
 }
 
 // The entries a warp holds (one per lane, at most 32, worker-major and index-sorted within a
@@ -211,15 +301,16 @@ constexpr int SPARSE_WINDOWS = 4;
 // One tile by one warp.  Returns true (to every lane) if the tile does not fit and has to be
 // done by the whole CTA with the dense accumulator.
 __device__ __forceinline__ bool sparse_tile_warp(const deco_pair *__restrict__ msg, uint64_t k_cap,
-                                                 const uint32_t *__restrict__ tile_start, uint32_t ntiles,
+                                                 const uint32_t *__restrict__ tile_start, uint64_t dir_stride,
+                                                 uint32_t ntiles,
                                                  uint32_t n, deco_pair *__restrict__ slot, uint64_t positions,
                                                  uint32_t *__restrict__ status, uint32_t tile)
 {
     const int lane = threadIdx.x & 31;
     uint32_t a = 0, b = 0;
     if (static_cast<uint32_t>(lane) < n) {
-        a = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile];
-        b = tile_start[static_cast<size_t>(lane) * (ntiles + 1) + tile + 1];
+        a = tile_start[static_cast<size_t>(lane) * dir_stride + tile];
+        b = tile_start[static_cast<size_t>(lane) * dir_stride + tile + 1];
     }
     const uint32_t len = b - a;
     uint32_t cap = len, longest = len;
@@ -309,7 +400,7 @@ __device__ __forceinline__ bool sparse_tile_warp(const deco_pair *__restrict__ m
 
 __global__ void __launch_bounds__(BLOCK)
 aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
-                        const uint32_t *__restrict__ tile_start, uint32_t ntiles, uint32_t n,
+                        const uint32_t *__restrict__ tile_start, uint64_t dir_stride, uint32_t ntiles, uint32_t n,
                         deco_pair *__restrict__ slot, uint64_t positions,
                         uint32_t *__restrict__ status)
 {
@@ -321,7 +412,8 @@ aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     __syncthreads();
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t tile = blockIdx.x * WARPS + w;
-    if (tile < ntiles && sparse_tile_warp(msg, k_cap, tile_start, ntiles, n, slot, positions, status, tile) &&
+    if (tile < ntiles &&
+        sparse_tile_warp(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status, tile) &&
         lane == 0)
         atomicOr(&s_heavy, 1u << w);
     __syncthreads();
@@ -331,7 +423,7 @@ aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     mask[threadIdx.x] = 0;
     __syncthreads();
     for (; heavy; heavy &= heavy - 1)
-        dense_tile(msg, k_cap, tile_start, ntiles, n, slot, positions, status,
+        dense_tile(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status,
                    blockIdx.x * WARPS + __ffs(heavy) - 1, acc, mask, s_w);
 }
 
@@ -353,8 +445,8 @@ aggregate_multi_kernel(const ServerLayer *__restrict__ table, const uint32_t *__
         const uint32_t tile = g - L.first_tile;
         const uint64_t positions = static_cast<uint64_t>(n) * L.k;
         if (tile == 0 && threadIdx.x == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
-        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles, n, L.slots + slot_write * (n * L.k_cap), positions,
-                   L.status, tile, acc, mask, s_w);
+        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles + 1, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
+                   positions, L.status, tile, acc, mask, s_w);
     }
 }
 
@@ -376,8 +468,8 @@ aggregate_sparse_multi_kernel(const ServerLayer *__restrict__ table, const uint3
             const uint32_t tile = g - L.first_tile;
             const uint64_t positions = static_cast<uint64_t>(n) * L.k;
             if (tile == 0 && lane == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
-            if (sparse_tile_warp(L.msg, L.k_cap, L.tile_start, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
-                                 positions, L.status, tile) && lane == 0)
+            if (sparse_tile_warp(L.msg, L.k_cap, L.tile_start, L.ntiles + 1, L.ntiles, n,
+                                 L.slots + slot_write * (n * L.k_cap), positions, L.status, tile) && lane == 0)
                 atomicOr(&s_heavy, 1u << w);
         }
     }
@@ -390,7 +482,7 @@ aggregate_sparse_multi_kernel(const ServerLayer *__restrict__ table, const uint3
     for (; heavy; heavy &= heavy - 1) {
         const uint32_t gh = blockIdx.x * WARPS + __ffs(heavy) - 1;
         const ServerLayer &L = table[tile_layer[gh]];
-        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
+        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles + 1, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
                    static_cast<uint64_t>(n) * L.k, L.status, gh - L.first_tile, acc, mask, s_w);
     }
 }
@@ -471,7 +563,7 @@ small_server_kernel(const SmallLayer *__restrict__ table, uint32_t n, uint32_t a
         mask[threadIdx.x] = 0;
         __syncthreads();
         const uint64_t positions = static_cast<uint64_t>(n) * L.k;
-        dense_tile(L.msg, L.k_cap, L.tile_start, 1, n, L.slots + slot_write * slot_len, positions,
+        dense_tile(L.msg, L.k_cap, L.tile_start, 2, 1, n, L.slots + slot_write * slot_len, positions,
                    L.status, 0, acc, mask, s_w);
         if (threadIdx.x == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
         __syncthreads();
@@ -541,15 +633,36 @@ cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s)
     if (c->n_total <= 32 && positions <= 80ull * c->ntiles) {
         // on average at most 80 entries per tile over all workers: a warp per tile
         aggregate_sparse_kernel<<<(c->ntiles + WARPS - 1) / WARPS, BLOCK, 0, s>>>(
-            c->msg, c->k_cap, c->tile_start, c->ntiles, c->n_total, slot, positions, c->dev_status);
+            c->msg_rows, c->msg_stride, c->dir_rows, c->dir_stride, c->ntiles, c->n_total, slot, positions,
+            c->dev_status);
         return cudaGetLastError();
     }
     // next to the streaming pass of the following iteration the aggregation takes half the
     // CTA slots it could hold, so that the pass keeps most of its loads in flight
     const uint32_t per_sm = (c->agg_stream && s == c->agg_stream) ? 3u : 6u;
     const uint32_t blocks = c->ntiles < 148u * per_sm ? c->ntiles : 148u * per_sm;
-    aggregate_kernel<<<blocks, BLOCK, 0, s>>>(c->msg, c->k_cap, c->tile_start, c->ntiles, c->n_total,
-                                              slot, positions, c->dev_status);
+    aggregate_kernel<<<blocks, BLOCK, 0, s>>>(c->msg_rows, c->msg_stride, c->dir_rows, c->dir_stride, c->ntiles,
+                                              c->n_total, slot, positions, c->dev_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_aggregate_dense(deco_ctx *c, float *slot, cudaStream_t s)
+{
+    c->launches += 1;
+    const uint32_t per_sm = (c->agg_stream && s == c->agg_stream) ? 3u : 6u;
+    const uint32_t blocks = c->ntiles < 148u * per_sm ? c->ntiles : 148u * per_sm;
+    aggregate_dense_kernel<<<blocks, BLOCK, 0, s>>>(c->msg_rows, c->msg_stride, c->dir_rows, c->dir_stride,
+                                                    c->ntiles, c->n_total, slot, c->dev_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_apply_dense(deco_ctx *c, const float *slot, float neg_scale, cudaStream_t s)
+{
+    uint64_t blocks = ((c->d >> 2) + 4 * 256 - 1) / (4 * 256);
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148ull * 8) blocks = 148ull * 8;
+    apply_dense_kernel<<<static_cast<uint32_t>(blocks), 256, 0, s>>>(slot, neg_scale, c->params, c->d);
+    c->launches += 1;
     return cudaGetLastError();
 }
 

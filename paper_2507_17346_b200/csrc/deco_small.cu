@@ -159,7 +159,8 @@ small_worker_kernel(const SmallLayer *__restrict__ table, const void *__restrict
         s.n_greater = n_greater;
         s.k_rem = take;
         s.exact = 0;
-        s.n_staged = 0;
+        s.staged_band = 0;
+        s.cert_key = SPEC_DISABLED;
         s.spec_key = SPEC_DISABLED;
     }
 }

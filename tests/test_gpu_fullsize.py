@@ -114,18 +114,26 @@ def _dense_from_messages(msg, n, k, d):
 def _check_aggregate(ctx, t, msg, S, n, k, d, rng):
     """The cached aggregate of step t: every touched index once, increasing, with the
     worker-order fp32 sum; and the oracle's aggregate on a sample of the touched indices."""
-    addr, positions = B.deco_get_aggregate(ctx, t)
-    assert positions == n * k
-    slot = B.view_i32(addr, (positions, 2))
-    keep = slot[:, 0] != -1
-    sidx = slot[keep, 0].long()
-    sval = slot[keep, 1].contiguous().view(torch.float32)
     touched = torch.zeros(d, dtype=torch.bool, device="cuda")
     for i in range(n):
         touched[msg[i, :k, 0].long()] = True
-    assert int(sidx.numel()) == int(touched.sum())
-    assert bool((sidx[1:] > sidx[:-1]).all()) and bool(touched[sidx].all())
-    assert bool((sval.view(torch.int32) == S[sidx].view(torch.int32)).all())
+    if 4 * n * k >= d:
+        # dense messages: the aggregate is kept as the plain vector, +0 where nothing was sent
+        vec = B.view_f32(B.deco_get_aggregate_vector(ctx, t), (d,))
+        assert bool((vec.view(torch.int32) == S.view(torch.int32)).all())
+        assert bool((vec.view(torch.int32)[~touched] == 0).all())
+        sidx = torch.nonzero(touched).flatten()
+        sval = vec[sidx]
+    else:
+        addr, positions = B.deco_get_aggregate(ctx, t)
+        assert positions == n * k
+        slot = B.view_i32(addr, (positions, 2))
+        keep = slot[:, 0] != -1
+        sidx = slot[keep, 0].long()
+        sval = slot[keep, 1].contiguous().view(torch.float32)
+        assert int(sidx.numel()) == int(touched.sum())
+        assert bool((sidx[1:] > sidx[:-1]).all()) and bool(touched[sidx].all())
+        assert bool((sval.view(torch.int32) == S[sidx].view(torch.int32)).all())
     del touched
     pick = sidx[torch.from_numpy(rng.integers(0, sidx.numel(), 100_000)).cuda()].unique()
     small = []

@@ -328,7 +328,7 @@ def test_per_layer_seeded_random_partitions(seed):
 @pytest.mark.parametrize("compressor", ["topk", "randk"])
 def test_worker_sharded_contexts_equal_the_single_job(compressor):
     """Five workers split 2 + 3 over two contexts on one GPU.  Each compresses its own workers;
-    the rows of the two exchange buffers are then copied across (what the all-gather does
+    the rows of the exchange buffer are then copied across (what the all-gather does
     between GPUs), and both replicas aggregate and update.  Local messages and residuals, the
     aggregate and both parameter replicas must equal the oracle's single five-worker job."""
     from oracle import dd_ef_sgd as O
@@ -352,12 +352,15 @@ def test_worker_sharded_contexts_equal_the_single_job(compressor):
             views = []
             for c, (base, cnt) in zip(ctxs, split):
                 B.deco_ef_compress(c, g[base:base + cnt])
-                views.append(B.exchange_views(c))
+                rows, x = B.exchange_view(c)
+                # one contiguous range of k (not k_cap) pairs and a directory per worker
+                assert x["row_words"] == (2 * ref["k"] + (d + 8191) // 8192 + 1 + 1) // 2 * 2
+                assert rows.is_contiguous() and rows.shape == (n, x["row_words"])
+                views.append(rows)
             for me, (base, cnt) in enumerate(split):               # the exchange, by copies
                 for other in range(len(split)):
                     if other != me:
-                        views[other][0][base:base + cnt].copy_(views[me][0][base:base + cnt])
-                        views[other][1][base:base + cnt].copy_(views[me][1][base:base + cnt])
+                        views[other][base:base + cnt].copy_(views[me][base:base + cnt])
             touched = np.unique(np.concatenate([s for s, _ in ref["msgs"]]))
             for c, (base, cnt) in zip(ctxs, split):
                 idx, val = read_messages(c, cnt, ref["k"])
@@ -388,10 +391,15 @@ def test_sharded_step_through_nccl_with_one_rank():
     d, n = 120_000, 4
     dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29541", rank=0, world_size=1,
                             device_id=torch.device("cuda", 0))
-    a = B.deco_init(d, n, 0.01, 2, 0.1)
-    b = B.deco_init(d, n, 0.01, 2, 0.1)
+    a = B.deco_init(d, n, 0.01, 2, 0.1, n_total=n, delta_max=0.05)
+    b = B.deco_init(d, n, 0.01, 2, 0.1, delta_max=0.05)
     try:
+        with pytest.raises(B.DecoError):                  # no exchange buffer without n_total
+            B.deco_get_exchange(b)
         for t in range(5):
+            if t == 3:                                     # the rows get longer
+                B.deco_set_policy(a, 0.05, 1)
+                B.deco_set_policy(b, 0.05, 1)
             g = _values("normal", n, d, t, torch.float32)
             B.deco_step_sharded(a, g)
             B.deco_ef_compress(b, g)
@@ -585,6 +593,53 @@ def test_checkpoint_and_resume_give_the_same_bits():
             assert e.value.status == B.DECO_ERR_INVALID_ARG
         finally:
             B.deco_destroy(c)
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_dense_messages_keep_the_aggregate_as_a_vector(mode):
+    """When the n messages hold at least d / 4 entries in all the cached aggregate is the plain
+    vector S[d] (same worker-order sums; +0 where nothing was sent) and the update sweeps it.
+    The density crosses that limit in both directions at run time, with a cache of several
+    slots, odd lengths and both gradient types; every buffer against the oracle."""
+    d, n = 150_003, 4
+    plan = {2: (0.02, 3), 4: (0.3, 1), 7: (0.07, 2), 9: (0.01, 0)}
+    for dtype, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        run_parity(d, n, 0.1, 2, 0.1, lambda t: _values("normal", n, d, t, dtype), steps=12,
+                   grad_dtype=name, policy_plan=plan, tau_max=3, delta_max=0.3, select_mode=mode)
+    run_parity(8193, 9, 0.05, 1, 0.1, lambda t: _values("coarse", 9, 8193, t, torch.float32), steps=4,
+               select_mode=mode)
+
+
+def test_checkpoint_with_vector_aggregates():
+    """Cached aggregates in both layouts travel through export / import."""
+    d, n = 120_001, 4
+    kw = dict(tau_max=3, delta_max=0.2)
+    a = B.deco_init(d, n, 0.1, 3, 0.1, **kw)
+    b = B.deco_init(d, n, 0.1, 3, 0.1, **kw)
+    try:
+        for t in range(6):
+            if t == 4:
+                B.deco_set_policy(a, 0.01, 3)            # the last two aggregates are pairs
+            B.deco_step(a, _values("normal", n, d, t, torch.float32))
+        B.deco_get_aggregate_vector(a, 3)
+        B.deco_get_aggregate(a, 5)
+        with pytest.raises(B.DecoError):
+            B.deco_get_aggregate(a, 3)
+        blob = B.deco_export_state(a)
+        assert len(blob) == B.deco_state_bytes(a)
+        B.deco_import_state(b, blob)
+        for t in range(6, 11):
+            g = _values("normal", n, d, t, torch.float32)
+            B.deco_step(a, g)
+            B.deco_step(b, g)
+        torch.cuda.synchronize()
+        ba, bb = B.deco_get_buffers(a), B.deco_get_buffers(b)
+        for name, shape in (("e", (n, ba["e_stride"])), ("params", (d,))):
+            assert torch.equal(B.view_i32(ba[name], shape), B.view_i32(bb[name], shape)), name
+        assert B.deco_get_stats(a)["device_status"] == 0 and B.deco_get_stats(b)["device_status"] == 0
     finally:
         B.deco_destroy(a)
         B.deco_destroy(b)

@@ -56,8 +56,11 @@ def test_reference_arm_prints_one_line_from_rank_zero():
 
 def _sharded_rank(rank, world, port, out):
     """Each rank plays the worker side of its own workers (with the oracle, on CPU), lays its
-    messages out as rows of the job-wide exchange buffers and all-gathers them with the
-    binding's helper; the server side then has to see the single-process result."""
+    messages out as rows of the job-wide exchange buffer — k pairs, then the tile directory,
+    padded to an even number of words, rows back to back — and all-gathers them with the
+    binding's helper in ONE collective; the server side then has to see the single-process
+    result.  Two rounds with different k (a policy change between iterations): the rows of the
+    second round have another length inside the same buffer."""
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
@@ -65,28 +68,37 @@ def _sharded_rank(rank, world, port, out):
     import numpy as np
     from oracle import dd_ef_sgd as O
     from paper_2507_17346_b200 import binding as B
-    d, n_total, k, tile = 20_000, 4, 37, 8192
+    d, n_total, k_cap, tile = 20_000, 4, 120, 8192
     per = n_total // world
     rng = np.random.default_rng(3)
-    a = rng.standard_normal((n_total, d)).astype(np.float32)          # same on every rank
     ntiles = (d + tile - 1) // tile
-    msg = torch.zeros((n_total, k, 2), dtype=torch.int32)
-    dirs = torch.zeros((n_total, ntiles + 1), dtype=torch.int32)
-    for w in range(rank * per, (rank + 1) * per):                      # the local workers only
-        sel, vals, _ = O.compress(a[w], k)
-        msg[w, :, 0] = torch.from_numpy(sel.astype(np.int64).astype(np.int32))
-        msg[w, :, 1] = torch.from_numpy(vals.view(np.int32))
-        dirs[w] = torch.from_numpy(np.searchsorted(sel, np.arange(ntiles + 1) * tile).astype(np.int32))
-    B.all_gather_rows(msg, rank * per, per)
-    B.all_gather_rows(dirs, rank * per, per)
-    got = [(msg[w, :, 0].numpy().astype(np.uint32), msg[w, :, 1].numpy().view(np.float32))
-           for w in range(n_total)]
-    S, _ = O.aggregate(got, d)
-    want = [O.compress(a[w], k)[:2] for w in range(n_total)]
-    S_want, _ = O.aggregate(want, d)
-    ok = bool(np.array_equal(S.view(np.uint32), S_want.view(np.uint32)))
-    for w in range(n_total):
-        ok = ok and dirs[w, -1].item() == k and np.array_equal(got[w][0], want[w][0])
+
+    def row_words(k):
+        return (2 * k + ntiles + 1 + 1) // 2 * 2
+
+    buf = torch.zeros(n_total * row_words(k_cap), dtype=torch.int32)     # sized for k_cap
+    ok = True
+    for k in (37, 120, 5):
+        a = rng.standard_normal((n_total, d)).astype(np.float32)          # same on every rank
+        rw = row_words(k)
+        rows = buf[:n_total * rw].view(n_total, rw)                       # contiguous prefix
+        rows.zero_()
+        for w in range(rank * per, (rank + 1) * per):                      # the local workers only
+            sel, vals, _ = O.compress(a[w], k)
+            rows[w, 0:2 * k:2] = torch.from_numpy(sel.astype(np.int64).astype(np.int32))
+            rows[w, 1:2 * k:2] = torch.from_numpy(vals.view(np.int32))
+            rows[w, 2 * k:2 * k + ntiles + 1] = torch.from_numpy(
+                np.searchsorted(sel, np.arange(ntiles + 1) * tile).astype(np.int32))
+        B.all_gather_rows(rows, rank * per, per)
+        got = [(rows[w, 0:2 * k:2].numpy().astype(np.uint32),
+                rows[w, 1:2 * k:2].numpy().copy().view(np.float32)) for w in range(n_total)]
+        S, _ = O.aggregate(got, d)
+        want = [O.compress(a[w], k)[:2] for w in range(n_total)]
+        S_want, _ = O.aggregate(want, d)
+        ok = ok and bool(np.array_equal(S.view(np.uint32), S_want.view(np.uint32)))
+        for w in range(n_total):
+            ok = ok and rows[w, 2 * k + ntiles].item() == k and np.array_equal(got[w][0], want[w][0])
+            ok = ok and rows[w, 2 * k].item() == 0
     with open(out + ".%d" % rank, "w") as fh:
         json.dump({"ok": ok}, fh)
     dist.destroy_process_group()
