@@ -244,7 +244,6 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     }
     need(dev_alloc(c, &c->slots, static_cast<uint64_t>(c->ring) * c->slot_pairs));
     need(dev_alloc(c, &c->stage, static_cast<uint64_t>(n) * c->stage_cap));
-    need(dev_alloc(c, &c->band, static_cast<uint64_t>(n) * c->stage_cap));
     // slices of 256 staged entries, plus one partial slice for every tile that has any
     c->work_cap = c->stage_cap / 256 + (c->stage_cap / 17 < c->ntiles ? c->stage_cap / 17 : c->ntiles) + 32;
     need(dev_alloc(c, &c->work, static_cast<uint64_t>(n) * c->work_cap));
@@ -267,6 +266,8 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     need(dev_alloc(c, &c->chunk_eqb, static_cast<uint64_t>(n) * c->nchunks));
     need(dev_alloc(c, &c->chunk_start, static_cast<uint64_t>(n) * (c->nchunks + 1)));
     need(dev_alloc(c, &c->dev_status, 4));
+    // the band list exists only where deco_set_policy can make the messages dense enough for it
+    if (c->k_cap * 32 >= d) need(dev_alloc(c, &c->band, static_cast<uint64_t>(n) * c->stage_cap));
     if (st == DECO_OK && query_fallback_grid(c) != cudaSuccess) st = DECO_ERR_CUDA;
     if (st == DECO_OK &&
         (cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) != cudaSuccess ||

@@ -129,11 +129,22 @@ __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t 
     }
 }
 
-// What the streaming pass staged for a worker, read through L2 (another CTA of the same launch
-// may have written the record): candidates in all, and those inside the band.
+// Loads of what earlier kernels, or earlier phases of the same cooperative launch, left behind.
+// As launches of their own the selection bodies use plain loads: every CTA of a grid reads the
+// same 64-byte selection record, which the L1 caches then serve once per SM (read through L2
+// by every warp, that one line becomes the bottleneck of a grid of a thousand CTAs).  Inside the
+// cooperative launch (COH), whose grids are small, they read through L2.
+template <bool COH, typename T>
+__device__ __forceinline__ T ldq(const T *p)
+{
+    return COH ? __ldcg(p) : *p;
+}
+
+// What the streaming pass staged for a worker: candidates in all, and those inside the band.
+template <bool COH>
 __device__ __forceinline__ void staged_counts(const SelectState &s, uint32_t &n_staged, uint32_t &n_band)
 {
-    const unsigned long long v = __ldcg(&s.staged_band);
+    const unsigned long long v = ldq<COH>(&s.staged_band);
     n_staged = static_cast<uint32_t>(v);
     n_band = static_cast<uint32_t>(v >> 32);
 }
@@ -867,18 +878,35 @@ ef_accumulate_body(const uint32_t tile, const uint32_t i, const bool rows_aligne
     }
 }
 
-template <int GT, bool ALIGNED, bool SPEC, bool RANDK, bool BAND>
-__global__ void __launch_bounds__(BLOCK, 3)
+template <int GT, bool ALIGNED, bool SPEC, bool RANDK>
+__global__ void __launch_bounds__(BLOCK)
 ef_accumulate_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
                      uint64_t d, uint64_t g_stride, float alpha, RandParams rk, SelectState *__restrict__ sel,
-                     deco_pair *__restrict__ stage, deco_pair *__restrict__ band, uint64_t stage_cap,
+                     deco_pair *__restrict__ stage, uint64_t stage_cap,
                      uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
                      uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
                      uint32_t ntiles)
 {
-    ef_accumulate_body<GT, ALIGNED, SPEC, RANDK, BAND>(blockIdx.x, blockIdx.y, true, e, e_stride, grads, d, g_stride,
-                                                 alpha, rk, sel, stage, band, stage_cap, tile_off, tile_cnt,
-                                                 tile_rej, tile_eq, ntiles);
+    ef_accumulate_body<GT, ALIGNED, SPEC, RANDK, false>(blockIdx.x, blockIdx.y, true, e, e_stride, grads, d,
+                                                        g_stride, alpha, rk, sel, stage, nullptr, stage_cap, tile_off,
+                                                        tile_cnt, tile_rej, tile_eq, ntiles);
+}
+
+// The same with the band list.  Left to itself the compiler takes more than 85 registers for
+// it, which would cost the third CTA per SM: the limit is forced here (and only here: forcing
+// it on the kernel above, which needs 80 by itself, makes that one slower).
+template <int GT, bool ALIGNED, bool RANDK>
+__global__ void __launch_bounds__(BLOCK, 3)
+ef_accumulate_band_kernel(float *__restrict__ e, uint64_t e_stride, const void *__restrict__ grads,
+                          uint64_t d, uint64_t g_stride, float alpha, RandParams rk, SelectState *__restrict__ sel,
+                          deco_pair *__restrict__ stage, deco_pair *__restrict__ band, uint64_t stage_cap,
+                          uint32_t *__restrict__ tile_off, uint32_t *__restrict__ tile_cnt,
+                          uint32_t *__restrict__ tile_rej, uint32_t *__restrict__ tile_eq,
+                          uint32_t ntiles)
+{
+    ef_accumulate_body<GT, ALIGNED, true, RANDK, true>(blockIdx.x, blockIdx.y, true, e, e_stride, grads, d,
+                                                       g_stride, alpha, rk, sel, stage, band, stage_cap, tile_off,
+                                                       tile_cnt, tile_rej, tile_eq, ntiles);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -949,6 +977,9 @@ struct SelectShared {
     uint32_t warp[WARPS];
     uint32_t out[2];
 };
+// One instance per kernel that runs any of the bodies (a variable of namespace scope, so that
+// every access is known to be a shared-memory access).
+__shared__ SelectShared sm;
 
 // Level A: histogram of the coarse bins of the band keys.  The last CTA of a worker to
 // arrive takes the decision: is the staged set usable (at least k candidates, so it contains
@@ -956,15 +987,16 @@ struct SelectShared {
 // certainty bound, so the threshold lies in the band), and which coarse bin holds the entry of
 // rank k - (candidates above the band).  If the set is not usable, or the threshold falls into
 // the shared top bin, the worker is handed to the multi-pass route.
-__device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i, SelectShared &sm)
+template <bool COH>
+__device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i)
 {
     SelectState &s = p.sel[i];
-    if (__ldcg(&s.exact)) return;
+    if (ldq<COH>(&s.exact)) return;
     uint32_t n_staged, n_band;
-    staged_counts(s, n_staged, n_band);
+    staged_counts<COH>(s, n_staged, n_band);
     const deco_pair *src = select_list(p, i, n_staged, n_band);
     const uint32_t n_cert = n_staged - n_band;
-    const uint32_t spec = __ldcg(&s.spec_key), shift = __ldcg(&s.rel_shift);
+    const uint32_t spec = ldq<COH>(&s.spec_key), shift = ldq<COH>(&s.rel_shift);
     const bool valid = n_staged >= p.k && n_staged <= p.stage_cap && n_cert < p.k;
     uint32_t *h = sm.h;
     if (valid) {
@@ -1008,21 +1040,22 @@ __device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i
 
 __global__ void __launch_bounds__(BLOCK) stage_hist_a_kernel(Sel p)
 {
-    __shared__ SelectShared sm;
-    stage_hist_a_body(p, blockIdx.y, sm);
+    stage_hist_a_body<false>(p, blockIdx.y);
 }
 
 // Level B: histogram of the low bits of the band keys that fell into the chosen A bin; the
 // last CTA of a worker to arrive fixes the threshold key and the number of ties to take.
-__device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i, SelectShared &sm)
+template <bool COH>
+__device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i)
 {
     SelectState &s = p.sel[i];
-    if (__ldcg(&s.exact)) return;
+    if (ldq<COH>(&s.exact)) return;
     uint32_t *h = sm.h;
     uint32_t n_staged, n_band;
-    staged_counts(s, n_staged, n_band);
-    const uint32_t spec = __ldcg(&s.spec_key), shift = __ldcg(&s.rel_shift);
-    const uint32_t a_sel = __ldcg(&s.prefix), above_a = __ldcg(&s.n_greater), k_rem = __ldcg(&s.k_rem);   // from level A
+    staged_counts<COH>(s, n_staged, n_band);
+    const uint32_t spec = ldq<COH>(&s.spec_key), shift = ldq<COH>(&s.rel_shift);
+    const uint32_t a_sel = ldq<COH>(&s.prefix), above_a = ldq<COH>(&s.n_greater),
+                   k_rem = ldq<COH>(&s.k_rem);                         // from level A
     const uint32_t low_mask = (1u << shift) - 1u;
     const deco_pair *src = select_list(p, i, n_staged, n_band);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
@@ -1069,8 +1102,7 @@ __device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i
 
 __global__ void __launch_bounds__(BLOCK) stage_hist_b_kernel(Sel p)
 {
-    __shared__ SelectShared sm;
-    stage_hist_b_body(p, blockIdx.y, sm);
+    stage_hist_b_body<false>(p, blockIdx.y);
 }
 
 // One CTA: ties are granted to chunks in index order until ties_take are used up, then every
@@ -1087,7 +1119,7 @@ __device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, 
     const uint32_t *tcnt = p.tile_cnt + static_cast<size_t>(i) * p.ntiles;
     const uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     const uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
-    const uint32_t ties = __ldcg(&p.sel[i].ties_take);
+    const uint32_t ties = p.sel[i].ties_take;
     const uint32_t per = (p.nchunks + blockDim.x - 1) / blockDim.x;
     const uint32_t lo = min(p.nchunks, threadIdx.x * per), hi = min(p.nchunks, lo + per);
     uint32_t eq_sum = 0;
@@ -1139,18 +1171,18 @@ __device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, 
 // Many chunks: their sums are taken in parallel, one warp per chunk (three coalesced loads
 // and a warp reduction; the CTAs stride over the chunks), and the last CTA of a worker to
 // arrive walks the chunks.
-__device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i, SelectShared &sm)
+__device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i)
 {
-    if (__ldcg(&p.sel[i].exact)) return;
+    if (p.sel[i].exact) return;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     for (uint32_t chunk = blockIdx.x * WARPS + w; chunk < p.nchunks; chunk += gridDim.x * WARPS) {
         const uint32_t tile = chunk * CHUNK_TILES + lane;
         const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
         uint32_t a = 0, b = 0, q = 0;
         if (tile < p.ntiles) {
-            a = __ldcg(&p.tile_cnt[ti]);
-            b = __ldcg(&p.tile_rej[ti]);
-            q = __ldcg(&p.tile_eq[ti]);
+            a = p.tile_cnt[ti];
+            b = p.tile_rej[ti];
+            q = p.tile_eq[ti];
         }
         for (int o = 16; o > 0; o >>= 1) {
             a += __shfl_down_sync(FULL, a, o);
@@ -1169,8 +1201,7 @@ __device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i, 
 
 __global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p)
 {
-    __shared__ SelectShared sm;
-    chunk_sums_body(p, blockIdx.y, sm);
+    chunk_sums_body(p, blockIdx.y);
 }
 
 // Classification.  With the threshold known every band entry below it is rejected: counted
@@ -1179,14 +1210,14 @@ __global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p)
 // CTA of a worker to arrive then walks the chunks once; with many, the chunk sums follow.
 // (The per-tile positions follow from these inside the emit step, so nothing here is serial
 // in the number of tiles.)
-__device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t i, uint32_t walk_here,
-                                                    SelectShared &sm)
+template <bool COH>
+__device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t i, uint32_t walk_here)
 {
     const SelectState &s = p.sel[i];
-    if (__ldcg(&s.exact)) return;
+    if (ldq<COH>(&s.exact)) return;
     uint32_t n_staged, n_band;
-    staged_counts(s, n_staged, n_band);
-    const uint32_t T = __ldcg(&s.threshold);
+    staged_counts<COH>(s, n_staged, n_band);
+    const uint32_t T = ldq<COH>(&s.threshold);
     const deco_pair *src = select_list(p, i, n_staged, n_band);
     uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
@@ -1240,8 +1271,7 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
 
 __global__ void __launch_bounds__(BLOCK) stage_classify_kernel(Sel p, uint32_t walk_here)
 {
-    __shared__ SelectShared sm;
-    stage_classify_body(p, blockIdx.y, walk_here, sm);
+    stage_classify_body<false>(p, blockIdx.y, walk_here);
 }
 
 // What a warp learns about the CHUNK_TILES tiles of one chunk from three coalesced loads and
@@ -1253,7 +1283,7 @@ struct TileInfo {
     uint32_t start;   // message position of the tile's first entry
 };
 
-template <bool WRITE_DIR>
+template <bool WRITE_DIR, bool COH>
 __device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint32_t chunk)
 {
     const int lane = threadIdx.x & 31;
@@ -1262,12 +1292,13 @@ __device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint3
     uint32_t cnt = 0, rej = 0, eq = 0;
     if (tile < p.ntiles) {
         cnt = p.tile_cnt[ti];
-        rej = __ldcg(&p.tile_rej[ti]);
-        eq = __ldcg(&p.tile_eq[ti]);
+        rej = ldq<COH>(&p.tile_rej[ti]);
+        eq = ldq<COH>(&p.tile_eq[ti]);
     }
-    const uint32_t ties = __ldcg(&p.sel[i].ties_take);
-    const uint32_t eqb0 = __ldcg(&p.chunk_eqb[static_cast<size_t>(i) * p.nchunks + chunk]);
-    const uint32_t start0 = __ldcg(&p.chunk_start[static_cast<size_t>(i) * (p.nchunks + 1) + chunk]);
+    const size_t cb = static_cast<size_t>(i) * p.nchunks + chunk, cs = static_cast<size_t>(i) * (p.nchunks + 1) + chunk;
+    const uint32_t ties = ldq<COH>(&p.sel[i].ties_take);
+    const uint32_t eqb0 = ldq<COH>(&p.chunk_eqb[cb]);
+    const uint32_t start0 = ldq<COH>(&p.chunk_start[cs]);
     const uint32_t eq_before = eqb0 + warp_incl_scan(eq) - eq;
     const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
     TileInfo t;
@@ -1338,12 +1369,13 @@ __device__ __forceinline__ uint32_t emit_segment_warp(const Sel &p, uint32_t i, 
 // Emit, directory part: CTA `cta` of `nctas`; a warp per chunk of CHUNK_TILES tiles (the CTAs
 // stride over the chunks) writes the directory and each lane walks its own tile if that holds
 // at most EMIT_LANE_MAX staged entries.
+template <bool COH>
 __device__ __forceinline__ void emit_directory_part(const Sel &p, const uint32_t i, uint32_t cta, uint32_t nctas)
 {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t T = __ldcg(&p.sel[i].threshold);
+    const uint32_t T = ldq<COH>(&p.sel[i].threshold);
     for (uint32_t chunk = cta * WARPS + w; chunk < p.nchunks; chunk += nctas * WARPS) {
-        const TileInfo t = chunk_header<true>(p, i, chunk);
+        const TileInfo t = chunk_header<true, COH>(p, i, chunk);
         const uint32_t tile = chunk * CHUNK_TILES + lane;
         if (t.cnt == 0 || t.cnt > EMIT_LANE_MAX) continue;
         const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
@@ -1372,11 +1404,12 @@ __device__ __forceinline__ void emit_directory_part(const Sel &p, const uint32_t
 // Emit, work-list part: the warps of CTA `cta` of `nctas` stride over the work list; a warp
 // that gets slice j > 0 of a tile first counts, with independent loads, what the slices before
 // it emit.
+template <bool COH>
 __device__ __forceinline__ void emit_items_part(const Sel &p, const uint32_t i, uint32_t cta, uint32_t nctas)
 {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t T = __ldcg(&p.sel[i].threshold);
-    const uint32_t n_items = min(__ldcg(&p.done[i * DONE_SLOTS + 5]), static_cast<uint32_t>(p.work_cap));
+    const uint32_t T = ldq<COH>(&p.sel[i].threshold);
+    const uint32_t n_items = min(ldq<COH>(&p.done[i * DONE_SLOTS + 5]), static_cast<uint32_t>(p.work_cap));
     const uint2 *work = p.work + static_cast<size_t>(i) * p.work_cap;
     const uint32_t warps = nctas * WARPS;
     for (uint32_t q = cta * WARPS + w; q < n_items; q += warps) {
@@ -1386,7 +1419,7 @@ __device__ __forceinline__ void emit_items_part(const Sel &p, const uint32_t i, 
             if (lane == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x321u, q);
             continue;
         }
-        const TileInfo t = chunk_header<false>(p, i, tile / CHUNK_TILES);
+        const TileInfo t = chunk_header<false, COH>(p, i, tile / CHUNK_TILES);
         const uint32_t my = tile % CHUNK_TILES;
         const uint32_t cnt = __shfl_sync(FULL, t.cnt, my), start = __shfl_sync(FULL, t.start, my);
         const uint32_t want = __shfl_sync(FULL, t.sel, my), take = __shfl_sync(FULL, t.take, my);
@@ -1431,9 +1464,9 @@ __device__ __forceinline__ void emit_items_part(const Sel &p, const uint32_t i, 
 // remaining CTAs the work list.
 __device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, uint32_t dir_ctas)
 {
-    if (__ldcg(&p.sel[i].exact)) return;
-    if (blockIdx.x < dir_ctas) emit_directory_part(p, i, blockIdx.x, dir_ctas);
-    else emit_items_part(p, i, blockIdx.x - dir_ctas, gridDim.x - dir_ctas);
+    if (p.sel[i].exact) return;
+    if (blockIdx.x < dir_ctas) emit_directory_part<false>(p, i, blockIdx.x, dir_ctas);
+    else emit_items_part<false>(p, i, blockIdx.x - dir_ctas, gridDim.x - dir_ctas);
 }
 
 __global__ void __launch_bounds__(BLOCK) emit_stage_kernel(Sel p, uint32_t dir_ctas)
@@ -1809,31 +1842,26 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_kernel(Sel p)
     exact_fallback_body(p, grid, h, s_a, s_b, s_out);
 }
 
-// ---- the whole selection of the streaming route in one cooperative launch: level A, level B,
-// classification, chunk sums and walk, emit, each separated from the next by a grid-wide
-// barrier (where the separate kernels have a launch boundary), then the multi-pass route for
-// the workers whose staged set was rejected, if there are any.  Grid: x = CTAs of a worker,
-// y = worker; every body strides over its work by gridDim.x.  Which barriers a CTA takes depends
-// only on kernel arguments and on a flag that is final after the first barrier, so the whole
-// grid takes the same ones.
-__global__ void __launch_bounds__(BLOCK, 3) select_chain_kernel(Sel p, uint32_t walk_here)
+// ---- small problems: the whole selection of the streaming route in one cooperative launch —
+// level A, level B, classification with the chunk walk, emit — each separated from the next by
+// a grid-wide barrier where the separate kernels have a launch boundary, then the multi-pass
+// route for the workers whose staged set was rejected, if there are any.  Grid: x = CTAs of a
+// worker, y = worker; every body strides over its work by gridDim.x.  Only for vectors of few
+// chunks (the classification's last CTA walks them itself).  Which barriers a CTA takes depends
+// on a flag that is final after the first barrier, so the whole grid takes the same ones.
+__global__ void __launch_bounds__(BLOCK, 3) select_chain_kernel(Sel p)
 {
     cg::grid_group grid = cg::this_grid();
-    __shared__ SelectShared sm;
     const uint32_t i = blockIdx.y;
-    stage_hist_a_body(p, i, sm);
+    stage_hist_a_body<true>(p, i);
     grid.sync();
-    stage_hist_b_body(p, i, sm);
+    stage_hist_b_body<true>(p, i);
     grid.sync();
-    stage_classify_body(p, i, walk_here, sm);
+    stage_classify_body<true>(p, i, 1u);
     grid.sync();
-    if (!walk_here) {
-        chunk_sums_body(p, i, sm);
-        grid.sync();
-    }
     if (!__ldcg(&p.sel[i].exact)) {
-        emit_directory_part(p, i, blockIdx.x, gridDim.x);
-        emit_items_part(p, i, blockIdx.x, gridDim.x);
+        emit_directory_part<true>(p, i, blockIdx.x, gridDim.x);
+        emit_items_part<true>(p, i, blockIdx.x, gridDim.x);
     }
     if (__ldcg(&p.status[3]) == 0) return;
     __syncthreads();
@@ -1923,23 +1951,20 @@ ef_accumulate_multi_kernel(const __grid_constant__ AccTable tab, const void *__r
 __global__ void __launch_bounds__(BLOCK) stage_hist_a_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
 {
     const Sel p = table[blockIdx.y / n].p;
-    __shared__ SelectShared sm;
-    stage_hist_a_body(p, blockIdx.y % n, sm);
+    stage_hist_a_body<false>(p, blockIdx.y % n);
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_hist_b_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
 {
     const Sel p = table[blockIdx.y / n].p;
-    __shared__ SelectShared sm;
-    stage_hist_b_body(p, blockIdx.y % n, sm);
+    stage_hist_b_body<false>(p, blockIdx.y % n);
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_classify_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
 {
     const MultiLayer &m = table[blockIdx.y / n];
     const Sel p = m.p;
-    __shared__ SelectShared sm;
-    stage_classify_body(p, blockIdx.y % n, m.walk_here, sm);
+    stage_classify_body<false>(p, blockIdx.y % n, m.walk_here);
 }
 
 __global__ void __launch_bounds__(BLOCK) chunk_sums_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
@@ -1947,8 +1972,7 @@ __global__ void __launch_bounds__(BLOCK) chunk_sums_multi_kernel(const MultiLaye
     const MultiLayer &m = table[blockIdx.y / n];
     if (m.walk_here) return;                                 // the classification did the walk
     const Sel p = m.p;
-    __shared__ SelectShared sm;
-    chunk_sums_body(p, blockIdx.y % n, sm);
+    chunk_sums_body(p, blockIdx.y % n);
 }
 
 __global__ void __launch_bounds__(BLOCK)
@@ -1981,7 +2005,7 @@ __global__ void __launch_bounds__(BLOCK) exact_fallback_multi_kernel(const Multi
 // The band list costs the streaming pass a second, unordered write of some candidates and a
 // few instructions per entry, and saves the selection kernels the candidates that are certain to
 // be selected.  That pays when the messages are dense (many candidates, most of them certain).
-bool band_route(const deco_ctx *c) { return c->k * 32 >= c->d; }
+bool band_route(const deco_ctx *c) { return c->band != nullptr && c->k * 32 >= c->d; }
 
 RandParams make_rand(const deco_ctx *c)
 {
@@ -2056,8 +2080,9 @@ uint32_t part_blocks(const deco_ctx *c, uint64_t items_per_worker, uint32_t item
 // ------------------------------------------------------------------------------------------
 bool streaming_route(const deco_ctx *c) { return c->select_mode == DECO_SELECT_AUTO; }
 
-// Up to this many staged pairs (estimated, all workers) the selection runs as one cooperative
-// launch; above it the separate kernels' higher occupancy outweighs their launch boundaries.
+// Up to this many staged pairs (estimated, all workers), and with few enough chunks for the
+// classification to walk them itself, the selection runs as one cooperative launch; beyond
+// that the separate kernels' higher occupancy outweighs their launch boundaries.
 constexpr uint64_t FUSED_CHAIN_MAX_PAIRS = 4ull << 20;
 
 cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s)
@@ -2079,9 +2104,14 @@ template <int GT, bool ALIGNED, bool SPEC, bool RANDK, bool BAND>
 static void launch_acc_variant(deco_ctx *c, const void *grads, float alpha, cudaStream_t s)
 {
     dim3 grid(c->ntiles, c->n);
-    ef_accumulate_kernel<GT, ALIGNED, SPEC, RANDK, BAND><<<grid, BLOCK, 0, s>>>(
-        c->e, c->e_stride, grads, c->d, c->g_stride, alpha, make_rand(c), c->sel, c->stage, c->band, c->stage_cap,
-        c->tile_off, c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
+    if (BAND)
+        ef_accumulate_band_kernel<GT, ALIGNED, RANDK><<<grid, BLOCK, 0, s>>>(
+            c->e, c->e_stride, grads, c->d, c->g_stride, alpha, make_rand(c), c->sel, c->stage, c->band,
+            c->stage_cap, c->tile_off, c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
+    else
+        ef_accumulate_kernel<GT, ALIGNED, SPEC, RANDK><<<grid, BLOCK, 0, s>>>(
+            c->e, c->e_stride, grads, c->d, c->g_stride, alpha, make_rand(c), c->sel, c->stage, c->stage_cap,
+            c->tile_off, c->tile_cnt, c->tile_rej, c->tile_eq, c->ntiles);
 }
 
 template <int GT, bool ALIGNED>
@@ -2161,14 +2191,14 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     const bool walk_here = c->nchunks <= 256;
     // the kernels from here on rewrite the messages and their directory, which the previous
     // iteration's aggregation may still be reading on the internal stream
-    if (c->chain_grid >= c->n && static_cast<uint64_t>(c->n) * (2 * c->k + 65536) <= FUSED_CHAIN_MAX_PAIRS) {
+    if (walk_here && c->chain_grid >= c->n &&
+        static_cast<uint64_t>(c->n) * (2 * c->k + 65536) <= FUSED_CHAIN_MAX_PAIRS) {
         // one cooperative launch for the whole chain: as many CTAs per worker as the separate
         // kernels would use, as far as they can all be resident at once
         if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();
         uint32_t gx = sgrid.x;
         if (gx > c->chain_grid / c->n) gx = c->chain_grid / c->n;
-        uint32_t walk = walk_here ? 1u : 0u;
-        void *args[] = {&p, &walk};
+        void *args[] = {&p};
         c->launches += 1;
         return cudaLaunchCooperativeKernel(reinterpret_cast<void *>(select_chain_kernel), dim3(gx, c->n),
                                            dim3(BLOCK), args, 0, s);
