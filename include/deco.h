@@ -152,7 +152,7 @@ deco_status deco_ef_compress(deco_ctx *ctx, const void *grads, void *stream);
  * "x = x - (1/n) sum_i Delta_{t-tau}^i", kept in the server's cache of stale updates):
  * S_t[j] = sum over workers, in worker order, of the values sent for index j, stored in cache
  * slot t mod (tau_max + 1): as (index, sum) pairs, or, when the n messages together hold at
- * least d / 4 entries, as the plain vector S_t[0 .. d) (see deco_get_aggregate_vector).  Must
+ * least d / 8 entries, as the plain vector S_t[0 .. d) (see deco_get_aggregate_vector).  Must
  * follow deco_ef_compress of the same iteration.
  */
 deco_status deco_aggregate_stale(deco_ctx *ctx, void *stream);
@@ -267,7 +267,7 @@ deco_status deco_get_buffers(deco_ctx *ctx, float **e, uint64_t *e_stride, deco_
  *   deco_get_aggregate         pair layout: DEVICE pointer to `positions` pairs; positions with
  *                              idx == DECO_NO_INDEX are unused, the others hold each touched
  *                              index once (increasing) with its fp32 sum
- *   deco_get_aggregate_vector  vector layout (messages of at least d / 4 entries in all):
+ *   deco_get_aggregate_vector  vector layout (messages of at least d / 8 entries in all):
  *                              DEVICE pointer to d fp32 values, S_step[j] at j, +0 where no
  *                              worker sent j
  * Each returns DECO_ERR_STATE when the aggregate is kept in the other layout (or is not cached).

@@ -237,7 +237,7 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     // be dense enough for the plain vector S[e_stride] to be the better layout, it has room for
     // that too (a context that is one layer of a layered one keeps the pair layout only)
     c->slot_pairs = static_cast<uint64_t>(c->n_total) * c->k_cap;
-    c->dense_capable = g_stride == 0 && c->slot_pairs * 4 >= d;
+    c->dense_capable = g_stride == 0 && c->slot_pairs * 8 >= d;
     if (c->dense_capable) {
         if (c->slot_pairs < c->e_stride / 2) c->slot_pairs = c->e_stride / 2;
         c->slot_pairs = (c->slot_pairs + 31) & ~31ull;  // vectors start on 256-byte boundaries

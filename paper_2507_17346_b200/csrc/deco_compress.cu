@@ -438,6 +438,7 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         if (t == 5) p.done[i * DONE_SLOTS + 5] = 0;         // length of the emit work list
         if (i == 0 && t == 0) p.status[3] = exact_all;
         if (t == 0) {
+            s.thr_prev = s.threshold;          // the last iteration's exact threshold
             s.prefix = 0;
             s.k_rem = p.k;
             s.n_greater = 0;
@@ -1902,6 +1903,50 @@ begin_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, const 
     begin_step_body<GT, MULTI_BEGIN_GROUPS>(p, blockIdx.y % n, g, alpha, 0u, m.S, (m.S + PER_CTA - 1) / PER_CTA);
 }
 
+// Start of an iteration without a sample: the speculative bound of every (layer, worker) row is
+// carried over from the exact thresholds of the two previous iterations, T1 (last) and T2 (the
+// one before): T1, raised by half of the last rise (error feedback keeps raising the threshold
+// during the first 1/delta iterations, ever more slowly) or lowered by the whole of the last
+// fall, and then lowered by a margin of 0.04 + 1.5 / sqrt(k) octaves for the fluctuation of
+// the k-th largest magnitude between iterations.  The bound only has to be below the new
+// threshold and not too far below: the count of staged candidates checks both, and a row where
+// it fails takes the multi-pass route for this iteration, whose cost is in proportion to the
+// layer.  A quantile estimate from a sample needs about 35 / delta keys per row however short the
+// layer is, which for hundreds of rows costs more than all the selection kernels together.
+// One CTA per row: clears the row's histograms and counters and re-arms its selection record.
+__global__ void __launch_bounds__(BEGIN_BLOCK)
+carry_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
+{
+    const Sel p = table[blockIdx.x / n].p;
+    const uint32_t i = blockIdx.x % n;
+    const int t = threadIdx.x;
+    uint32_t *hz = hist_of(p, i, 0, 0);
+    for (int q = t; q < 2 * RADIX_LEVELS * RADIX_BINS; q += BEGIN_BLOCK) hz[q] = 0;
+    if (t < DONE_SLOTS && t != 3) p.done[i * DONE_SLOTS + t] = 0;
+    if (t != 0) return;
+    if (i == 0) p.status[3] = 0;
+    SelectState &s = p.sel[i];
+    const uint32_t T1 = s.threshold, T2 = s.thr_prev;
+    const double margin_oct = fmin(1.0, 0.04 + 1.5 / sqrt(static_cast<double>(p.k)));
+    const long long margin = static_cast<long long>(margin_oct * 8388608.0);     // key units per octave: 2^23
+    long long step = static_cast<long long>(T1) - static_cast<long long>(T2);
+    if (step > 0) step = step > (1ll << 23) ? (1ll << 22) : step / 2;
+    long long bound = static_cast<long long>(T1) + step - margin;
+    if (bound < 0) bound = 0;
+    if (bound > 0x7F000000ll) bound = 0x7F000000ll;
+    s.thr_prev = T1;
+    s.prefix = 0;
+    s.k_rem = p.k;
+    s.n_greater = 0;
+    s.threshold = 0;
+    s.ties_take = 0;
+    s.exact = 0;
+    s.spec_key = static_cast<uint32_t>(bound) & ~((1u << p.bound_low_bit) - 1u);
+    s.cert_key = SPEC_DISABLED;
+    s.staged_band = 0;
+    s.rel_shift = margin_oct <= 0.2 ? 10u : 12u;
+}
+
 // The streaming pass of many layers.  Its per-layer arguments travel as a kernel parameter
 // (constant bank: no dependent global load before the tile's own loads can be issued); the
 // layer of a tile is found by bisection over the layers' first tiles.  ALIGNED: the launch for
@@ -2212,10 +2257,10 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
         c->launches += 1;
     }
     if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();
-    // directory CTAs (a warp per chunk), then the CTAs whose warps stride over the work list:
-    // enough of them for one slice per warp at about 1.3 k staged entries, capped at a few
-    // waves of the device
     {
+        // directory CTAs (a warp per chunk), then the CTAs whose warps stride over the work list:
+        // enough of them for one slice per warp at about 1.3 k staged entries, capped at a few
+        // waves of the device
         const uint32_t dir_ctas = (c->nchunks + WARPS - 1) / WARPS;
         const uint64_t staged = 13 * c->k / 10, many = staged / (EMIT_LANE_MAX + 1);
         const uint64_t est_items = staged / EMIT_SLICE + (many < c->ntiles ? many : c->ntiles);
@@ -2238,6 +2283,10 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
 // Worker side of many contexts (the layers of the per-layer variant) in a fixed number of
 // launches.
 // ------------------------------------------------------------------------------------------
+// The first iterations under a policy take their bound from a sample: the thresholds on record
+// are those of another k, and right after the start they rise too fast to extrapolate.
+constexpr uint32_t CARRY_AFTER = 4;
+
 struct MultiPlan {
     std::vector<deco_ctx *> layers;
     std::vector<uint64_t> g_off;
@@ -2247,6 +2296,9 @@ struct MultiPlan {
     int grad_dtype = DECO_F32;
     uint32_t fallback_grid = 0;
     bool dirty = true;
+    // iterations run since the table was last rebuilt (a policy change): the bound is carried
+    // over once the thresholds of enough iterations under the current policy are on record
+    uint32_t age = 0;
     // streaming pass: the layers in groups of at most ACC_LAYERS_MAX, one launch (or two) each
     struct AccGroup {
         AccTable tab;
@@ -2363,7 +2415,10 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
     // the host table is pageable: the copy has left it when the call returns
     const cudaError_t err = cudaMemcpyAsync(mp->dev, mp->host.data(), sizeof(MultiLayer) * L,
                                             cudaMemcpyHostToDevice, s);
-    if (err == cudaSuccess) mp->dirty = false;
+    if (err == cudaSuccess) {
+        mp->dirty = false;
+        mp->age = 0;
+    }
     return err;
 }
 
@@ -2375,8 +2430,13 @@ cudaError_t multi_compress(MultiPlan *mp, const void *grads, float alpha, cudaSt
     }
     const uint32_t L = static_cast<uint32_t>(mp->layers.size()), n = mp->n, rows = L * n;
     const bool bf16 = mp->grad_dtype == DECO_BF16;
-    if (bf16) begin_step_multi_kernel<1><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
-    else begin_step_multi_kernel<0><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
+    if (mp->age >= CARRY_AFTER)
+        carry_step_multi_kernel<<<rows, BEGIN_BLOCK, 0, s>>>(mp->dev, n);
+    else if (bf16)
+        begin_step_multi_kernel<1><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
+    else
+        begin_step_multi_kernel<0><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
+    mp->age += 1;
     const uint64_t g_stride = mp->layers[0]->g_stride;
     for (const MultiPlan::AccGroup &grp : mp->acc) {
         const dim3 agrid(grp.tiles, n);

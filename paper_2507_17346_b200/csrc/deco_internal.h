@@ -45,7 +45,8 @@ struct SelectState {
     unsigned long long staged_band;
     uint32_t exact_total;   // cumulative count of steps that took the multi-pass path
     uint32_t rel_shift;     // log2 width of a coarse bin of the band-key histogram (10..12)
-    uint32_t pad[4];
+    uint32_t thr_prev;      // threshold of the iteration before the last one (for a carried bound)
+    uint32_t pad[3];
 };
 static_assert(sizeof(SelectState) == 64, "one line per worker");
 static_assert(offsetof(SelectState, staged_band) % 8 == 0, "64-bit atomic target");
@@ -283,10 +284,10 @@ cudaError_t launch_aggregate(deco_ctx *c, deco_pair *slot, cudaStream_t s);
 // the same with the aggregate kept as a plain vector of ntiles * TILE entries (dense messages)
 cudaError_t launch_aggregate_dense(deco_ctx *c, float *slot, cudaStream_t s);
 cudaError_t launch_apply_dense(deco_ctx *c, const float *slot, float neg_scale, cudaStream_t s);
-// dense when the messages of an iteration hold at least d / 4 entries in all
+// dense when the messages of an iteration hold at least d / 8 entries in all
 inline bool aggregate_as_vector(const deco_ctx *c, uint64_t k)
 {
-    return c->dense_capable && static_cast<uint64_t>(c->n_total) * k * 4 >= c->d;
+    return c->dense_capable && static_cast<uint64_t>(c->n_total) * k * 8 >= c->d;
 }
 cudaError_t launch_apply(deco_ctx *c, const deco_pair *slot, uint64_t positions, float neg_scale,
                          cudaStream_t s);

@@ -169,6 +169,9 @@ aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
 // Dense messages (n k entries in all comparable with d): the aggregate is kept as the plain
 // vector S[0 .. tiles * TILE) with +0 where no worker sent the index.  Same accumulator, same
 // worker order; the tile is then written out whole, with no mask and no compaction.
+constexpr int DENSE_BATCH = 4;      // workers whose entries of a tile are fetched together
+constexpr int DENSE_ROUNDS = 4;     // entries per thread and worker held at once
+
 __global__ void __launch_bounds__(BLOCK)
 aggregate_dense_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
                        const uint32_t *__restrict__ tile_start, uint64_t dir_stride, uint32_t ntiles, uint32_t n,
@@ -179,32 +182,73 @@ aggregate_dense_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     __syncthreads();
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const uint32_t first = tile * static_cast<uint32_t>(TILE);
-        for (uint32_t i = 0; i < n; ++i) {                 // worker order 0..n-1
-            const uint32_t a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
-            const uint32_t b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
-            if (b <= a) continue;                          // the same for the whole CTA
-            const deco_pair *src = msg + static_cast<size_t>(i) * k_cap;
-            for (uint32_t p0 = a; p0 < b; p0 += 4 * BLOCK) {   // four loads in flight
-                deco_pair prs[4];
+        for (uint32_t i0 = 0; i0 < n; i0 += DENSE_BATCH) {
+            // the ranges of a batch of workers, then all their entries, are fetched before the
+            // first use; the additions follow in worker order with a barrier between workers
+            uint32_t a[DENSE_BATCH], b[DENSE_BATCH];
+            bool fits = true;
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const uint32_t p = p0 + r * BLOCK + threadIdx.x;
-                    prs[r].idx = DECO_NO_INDEX;
-                    prs[r].val = 0.0f;
-                    if (p < b) prs[r] = src[p];
+            for (int w = 0; w < DENSE_BATCH; ++w) {
+                a[w] = b[w] = 0;
+                if (i0 + w < n) {
+                    a[w] = tile_start[static_cast<size_t>(i0 + w) * dir_stride + tile];
+                    b[w] = tile_start[static_cast<size_t>(i0 + w) * dir_stride + tile + 1];
                 }
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    if (prs[r].idx == DECO_NO_INDEX) continue;
-                    const uint32_t loc = prs[r].idx - first;
-                    if (loc >= static_cast<uint32_t>(TILE)) {
-                        latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, prs[r].idx);
-                        continue;
-                    }
-                    acc[loc] = acc[loc] + prs[r].val;      // indices are unique per worker
-                }
+                fits = fits && b[w] - a[w] <= static_cast<uint32_t>(DENSE_ROUNDS * BLOCK);
             }
-            __syncthreads();
+            if (fits) {
+                deco_pair pre[DENSE_BATCH][DENSE_ROUNDS];
+#pragma unroll
+                for (int w = 0; w < DENSE_BATCH; ++w)
+#pragma unroll
+                    for (int r = 0; r < DENSE_ROUNDS; ++r) {
+                        const uint32_t p = a[w] + r * BLOCK + threadIdx.x;
+                        pre[w][r].idx = DECO_NO_INDEX;
+                        pre[w][r].val = 0.0f;
+                        if (p < b[w]) pre[w][r] = msg[static_cast<size_t>(i0 + w) * k_cap + p];
+                    }
+#pragma unroll
+                for (int w = 0; w < DENSE_BATCH; ++w) {
+                    if (b[w] <= a[w]) continue;                    // the same for the whole CTA
+#pragma unroll
+                    for (int r = 0; r < DENSE_ROUNDS; ++r) {
+                        if (pre[w][r].idx == DECO_NO_INDEX) continue;
+                        const uint32_t loc = pre[w][r].idx - first;
+                        if (loc >= static_cast<uint32_t>(TILE)) {
+                            latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pre[w][r].idx);
+                            continue;
+                        }
+                        acc[loc] = acc[loc] + pre[w][r].val;       // indices are unique per worker
+                    }
+                    __syncthreads();
+                }
+                continue;
+            }
+            for (int w = 0; w < DENSE_BATCH; ++w) {                // a worker with more entries in the tile
+                if (b[w] <= a[w]) continue;
+                const deco_pair *src = msg + static_cast<size_t>(i0 + w) * k_cap;
+                for (uint32_t p0 = a[w]; p0 < b[w]; p0 += 4 * BLOCK) {   // four loads in flight
+                    deco_pair prs[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const uint32_t p = p0 + r * BLOCK + threadIdx.x;
+                        prs[r].idx = DECO_NO_INDEX;
+                        prs[r].val = 0.0f;
+                        if (p < b[w]) prs[r] = src[p];
+                    }
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        if (prs[r].idx == DECO_NO_INDEX) continue;
+                        const uint32_t loc = prs[r].idx - first;
+                        if (loc >= static_cast<uint32_t>(TILE)) {
+                            latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, prs[r].idx);
+                            continue;
+                        }
+                        acc[loc] = acc[loc] + prs[r].val;
+                    }
+                }
+                __syncthreads();
+            }
         }
         float4 *out = reinterpret_cast<float4 *>(slot + static_cast<size_t>(tile) * TILE);
         float4 *acc4 = reinterpret_cast<float4 *>(acc);
@@ -534,15 +578,33 @@ apply_kernel(const deco_pair *__restrict__ slot, uint64_t positions, float neg_s
              float *__restrict__ params, uint64_t d, uint32_t *__restrict__ status)
 {
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
-    for (uint64_t p = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-         p < positions; p += stride) {
-        const deco_pair pr = slot[p];
-        if (pr.idx == DECO_NO_INDEX) continue;
-        if (pr.idx >= d) {
-            latch(status, DECO_ERR_DEVICE_CHECK, 0x500u, pr.idx);
-            continue;
+    // four independent entries per thread and trip (the entries of a slot are distinct), so that
+    // the dependent pair -> parameter loads of four entries overlap
+    for (uint64_t p0 = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p0 < positions;
+         p0 += 4 * stride) {
+        deco_pair pr[4];
+        float x[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const uint64_t p = p0 + r * stride;
+            pr[r].idx = DECO_NO_INDEX;
+            pr[r].val = 0.0f;
+            if (p < positions) pr[r] = slot[p];
         }
-        params[pr.idx] = __fmaf_rn(neg_scale, pr.val, params[pr.idx]);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            x[r] = 0.0f;
+            if (pr[r].idx == DECO_NO_INDEX) continue;
+            if (pr[r].idx >= d) {
+                latch(status, DECO_ERR_DEVICE_CHECK, 0x500u, pr[r].idx);
+                pr[r].idx = DECO_NO_INDEX;
+                continue;
+            }
+            x[r] = params[pr[r].idx];
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+            if (pr[r].idx != DECO_NO_INDEX) params[pr[r].idx] = __fmaf_rn(neg_scale, pr[r].val, x[r]);
     }
 }
 
@@ -670,7 +732,7 @@ cudaError_t launch_apply(deco_ctx *c, const deco_pair *slot, uint64_t positions,
                          cudaStream_t s)
 {
     if (positions == 0) return cudaSuccess;
-    uint64_t blocks = (positions + 255) / 256;
+    uint64_t blocks = (positions + 4 * 256 - 1) / (4 * 256);
     if (blocks > 148ull * 16) blocks = 148ull * 16;
     apply_kernel<<<static_cast<uint32_t>(blocks), 256, 0, s>>>(slot, positions, neg_scale,
                                                                c->params, c->d, c->dev_status);

@@ -196,9 +196,12 @@ def run_layered_parity(layer_offsets, n, delta, tau, lr, grad_fn, steps, grad_dt
                     "step %d: aggregate" % t
             x = B.view_f32(info["params"], (d,), device).cpu().numpy()
             assert np.array_equal(bits(x), bits(orc.x)), "step %d: parameters" % t
+        multipass = 0
         for sub, _, _ in layers:
             st = B.deco_get_stats(sub)
             assert st["device_status"] == 0 and st["step"] == steps
+            multipass += st["exact_pass_workers"]
         assert B.deco_layered_info(ctx)["step"] == steps
+        return multipass
     finally:
         B.deco_layered_destroy(ctx)

@@ -117,7 +117,7 @@ def _check_aggregate(ctx, t, msg, S, n, k, d, rng):
     touched = torch.zeros(d, dtype=torch.bool, device="cuda")
     for i in range(n):
         touched[msg[i, :k, 0].long()] = True
-    if 4 * n * k >= d:
+    if 8 * n * k >= d:
         # dense messages: the aggregate is kept as the plain vector, +0 where nothing was sent
         vec = B.view_f32(B.deco_get_aggregate_vector(ctx, t), (d,))
         assert bool((vec.view(torch.int32) == S.view(torch.int32)).all())

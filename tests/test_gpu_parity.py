@@ -263,6 +263,33 @@ def test_per_layer_topk_short_layers_batch(kind):
                            tau_max=3, delta_max=1.0)
 
 
+def test_per_layer_bound_carried_over_between_iterations():
+    """After a few iterations under one policy the per-layer path takes its speculative bound
+    from the previous iterations' exact thresholds instead of a sample.  Stationary gradients:
+    no row may need the multi-pass route once the bound is carried (iterations 4 to 13).  Then a
+    collapse and a jump of the gradient scale, which a carried bound cannot foresee: the count of
+    staged candidates must catch both and the rows take the multi-pass route, still bit for bit."""
+    lengths = [9000, 50_000, 200_003, 8193, 31, 120_000]
+    offsets = [0]
+    for ln in lengths:
+        offsets.append(offsets[-1] + ln)
+    d, n = offsets[-1], 3
+
+    def steady(t, dtype=torch.float32):
+        return _values("normal", n, d, t, dtype)
+
+    for dtype, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        assert run_layered_parity(offsets, n, 0.01, 2, 0.1, lambda t: steady(t, dtype), steps=14,
+                                  grad_dtype=name) == 0
+
+    def jumpy(t):
+        scale = 1.0 if t < 7 else (1e-3 if t < 10 else 300.0)
+        return (steady(t) * scale).contiguous()
+
+    assert run_layered_parity(offsets, n, 0.01, 1, 0.1, jumpy, steps=13) > 0
+    run_layered_parity(offsets, n, 0.02, 1, 0.1, lambda t: _values("coarse", n, d, t, torch.float32), steps=9)
+
+
 def test_per_layer_random_k_equals_one_context_per_layer():
     """Random-k per layer (layer l draws from the stream seeded seed + l) keeps the route that
     steps every layer's context on its own; it must give what separate ordinary contexts give
@@ -550,9 +577,9 @@ def test_fused_step_with_a_long_aggregation(tau):
         assert torch.equal(B.view_i32(ba["params"], (d,)), B.view_i32(bb["params"], (d,)))
         assert torch.equal(B.view_i32(ba["e"], (n, ba["e_stride"])), B.view_i32(bb["e"], (n, bb["e_stride"])))
         for s_ in range(12 - tau, 12):                           # the aggregates still cached
-            pa, na = B.deco_get_aggregate(a, s_)
-            pb, nb = B.deco_get_aggregate(b, s_)
-            assert na == nb and torch.equal(B.view_i32(pa, (na, 2)), B.view_i32(pb, (nb, 2)))
+            va = B.view_i32(B.deco_get_aggregate_vector(a, s_), (d,))   # dense messages: vector layout
+            vb = B.view_i32(B.deco_get_aggregate_vector(b, s_), (d,))
+            assert torch.equal(va, vb)
         assert B.deco_get_stats(a)["device_status"] == 0
     finally:
         B.deco_destroy(a)
@@ -600,7 +627,7 @@ def test_checkpoint_and_resume_give_the_same_bits():
 
 @pytest.mark.parametrize("mode", MODES)
 def test_dense_messages_keep_the_aggregate_as_a_vector(mode):
-    """When the n messages hold at least d / 4 entries in all the cached aggregate is the plain
+    """When the n messages hold at least d / 8 entries in all the cached aggregate is the plain
     vector S[d] (same worker-order sums; +0 where nothing was sent) and the update sweeps it.
     The density crosses that limit in both directions at run time, with a cache of several
     slots, odd lengths and both gradient types; every buffer against the oracle."""
