@@ -438,7 +438,8 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         if (t == 5) p.done[i * DONE_SLOTS + 5] = 0;         // length of the emit work list
         if (i == 0 && t == 0) p.status[3] = exact_all;
         if (t == 0) {
-            s.thr_prev = s.threshold;          // the last iteration's exact threshold
+            s.thr_prev2 = s.thr_prev;          // the last iterations' exact thresholds
+            s.thr_prev = s.threshold;
             s.prefix = 0;
             s.k_rem = p.k;
             s.n_greater = 0;
@@ -1883,7 +1884,7 @@ struct MultiLayer {
     uint32_t S;              // sample groups of begin_step
     uint32_t walk_here;      // classification walks the chunks itself (few chunks)
     uint32_t rows_aligned;   // the layer's gradient rows start on 16-byte boundaries
-    uint32_t pad;
+    uint32_t carry;          // the layer's bound is carried over between iterations (short layers)
 };
 
 // With hundreds of (layer, worker) rows the sampling kernel is bound by the number of CTAs it
@@ -1893,10 +1894,11 @@ constexpr int MULTI_BEGIN_GROUPS = 4;
 template <int GT>
 __global__ void __launch_bounds__(BEGIN_BLOCK, 2)
 begin_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, const void *__restrict__ grads,
-                        float alpha)
+                        float alpha, uint32_t carrying)
 {
     const MultiLayer &m = table[blockIdx.y / n];
     constexpr uint32_t PER_CTA = MULTI_BEGIN_GROUPS * BEGIN_BLOCK;
+    if (carrying && m.carry) return;                         // carry_step_multi_kernel's row
     if (blockIdx.x * PER_CTA >= m.S) return;
     const Sel p = m.p;
     const char *g = static_cast<const char *>(grads) + m.g_off * (GT ? 2 : 4);
@@ -1904,19 +1906,24 @@ begin_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, const 
 }
 
 // Start of an iteration without a sample: the speculative bound of every (layer, worker) row is
-// carried over from the exact thresholds of the two previous iterations, T1 (last) and T2 (the
-// one before): T1, raised by half of the last rise (error feedback keeps raising the threshold
-// during the first 1/delta iterations, ever more slowly) or lowered by the whole of the last
-// fall, and then lowered by a margin of 0.04 + 1.5 / sqrt(k) octaves for the fluctuation of
-// the k-th largest magnitude between iterations.  The bound only has to be below the new
-// threshold and not too far below: the count of staged candidates checks both, and a row where
-// it fails takes the multi-pass route for this iteration, whose cost is in proportion to the
-// layer.  A quantile estimate from a sample needs about 35 / delta keys per row however short the
-// layer is, which for hundreds of rows costs more than all the selection kernels together.
+// carried over from the exact thresholds T1, T2, T3 of the three previous iterations (newest
+// first).  With the steps r1 = T1 - T2 and r2 = T2 - T3 (in key units, 2^23 to the octave):
+//   trend   while error feedback still raises the threshold (both steps up) three quarters of
+//           the smaller step is added: the rises shrink from iteration to iteration, and the
+//           entries that error feedback piles up just below the threshold make a bound that
+//           lags behind it stage many times k candidates; a fall is followed in full;
+//   swing   |r1 - r2|, the amplitude where the threshold moves back and forth, is subtracted;
+//   margin  0.04 + 1.5 / sqrt(k) octaves for the fluctuation of the k-th largest magnitude.
+// The bound only has to be below the new threshold and not too far below: the count of staged
+// candidates checks both, and a row where it fails takes the multi-pass route for this
+// iteration, whose cost is in proportion to the layer.  A quantile estimate from a sample needs
+// about 35 / delta keys per row however short the layer is, which for hundreds of rows costs
+// more than all the selection kernels together.
 // One CTA per row: clears the row's histograms and counters and re-arms its selection record.
 __global__ void __launch_bounds__(BEGIN_BLOCK)
 carry_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
 {
+    if (!table[blockIdx.x / n].carry) return;                // begin_step_multi_kernel's row
     const Sel p = table[blockIdx.x / n].p;
     const uint32_t i = blockIdx.x % n;
     const int t = threadIdx.x;
@@ -1926,15 +1933,20 @@ carry_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
     if (t != 0) return;
     if (i == 0) p.status[3] = 0;
     SelectState &s = p.sel[i];
-    const uint32_t T1 = s.threshold, T2 = s.thr_prev;
+    // (the multi-pass route, when a row takes it, leaves its thresholds on record as well)
+    const long long T1 = s.threshold, T2 = s.thr_prev, T3 = s.thr_prev2;
     const double margin_oct = fmin(1.0, 0.04 + 1.5 / sqrt(static_cast<double>(p.k)));
     const long long margin = static_cast<long long>(margin_oct * 8388608.0);     // key units per octave: 2^23
-    long long step = static_cast<long long>(T1) - static_cast<long long>(T2);
-    if (step > 0) step = step > (1ll << 23) ? (1ll << 22) : step / 2;
-    long long bound = static_cast<long long>(T1) + step - margin;
+    const long long r1 = T1 - T2, r2 = T2 - T3;
+    const long long trend = (r1 > 0 && r2 > 0) ? 3 * (r1 < r2 ? r1 : r2) / 4 : (r1 < 0 ? r1 : 0);
+    const long long swing = r1 > r2 ? r1 - r2 : r2 - r1;
+    long long bound = T1 + trend - swing - margin;
     if (bound < 0) bound = 0;
     if (bound > 0x7F000000ll) bound = 0x7F000000ll;
-    s.thr_prev = T1;
+    // level A resolves 4095 coarse bins above the bound: half an octave of 2^10-wide ones
+    const bool narrow = margin + swing + (trend < 0 ? -trend : trend) <= (1ll << 23) / 5;
+    s.thr_prev2 = static_cast<uint32_t>(T2);
+    s.thr_prev = static_cast<uint32_t>(T1);
     s.prefix = 0;
     s.k_rem = p.k;
     s.n_greater = 0;
@@ -1944,7 +1956,7 @@ carry_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
     s.spec_key = static_cast<uint32_t>(bound) & ~((1u << p.bound_low_bit) - 1u);
     s.cert_key = SPEC_DISABLED;
     s.staged_band = 0;
-    s.rel_shift = margin_oct <= 0.2 ? 10u : 12u;
+    s.rel_shift = narrow ? 10u : 12u;
 }
 
 // The streaming pass of many layers.  Its per-layer arguments travel as a kernel parameter
@@ -2286,6 +2298,9 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
 // The first iterations under a policy take their bound from a sample: the thresholds on record
 // are those of another k, and right after the start they rise too fast to extrapolate.
 constexpr uint32_t CARRY_AFTER = 4;
+// Layers up to this length carry their bound; longer ones keep the sample: there the sample is a
+// small part of the layer's work, and a bound that fails costs five passes over the layer.
+constexpr uint64_t CARRY_MAX_ENTRIES = 3ull << 20;
 
 struct MultiPlan {
     std::vector<deco_ctx *> layers;
@@ -2299,6 +2314,7 @@ struct MultiPlan {
     // iterations run since the table was last rebuilt (a policy change): the bound is carried
     // over once the thresholds of enough iterations under the current policy are on record
     uint32_t age = 0;
+    bool any_carry = false, any_sampled = false;     // layers on either side of CARRY_MAX_ENTRIES
     // streaming pass: the layers in groups of at most ACC_LAYERS_MAX, one launch (or two) each
     struct AccGroup {
         AccTable tab;
@@ -2365,6 +2381,7 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
         m.g_off = mp->g_off[l];
         m.S = sample_groups(c->d, c->k);
         m.walk_here = c->nchunks <= 256 ? 1u : 0u;
+        m.carry = c->d <= CARRY_MAX_ENTRIES ? 1u : 0u;
         m.rows_aligned = ((mp->g_off[l] * esz) % 16 == 0 && (c->g_stride * esz) % 16 == 0) ? 1u : 0u;
         begin_max = std::max<uint64_t>(begin_max, (m.S + MULTI_BEGIN_GROUPS * BEGIN_BLOCK - 1) /
                                                       (MULTI_BEGIN_GROUPS * BEGIN_BLOCK));
@@ -2418,6 +2435,8 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
     if (err == cudaSuccess) {
         mp->dirty = false;
         mp->age = 0;
+        mp->any_carry = mp->any_sampled = false;
+        for (const MultiLayer &m : mp->host) (m.carry ? mp->any_carry : mp->any_sampled) = true;
     }
     return err;
 }
@@ -2430,12 +2449,16 @@ cudaError_t multi_compress(MultiPlan *mp, const void *grads, float alpha, cudaSt
     }
     const uint32_t L = static_cast<uint32_t>(mp->layers.size()), n = mp->n, rows = L * n;
     const bool bf16 = mp->grad_dtype == DECO_BF16;
-    if (mp->age >= CARRY_AFTER)
-        carry_step_multi_kernel<<<rows, BEGIN_BLOCK, 0, s>>>(mp->dev, n);
-    else if (bf16)
-        begin_step_multi_kernel<1><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
-    else
-        begin_step_multi_kernel<0><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha);
+    const uint32_t carrying = (mp->age >= CARRY_AFTER && mp->any_carry) ? 1u : 0u;
+    if (carrying) carry_step_multi_kernel<<<rows, BEGIN_BLOCK, 0, s>>>(mp->dev, n);
+    if (!carrying || mp->any_sampled) {
+        if (bf16)
+            begin_step_multi_kernel<1><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha,
+                                                                                       carrying);
+        else
+            begin_step_multi_kernel<0><<<dim3(mp->begin_ctas, rows), BEGIN_BLOCK, 0, s>>>(mp->dev, n, grads, alpha,
+                                                                                       carrying);
+    }
     mp->age += 1;
     const uint64_t g_stride = mp->layers[0]->g_stride;
     for (const MultiPlan::AccGroup &grp : mp->acc) {

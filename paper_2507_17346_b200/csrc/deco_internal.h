@@ -45,8 +45,9 @@ struct SelectState {
     unsigned long long staged_band;
     uint32_t exact_total;   // cumulative count of steps that took the multi-pass path
     uint32_t rel_shift;     // log2 width of a coarse bin of the band-key histogram (10..12)
-    uint32_t thr_prev;      // threshold of the iteration before the last one (for a carried bound)
-    uint32_t pad[3];
+    uint32_t thr_prev;      // thresholds of the two iterations before the last one, newest first
+    uint32_t thr_prev2;     // (for a carried bound)
+    uint32_t pad[2];
 };
 static_assert(sizeof(SelectState) == 64, "one line per worker");
 static_assert(offsetof(SelectState, staged_band) % 8 == 0, "64-bit atomic target");
