@@ -260,10 +260,10 @@ def dtype_label(wl):
 # captured at full size; the others at reduced size (--scale) and are scaled by the entry count:
 # the kernel streams every entry once, so its traffic grows in proportion.
 NCU_TRAFFIC_BYTES = {
-    "resnet18": 1075.3e6,
-    "gpt2_small": 1585.7e6 * (995518464 / 163946496),
-    "decoder_1b": 2110.6e6 * (4400193536 / 216158400),
-    "sweep_100m": 1155.0e6 * (400000000 / 100000000),
+    "resnet18": 1072.9e6,
+    "gpt2_small": 1583.8e6 * (995518464 / 163946496),
+    "decoder_1b": 2108.3e6 * (4400193536 / 216158400),
+    "sweep_100m": 1150.4e6 * (400000000 / 100000000),
 }
 
 
