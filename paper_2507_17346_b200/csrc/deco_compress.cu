@@ -938,9 +938,11 @@ __device__ void scan_tiles_body(const Sel &p, uint32_t i, uint32_t *s_w, bool st
 constexpr uint32_t EMIT_SLICE = 256;
 constexpr uint32_t EMIT_LANE_MAX = 16;
 
-__device__ __forceinline__ uint32_t emit_items_of(uint32_t cnt)
+// whole_tiles: with dense messages every tile holds hundreds of staged entries and there are
+// tiles enough to fill the machine: one warp walks the whole tile (no slice is read twice).
+__device__ __forceinline__ uint32_t emit_items_of(uint32_t cnt, bool whole_tiles)
 {
-    return cnt > EMIT_LANE_MAX ? (cnt + EMIT_SLICE - 1) / EMIT_SLICE : 0u;
+    return cnt > EMIT_LANE_MAX ? (whole_tiles ? 1u : (cnt + EMIT_SLICE - 1) / EMIT_SLICE) : 0u;
 }
 
 // Work list of a worker: one (tile, slice) entry per slice; every thread looks at one tile, a
@@ -955,7 +957,7 @@ __device__ __forceinline__ void build_emit_work(const Sel &p, uint32_t i)
     for (uint32_t tile = blockIdx.x * BLOCK + threadIdx.x; tile < tiles_up;
          tile += gridDim.x * BLOCK) {
         const uint32_t items =
-            tile < p.ntiles ? emit_items_of(p.tile_cnt[static_cast<size_t>(i) * p.ntiles + tile]) : 0u;
+            tile < p.ntiles ? emit_items_of(p.tile_cnt[static_cast<size_t>(i) * p.ntiles + tile], p.use_band != 0) : 0u;
         const uint32_t incl = warp_incl_scan(items);
         const uint32_t total = __shfl_sync(FULL, incl, 31);
         if (total == 0) continue;
@@ -1207,7 +1209,7 @@ __global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p)
 }
 
 // Classification.  With the threshold known every band entry below it is rejected: counted
-// for its tile and given its value back in e; entries equal to it are counted as ties.  (The
+// for its tile; entries equal to it are counted as ties.  (The
 // candidates above the band are above the threshold.)  With few chunks (walk_here) the last
 // CTA of a worker to arrive then walks the chunks once; with many, the chunk sums follow.
 // (The per-tile positions follow from these inside the emit step, so nothing here is serial
@@ -1223,7 +1225,6 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
     const deco_pair *src = select_list(p, i, n_staged, n_band);
     uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
-    float *erow = p.e + static_cast<size_t>(i) * p.e_stride;
     const int lane = threadIdx.x & 31;
     for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
          base += gridDim.x * (4 * BLOCK)) {
@@ -1248,27 +1249,9 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
                 atomicAdd(cls == 1 ? &rej[tile] : &eqc[tile], static_cast<uint32_t>(__popc(grp)));
         }
     }
-    const bool last = last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &sm.misc[2]);
-    // after the arrival, off the critical path: undo the +0 guess for the rejected entries
-    auto write_back_rejected = [&]() {
-        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
-             base += gridDim.x * (4 * BLOCK)) {
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const uint32_t q = base + r * BLOCK + threadIdx.x;
-                if (q < n_band) {
-                    const deco_pair pr = src[q];
-                    if (key_of(p, i, pr) < T && pr.idx < p.d) erow[pr.idx] = pr.val;
-                }
-            }
-        }
-    };
-    if (!last) {
-        write_back_rejected();
-        return;
-    }
+    // (the rejected entries get their value back in e from emit, which reads every staged pair anyway)
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &sm.misc[2])) return;
     if (walk_here) chunk_walk(p, i, sm.scan, false);
-    write_back_rejected();
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_classify_kernel(Sel p, uint32_t walk_here)
@@ -1319,7 +1302,8 @@ __device__ __forceinline__ TileInfo chunk_header(const Sel &p, uint32_t i, uint3
 
 // The whole warp filters staged entries [begin, end) of one tile's segment, in order, into the
 // message; `written` entries of the tile were emitted and `ties_seen` ties met before `begin`.
-// The selected entries are already +0 in e; ties that are not taken get their value back.
+// The selected entries are already +0 in e; the others (below the threshold, or ties that are not
+// taken) get their value back: the +0 guess of the streaming pass is undone here.
 // Returns the number of entries written.
 __device__ __forceinline__ uint32_t emit_segment_warp(const Sel &p, uint32_t i, uint32_t tile,
                                                       uint32_t off, uint32_t begin, uint32_t end,
@@ -1343,7 +1327,8 @@ __device__ __forceinline__ uint32_t emit_segment_warp(const Sel &p, uint32_t i, 
         for (int r = 0; r < 4; ++r) {
             const deco_pair pr = prs[r];
             bool gt = false, eq = false;
-            if (base + r * 32 + lane < end) {
+            const bool in = base + r * 32 + lane < end;
+            if (in) {
                 const uint32_t key = key_of(p, i, pr);
                 gt = key > T;
                 eq = key == T;
@@ -1360,7 +1345,7 @@ __device__ __forceinline__ uint32_t emit_segment_warp(const Sel &p, uint32_t i, 
                     latch(p.status, DECO_ERR_DEVICE_CHECK, 0x310u, tile);
                 }
             }
-            if (eq && !pick && pr.idx < p.d) erow[pr.idx] = pr.val;   // tie not taken: undo the guess
+            if (in && !pick && pr.idx < p.d) erow[pr.idx] = pr.val;   // not selected: undo the guess
             written += __popc(pick_mask);
             ties_seen += __popc(eq_mask);
         }
@@ -1395,8 +1380,8 @@ __device__ __forceinline__ void emit_directory_part(const Sel &p, const uint32_t
                 const uint32_t pos = t.start + written++;
                 if (pos < p.k && pr.idx < p.d) out[pos] = pr;
                 else latch(p.status, DECO_ERR_DEVICE_CHECK, 0x312u, tile);
-            } else if (eq && pr.idx < p.d) {
-                erow[pr.idx] = pr.val;                       // tie not taken: undo the guess
+            } else if (pr.idx < p.d) {
+                erow[pr.idx] = pr.val;                       // not selected: undo the guess
             }
         }
         if (written != t.sel) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x313u, tile);
@@ -1426,12 +1411,13 @@ __device__ __forceinline__ void emit_items_part(const Sel &p, const uint32_t i, 
         const uint32_t cnt = __shfl_sync(FULL, t.cnt, my), start = __shfl_sync(FULL, t.start, my);
         const uint32_t want = __shfl_sync(FULL, t.sel, my), take = __shfl_sync(FULL, t.take, my);
         const uint32_t off = p.tile_off[static_cast<size_t>(i) * p.ntiles + tile];
-        const uint32_t begin = slice * EMIT_SLICE;
+        const uint32_t slice_len = p.use_band ? static_cast<uint32_t>(TILE) : EMIT_SLICE;
+        const uint32_t begin = slice * slice_len;
         if (begin >= cnt) {
             if (lane == 0) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x322u, tile);
             continue;
         }
-        const uint32_t end = min(cnt, begin + EMIT_SLICE);
+        const uint32_t end = min(cnt, begin + slice_len);
         uint32_t written = 0, ties_seen = 0;
         if (begin) {
             // what slices 0..slice-1 emit: the entries above the threshold plus the ties
