@@ -440,6 +440,7 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         if (t == 0) {
             s.thr_prev2 = s.thr_prev;          // the last iterations' exact thresholds
             s.thr_prev = s.threshold;
+            s.swing = 0;
             s.prefix = 0;
             s.k_rem = p.k;
             s.n_greater = 0;
@@ -1898,7 +1899,9 @@ begin_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, const 
 //           the smaller step is added: the rises shrink from iteration to iteration, and the
 //           entries that error feedback piles up just below the threshold make a bound that
 //           lags behind it stage many times k candidates; a fall is followed in full;
-//   swing   |r1 - r2|, the amplitude where the threshold moves back and forth, is subtracted;
+//   swing   |r1 - r2|, the amplitude where the threshold moves back and forth, is subtracted
+//           (kept as a maximum that decays by a quarter per iteration: a row whose threshold
+//           has swung keeps a wider berth for some iterations);
 //   margin  0.04 + 1.5 / sqrt(k) octaves for the fluctuation of the k-th largest magnitude.
 // The bound only has to be below the new threshold and not too far below: the count of staged
 // candidates checks both, and a row where it fails takes the multi-pass route for this
@@ -1925,7 +1928,11 @@ carry_step_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
     const long long margin = static_cast<long long>(margin_oct * 8388608.0);     // key units per octave: 2^23
     const long long r1 = T1 - T2, r2 = T2 - T3;
     const long long trend = (r1 > 0 && r2 > 0) ? 3 * (r1 < r2 ? r1 : r2) / 4 : (r1 < 0 ? r1 : 0);
-    const long long swing = r1 > r2 ? r1 - r2 : r2 - r1;
+    long long swing = r1 > r2 ? r1 - r2 : r2 - r1;
+    const long long remembered = 3 * static_cast<long long>(s.swing) / 4;
+    if (swing < remembered) swing = remembered;
+    if (swing > (1ll << 24)) swing = 1ll << 24;
+    s.swing = static_cast<uint32_t>(swing);
     long long bound = T1 + trend - swing - margin;
     if (bound < 0) bound = 0;
     if (bound > 0x7F000000ll) bound = 0x7F000000ll;

@@ -47,7 +47,8 @@ struct SelectState {
     uint32_t rel_shift;     // log2 width of a coarse bin of the band-key histogram (10..12)
     uint32_t thr_prev;      // thresholds of the two iterations before the last one, newest first
     uint32_t thr_prev2;     // (for a carried bound)
-    uint32_t pad[2];
+    uint32_t swing;         // decaying maximum of the threshold's change of step, in key units
+    uint32_t pad[1];
 };
 static_assert(sizeof(SelectState) == 64, "one line per worker");
 static_assert(offsetof(SelectState, staged_band) % 8 == 0, "64-bit atomic target");
