@@ -64,6 +64,7 @@ void free_all(deco_ctx *c)
     cudaFree(c->chunk_start);
     cudaFree(c->sample_keys);
     cudaFree(c->sample_hist);
+    cudaFree(c->sample_win);
     cudaFree(c->done);
     cudaFree(c->dev_status);
     cudaFree(c->grads_staging);
@@ -88,6 +89,8 @@ deco_status zero_state(deco_ctx *c, cudaStream_t s)
         err = cudaMemsetAsync(c->done, 0, sizeof(uint32_t) * c->n * DONE_SLOTS, s);
     if (err == cudaSuccess)
         err = cudaMemsetAsync(c->sample_hist, 0, sizeof(uint32_t) * c->n * SAMPLE_BINS, s);
+    if (err == cudaSuccess)
+        err = cudaMemsetAsync(c->sample_win, 0, sizeof(uint32_t) * c->n * WINDOW_WORDS, s);
     if (err == cudaSuccess)
         err = c->packed ? cudaMemsetAsync(c->xchg, 0, sizeof(uint32_t) * c->n_total * c->xrow_cap, s)
                         : cudaMemsetAsync(c->tile_start, 0, sizeof(uint32_t) * c->n * (c->ntiles + 1), s);
@@ -251,6 +254,7 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
     need(dev_alloc(c, &c->done, static_cast<uint64_t>(n) * DONE_SLOTS));
     need(dev_alloc(c, &c->sample_keys, static_cast<uint64_t>(n) * SAMPLE_KEYS));
     need(dev_alloc(c, &c->sample_hist, static_cast<uint64_t>(n) * SAMPLE_BINS));
+    need(dev_alloc(c, &c->sample_win, static_cast<uint64_t>(n) * WINDOW_WORDS));
     need(dev_alloc(c, &c->sel, n));
     need(dev_alloc(c, &c->tile_gt, static_cast<uint64_t>(n) * c->ntiles));
     need(dev_alloc(c, &c->tile_eq, static_cast<uint64_t>(n) * c->ntiles));

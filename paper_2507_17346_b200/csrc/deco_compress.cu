@@ -94,6 +94,7 @@ struct Sel {
     uint32_t *done;          // [n][DONE_SLOTS] CTA arrival counters
     uint32_t *sample_keys;   // [n][4 * SAMPLE_CHUNKS] keys of the sample
     uint32_t *sample_hist;   // [n][SAMPLE_BINS] sample keys per bin of their top bits; cleared by its reader
+    uint32_t *sample_win;    // [n][WINDOW_WORDS] fine histogram around the previous bound; cleared by its reader
     uint32_t *tile_gt, *tile_eq, *tile_take, *tile_start, *tile_off, *tile_cnt, *tile_rej;
     uint32_t nchunks;        // chunks of CHUNK_TILES tiles
     uint32_t *chunk_cnt, *chunk_rej, *chunk_eq;   // [n][nchunks] staged / rejected / ties
@@ -397,7 +398,9 @@ constexpr int SAMPLE_BINS_PER_THREAD = SAMPLE_HIST_BINS / BEGIN_BLOCK;
 constexpr int SAMPLE_WARP_LIST = 256;                      // list slots per warp in the search
 static_assert(4 * SAMPLE_CHUNKS == SAMPLE_KEYS, "sample buffer size");
 static_assert(SAMPLE_HIST_BINS == SAMPLE_BINS, "sample histogram size");
-static_assert(SAMPLE_HIST_BINS <= (BEGIN_BLOCK / 32) * SAMPLE_WARP_LIST, "histogram shares the list storage");
+static_assert(SAMPLE_HIST_BINS + WINDOW_WORDS <= (BEGIN_BLOCK / 32) * SAMPLE_WARP_LIST,
+              "both histograms share the list storage");
+static_assert((WINDOW_BINS << WINDOW_SUB_BITS) == BEGIN_BLOCK, "one fine bin per thread of the last CTA");
 
 // Number of sample groups S.  A group costs two random line fetches (e and g); a candidate
 // that is staged and then rejected costs about as much (its +0 guess is undone), and their
@@ -467,6 +470,15 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
                        static_cast<size_t>(i) * p.g_stride * (GT ? 2 : 4);
     const uint64_t nchunks = (p.d + 3) >> 2;
     uint4 *skeys = reinterpret_cast<uint4 *>(p.sample_keys) + static_cast<size_t>(i) * SAMPLE_CHUNKS;
+    // Window of WINDOW_BINS coarse bins (one octave) around the previous iteration's bound, each
+    // bin cut into 64: when the sampled ranks fall inside it (they do unless the gradients'
+    // scale jumps) the last CTA reads the bounds off this histogram and never looks at the
+    // sample keys again.  hint_key was written by the previous launch; nothing writes it here
+    // before the last CTA does.
+    const uint32_t hint_bin = min(s.hint_key >> p.sample_shift, SAMPLE_HIST_BINS - 1);
+    const uint32_t win_lo = min(hint_bin > WINDOW_BINS / 2 ? hint_bin - WINDOW_BINS / 2 : 0u,
+                                SAMPLE_HIST_BINS - WINDOW_BINS);
+    uint32_t *s_win = s_buf + SAMPLE_HIST_BINS;               // WINDOW_WORDS words behind the coarse histogram
     {
         // G sample groups per thread, all loads issued before the first use
         uint32_t kk[G][4];
@@ -500,7 +512,9 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         // with the same bin elect one of them to add the group's size
 #pragma unroll
         for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) s_buf[c * BEGIN_BLOCK + t] = 0;
+        for (uint32_t q = t; q < WINDOW_WORDS; q += BEGIN_BLOCK) s_win[q] = 0;
         __syncthreads();
+        uint32_t above_window = 0;
 #pragma unroll
         for (int gq = 0; gq < G; ++gq) {
 #pragma unroll
@@ -509,13 +523,27 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
                 const uint32_t hb = key ? min(key >> p.sample_shift, SAMPLE_HIST_BINS - 1) : SAMPLE_HIST_BINS;
                 const uint32_t grp = __match_any_sync(FULL, hb);
                 if (hb < SAMPLE_HIST_BINS && (t & 31) == __ffs(grp) - 1) atomicAdd(&s_buf[hb], __popc(grp));
+                if (hb < SAMPLE_HIST_BINS && hb >= win_lo) {
+                    if (hb >= win_lo + WINDOW_BINS) {
+                        above_window += 1;
+                    } else {
+                        const uint32_t sub = (key >> (p.sample_shift - WINDOW_SUB_BITS)) & ((1u << WINDOW_SUB_BITS) - 1u);
+                        atomicAdd(&s_win[((hb - win_lo) << WINDOW_SUB_BITS) + sub], 1u);
+                    }
+                }
             }
         }
+        above_window = __reduce_add_sync(FULL, above_window);
+        if ((t & 31) == 0 && above_window) atomicAdd(&s_win[WINDOW_WORDS - 1], above_window);
         __syncthreads();
 #pragma unroll
         for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) {
             const uint32_t v = s_buf[c * BEGIN_BLOCK + t];
             if (v) atomicAdd(&p.sample_hist[i * SAMPLE_HIST_BINS + c * BEGIN_BLOCK + t], v);
+        }
+        for (uint32_t q = t; q < WINDOW_WORDS; q += BEGIN_BLOCK) {
+            const uint32_t v = s_win[q];
+            if (v) atomicAdd(&p.sample_win[i * WINDOW_WORDS + q], v);
         }
     }
     // the arrival counter resets itself: only the last CTA touches it afterwards
@@ -545,11 +573,52 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         if (p.rk.on) rel_shift = 10u;          // uniform 23-bit priorities: 4095 << 10 is half the range
     }
     uint32_t *gh = p.sample_hist + i * SAMPLE_HIST_BINS;
+    uint32_t *gw = p.sample_win + i * WINDOW_WORDS;
+    // fine bin WINDOW-1-t of the window belongs to thread t, so that the prefix over threads
+    // counts the sample keys in higher fine bins; both histograms are left cleared
+    const uint32_t fine = (WINDOW_BINS << WINDOW_SUB_BITS) - 1u - t;
+    const uint32_t in_fine = __ldcg(&gw[fine]);
+    const uint32_t above_window = __ldcg(&gw[WINDOW_WORDS - 1]);
+    gw[fine] = 0;
     if (R > m_total) {                         // the sample cannot bound the threshold
-        if (t == 0) s.spec_key = 0;            // stage everything: the count check decides
+        if (t == 0) {
+            s.spec_key = 0;                    // stage everything: the count check decides
+            s.hint_key = 0;
+            gw[WINDOW_WORDS - 1] = 0;
+        }
 #pragma unroll
         for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) gh[c * BEGIN_BLOCK + t] = 0;
         return;
+    }
+    {
+        // Both sampled ranks inside the window: the bounds are edges of its fine bins (1/1024 of
+        // an octave wide), and the sample keys are not looked at again.
+        uint32_t tot;
+        const uint32_t higher = above_window + block_excl_scan(in_fine, s_w, tot);
+        if (t == 0) {
+            s_flag = 0xFFFFFFFFu;
+            s_hi = R_hi ? 0xFFFFFFFFu : SPEC_DISABLED;
+            gw[WINDOW_WORDS - 1] = 0;
+        }
+        __syncthreads();
+        const uint32_t sub_shift = p.sample_shift - WINDOW_SUB_BITS;
+        const uint32_t edge = ((win_lo << WINDOW_SUB_BITS) + fine) << sub_shift;     // lower edge of my fine bin
+        if (higher < R && higher + in_fine >= R) s_flag = edge;
+        if (R_hi && higher < R_hi && higher + in_fine >= R_hi) s_hi = edge + (1u << sub_shift);
+        __syncthreads();
+        const uint32_t w_bound = s_flag, w_cert = s_hi;
+        __syncthreads();
+        if (w_bound != 0xFFFFFFFFu && w_cert != 0xFFFFFFFFu) {
+#pragma unroll
+            for (int c = 0; c < SAMPLE_BINS_PER_THREAD; ++c) gh[c * BEGIN_BLOCK + t] = 0;
+            if (t == 0) {
+                s.spec_key = w_bound;
+                s.cert_key = w_cert;
+                s.rel_shift = rel_shift;
+                s.hint_key = w_bound;
+            }
+            return;
+        }
     }
     // Largest key prefix v (a multiple of 2^bound_low_bit) with  #(sample keys >= v) >= R.
     // The top bits come from the histogram the sampling CTAs filled: thread t looks at bins
@@ -681,6 +750,7 @@ __device__ __forceinline__ void begin_step_body(const Sel &p, const uint32_t i, 
         s.spec_key = bound;                    // lower edge of a 2^bound_low_bit-wide key bin
         s.cert_key = s_hi;                     // above the bound's own histogram bin
         s.rel_shift = rel_shift;
+        s.hint_key = bound;                    // centre of the next iteration's window
     }
 }
 
@@ -2084,6 +2154,7 @@ Sel make_sel(const deco_ctx *c)
     p.done = c->done;
     p.sample_keys = c->sample_keys;
     p.sample_hist = c->sample_hist;
+    p.sample_win = c->sample_win;
     p.tile_gt = c->tile_gt;
     p.tile_eq = c->tile_eq;
     p.tile_take = c->tile_take;

@@ -48,7 +48,7 @@ struct SelectState {
     uint32_t thr_prev;      // thresholds of the two iterations before the last one, newest first
     uint32_t thr_prev2;     // (for a carried bound)
     uint32_t swing;         // decaying maximum of the threshold's change of step, in key units
-    uint32_t pad[1];
+    uint32_t hint_key;      // the last iteration's speculative bound: where the sample's fine histogram is centred
 };
 static_assert(sizeof(SelectState) == 64, "one line per worker");
 static_assert(offsetof(SelectState, staged_band) % 8 == 0, "64-bit atomic target");
@@ -62,6 +62,11 @@ constexpr uint32_t CHUNK_TILES = 32;
 // Keys of the per-iteration sample kept per worker (8192 groups of 4 entries).
 constexpr uint32_t SAMPLE_KEYS = 131072;
 constexpr uint32_t SAMPLE_BINS = 4096;                  // bins of the sample histogram
+// Fine histogram of the sample around the previous bound: WINDOW_BINS coarse bins, each cut into
+// 64, one counter each; one more word counts the sample keys above the window.
+constexpr uint32_t WINDOW_BINS = 16;
+constexpr uint32_t WINDOW_SUB_BITS = 6;
+constexpr uint32_t WINDOW_WORDS = (WINDOW_BINS << WINDOW_SUB_BITS) + 1;
 
 struct Slot {
     uint64_t step = 0;
@@ -125,6 +130,7 @@ struct deco_ctx {
     uint32_t *done = nullptr;           // [n][DONE_SLOTS] CTA arrival counters
     uint32_t *sample_keys = nullptr;    // [n][SAMPLE_KEYS] keys of the per-iteration sample
     uint32_t *sample_hist = nullptr;    // [n][SAMPLE_BINS] sample keys per bin of their top bits (self-clearing)
+    uint32_t *sample_win = nullptr;     // [n][WINDOW_WORDS] fine histogram around the previous bound (self-clearing)
     uint32_t fallback_grid = 0;         // CTAs of the cooperative fallback launch
     uint32_t chain_grid = 0;            // most CTAs the cooperative selection launch may have
     deco::SelectState *sel = nullptr;   // [n]
