@@ -10,9 +10,12 @@
 // on the guess that they will be selected.  The exact threshold is then found by a two-level
 // radix selection over the staged pairs only (on key - spec_key), a classification pass counts
 // the rejected entries and the ties per tile and per chunk of tiles, the message is an ordered
-// filter of the staged pairs, and the few that are not selected get their value back.
-// The count of staged pairs proves the bound was valid (>= k of them); if it was not, or the
-// staging area overflowed, that worker takes the second route in the same call.
+// filter of the staged pairs, and the staged entries that are not selected get their value back
+// as the filter passes over them.  The count of staged pairs proves the bound was valid (>= k of
+// them); if it was not, or the staging area overflowed, that worker takes the second route in
+// the same call.  For dense messages (delta >= 1/32) the sample also fixes an upper bound
+// `cert_key` of the threshold: staged entries above it are selected for certain (again proved by
+// a count), and the selection and classification read only the band between the two bounds.
 //
 // Multi-pass route (DECO_SELECT_EXACT_PASSES, and the fallback of the first): three radix
 // histogram passes over e fix the threshold key, one pass counts per tile, one pass emits.
