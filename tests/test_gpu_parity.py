@@ -352,28 +352,29 @@ def test_per_layer_seeded_random_partitions(seed):
                            delta_max=max(delta, delta2))
 
 
-@pytest.mark.parametrize("compressor", ["topk", "randk"])
-def test_worker_sharded_contexts_equal_the_single_job(compressor):
+@pytest.mark.parametrize("compressor,delta,delta2", [("topk", 0.004, 0.02), ("randk", 0.004, 0.02),
+                                                     ("topk", 0.06, 0.01)])
+def test_worker_sharded_contexts_equal_the_single_job(compressor, delta, delta2):
     """Five workers split 2 + 3 over two contexts on one GPU.  Each compresses its own workers;
     the rows of the exchange buffer are then copied across (what the all-gather does
     between GPUs), and both replicas aggregate and update.  Local messages and residuals, the
     aggregate and both parameter replicas must equal the oracle's single five-worker job."""
     from oracle import dd_ef_sgd as O
     from tests.parity import bits, read_aggregate, read_e, read_messages, read_params
-    d, n, delta, tau, lr = 70_004, 5, 0.004, 1, 0.1
+    d, n, tau, lr = 70_004, 5, 1, 0.1
     split = [(0, 2), (2, 3)]
     comp = B.DECO_COMPRESSOR_RANDK if compressor == "randk" else B.DECO_COMPRESSOR_TOPK
     ctxs = [B.deco_init(d, cnt, delta, tau, lr, n_total=n, worker_base=base, compressor=comp,
-                        seed=99, tau_max=2, delta_max=0.02) for base, cnt in split]
+                        seed=99, tau_max=2, delta_max=max(delta, delta2)) for base, cnt in split]
     orc = O.DDEFSGD(d, n, delta, tau, lr, compressor=compressor, seed=99)
     try:
         with pytest.raises(B.DecoError):
             B.deco_step(ctxs[0], torch.zeros((2, d), device="cuda"))
         for t in range(6):
-            if t == 3:
+            if t == 3:                                   # the rows change length (and the aggregate its layout)
                 for c in ctxs:
-                    B.deco_set_policy(c, 0.02, 2)
-                orc.set_policy(0.02, 2)
+                    B.deco_set_policy(c, delta2, 2)
+                orc.set_policy(delta2, 2)
             g = _values("normal", n, d, t, torch.float32)
             ref = orc.step(W.to_numpy_bits(g))
             views = []
@@ -396,7 +397,7 @@ def test_worker_sharded_contexts_equal_the_single_job(compressor):
                     assert np.array_equal(bits(val[i]), bits(ref["msgs"][base + i][1]))
                 assert np.array_equal(bits(read_e(c, cnt, d)), bits(orc.e[base:base + cnt]))
                 B.deco_aggregate_stale(c)
-                aidx, aval = read_aggregate(c, t)
+                aidx, aval = read_aggregate(c, t, 0, d, touched)
                 assert np.array_equal(aidx, touched), t
                 assert np.array_equal(bits(aval), bits(ref["S"][touched])), t
                 B.deco_apply_update(c)
