@@ -615,7 +615,7 @@ def run_ours(args):
         others = {}
         for name in OTHER_WORKLOADS:
             owl = workload_for(args, name)
-            osteps = min(default_steps(grad_bytes(owl)), 400)
+            osteps = min(default_steps(grad_bytes(owl)), 150)
             r = time_workload(B, W, owl, args, osteps, 10, local, world, rank, dist)
             others[name] = summary_of(r, owl)
         others["sweep_100m"]["delta_tau_grid_and_adaptive_run"] = run_sweep(B, W, args, local)
