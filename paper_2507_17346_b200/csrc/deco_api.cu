@@ -74,6 +74,7 @@ void free_all(deco_ctx *c)
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->ev_emit) cudaEventDestroy(c->ev_emit);
     if (c->ev_agg) cudaEventDestroy(c->ev_agg);
+    if (c->ev_pass) cudaEventDestroy(c->ev_pass);
     if (c->side_stream) cudaStreamDestroy(c->side_stream);
     if (c->agg_stream) cudaStreamDestroy(c->agg_stream);
 }
@@ -107,6 +108,10 @@ inline cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
 // cache or the device status from the host, or hand out pointers).
 inline cudaError_t drain_internal(deco_ctx *c)
 {
+    if (c->agg_deferred) {
+        const cudaError_t err = launch_deferred_aggregate(c);
+        if (err != cudaSuccess) return err;
+    }
     c->agg_pending = false;
     if (!c->side_stream) return cudaSuccess;
     const cudaError_t err = cudaStreamSynchronize(c->side_stream);
@@ -129,6 +134,24 @@ void mark(deco_ctx *c, int which, cudaStream_t s)
 }
 
 }  // namespace
+
+cudaError_t deco::launch_deferred_aggregate(deco_ctx *c)
+{
+    if (!c->agg_deferred) return cudaSuccess;
+    c->agg_deferred = false;
+    // ev_emit: the messages of that iteration are complete
+    cudaError_t err = cudaStreamWaitEvent(c->agg_stream, c->ev_emit, 0);
+    if (err != cudaSuccess) return err;
+    deco_pair *slot = c->slots + static_cast<uint64_t>(c->agg_slot) * c->slot_pairs;
+    mark(c, 3, c->agg_stream);
+    err = c->agg_dense ? launch_aggregate_dense(c, reinterpret_cast<float *>(slot), c->agg_stream)
+                       : launch_aggregate(c, slot, c->agg_stream);
+    if (err != cudaSuccess) return err;
+    mark(c, 4, c->agg_stream);
+    err = cudaEventRecord(c->ev_agg, c->agg_stream);
+    c->agg_pending = true;
+    return err;
+}
 
 extern "C" const char *deco_status_string(deco_status s)
 {
@@ -279,7 +302,8 @@ deco_status deco::init_context(deco_ctx **out, uint64_t d, uint32_t n, double de
          cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
          cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
          cudaEventCreateWithFlags(&c->ev_emit, cudaEventDisableTiming) != cudaSuccess ||
-         cudaEventCreateWithFlags(&c->ev_agg, cudaEventDisableTiming) != cudaSuccess))
+         cudaEventCreateWithFlags(&c->ev_agg, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&c->ev_pass, cudaEventDisableTiming) != cudaSuccess))
         st = DECO_ERR_CUDA;
     if (st == DECO_OK) st = zero_state(c, nullptr);
     if (st == DECO_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) st = DECO_ERR_CUDA;
@@ -482,37 +506,84 @@ extern "C" deco_status deco_step(deco_ctx *c, const void *grads, void *stream)
         if (st == DECO_OK) st = deco_apply_update(c, stream);
         return st;
     }
-    // tau >= 1: the aggregates due now were cached in earlier iterations and touch neither e
-    // nor the messages, so their update runs on an internal stream next to the streaming
-    // pass.  It is forked from and joined back into the caller's stream inside this call: e,
-    // the messages and the parameters are complete, in stream order, when the caller's stream
-    // passes the call.
     if (reinterpret_cast<uintptr_t>(grads) & (c->g_stride != c->d ? 1u : 15u)) return DECO_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);
-    if (cudaEventRecord(c->ev_fork, s) != cudaSuccess) return DECO_ERR_CUDA;
-    if (cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0) != cudaSuccess) return DECO_ERR_CUDA;
-    // the only aggregation that can still be running is that of iteration t - 1, which is
-    // due now only if tau = 1
-    if (c->tau <= 1 && cudaStreamWaitEvent(c->side_stream, c->ev_agg, 0) != cudaSuccess)
-        return DECO_ERR_CUDA;
-    mark(c, 5, c->side_stream);
-    deco_status st = apply_due(c, c->side_stream);
-    mark(c, 6, c->side_stream);
-    if (cudaEventRecord(c->ev_join, c->side_stream) != cudaSuccess) return DECO_ERR_CUDA;
-    if (st == DECO_OK) st = deco_ef_compress(c, grads, stream);
-    if (st != DECO_OK) return st;
-    // This iteration's aggregate is not needed before iteration t + tau: it goes onto a second
-    // internal stream behind the messages and may run next to whatever the caller's stream
-    // does next (the streaming pass of the following iteration).  Every later launch that
-    // rewrites the messages or reads the cache orders itself after ev_agg.
+    // Where the server side of an iteration runs.  The streaming pass keeps the whole register
+    // file busy, and a kernel beside it only displaces its CTAs; the selection that follows it
+    // is a chain of short launches.  When that chain is separate launches, the server side
+    // goes behind the pass: the aggregation of the previous iteration's messages (booked then,
+    // launched now; this iteration's emit, which rewrites the messages, waits for it) and the
+    // update with the aggregates that are due (cached in earlier iterations; it touches neither
+    // e nor the messages).  When the chain is one cooperative launch (short vectors), which
+    // would wait for every other kernel to leave the device, the update is forked off at the
+    // start and the aggregation is launched right behind the emit, next to the following pass.
+    // Either way the update is joined back into the caller's stream inside this call: e, the
+    // messages and the parameters are complete, in stream order, when the caller's stream
+    // passes the call.
+    const bool behind_pass = selection_is_separate_launches(c);
+    c->k_of_msg = c->k;
+    set_message_layout(c, c->k);
+    deco_status st = DECO_OK;
+    if (!behind_pass) {
+        if (cudaEventRecord(c->ev_fork, s) != cudaSuccess) return DECO_ERR_CUDA;
+        if (cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0) != cudaSuccess) return DECO_ERR_CUDA;
+        // the only aggregation that can still be outstanding is that of iteration t - 1,
+        // which is due now only if tau = 1
+        if (c->tau <= 1) {
+            if (launch_deferred_aggregate(c) != cudaSuccess) return DECO_ERR_CUDA;
+            if (c->agg_pending && cudaStreamWaitEvent(c->side_stream, c->ev_agg, 0) != cudaSuccess)
+                return DECO_ERR_CUDA;
+        }
+        mark(c, 5, c->side_stream);
+        st = apply_due(c, c->side_stream);
+        mark(c, 6, c->side_stream);
+        if (cudaEventRecord(c->ev_join, c->side_stream) != cudaSuccess) return DECO_ERR_CUDA;
+        if (st != DECO_OK) return st;
+    }
+    cudaError_t err = launch_begin_step(c, grads, s);
+    mark(c, 0, s);
+    if (err == cudaSuccess) err = launch_accumulate(c, grads, s);
+    mark(c, 1, s);
+    if (err == cudaSuccess) err = cudaEventRecord(c->ev_pass, s);
+    if (err != cudaSuccess) return DECO_ERR_CUDA;
+    if (c->agg_deferred) {
+        if (cudaStreamWaitEvent(c->agg_stream, c->ev_pass, 0) != cudaSuccess) return DECO_ERR_CUDA;
+        if (launch_deferred_aggregate(c) != cudaSuccess) return DECO_ERR_CUDA;
+    } else if (behind_pass) {
+        mark(c, 3, c->agg_stream);          // nothing to aggregate: an empty interval
+        mark(c, 4, c->agg_stream);
+    }
+    if (behind_pass) {
+        if (cudaStreamWaitEvent(c->side_stream, c->ev_pass, 0) != cudaSuccess) return DECO_ERR_CUDA;
+        if (c->tau <= 1 && c->agg_pending && cudaStreamWaitEvent(c->side_stream, c->ev_agg, 0) != cudaSuccess)
+            return DECO_ERR_CUDA;
+        mark(c, 5, c->side_stream);
+        st = apply_due(c, c->side_stream);
+        mark(c, 6, c->side_stream);
+        if (cudaEventRecord(c->ev_join, c->side_stream) != cudaSuccess) return DECO_ERR_CUDA;
+        if (st != DECO_OK) return st;
+    }
+    err = launch_selection(c, s);
+    mark(c, 2, s);
+    if (err != cudaSuccess) return DECO_ERR_CUDA;
+    // This iteration's aggregate is not needed before iteration t + tau: the ring slot is booked
+    // now, the launch goes onto a second internal stream and is not joined.  Every later launch
+    // that rewrites the messages or reads the cache orders itself after it (wait_for_aggregate).
+    const uint32_t si = static_cast<uint32_t>(c->t % c->ring);
+    Slot &sl = c->slot_info[si];
+    if (sl.valid) return DECO_ERR_STATE;    // cannot happen while tau <= tau_max
+    const bool dense = aggregate_as_vector(c, c->k_of_msg);
+    sl.step = c->t;
+    sl.positions = dense ? c->d : static_cast<uint64_t>(c->n_total) * c->k_of_msg;
+    sl.dense = dense;
+    sl.valid = true;
     if (cudaEventRecord(c->ev_emit, s) != cudaSuccess) return DECO_ERR_CUDA;
-    if (cudaStreamWaitEvent(c->agg_stream, c->ev_emit, 0) != cudaSuccess) return DECO_ERR_CUDA;
-    st = deco_aggregate_stale(c, c->agg_stream);
-    if (st != DECO_OK) return st;
-    if (cudaEventRecord(c->ev_agg, c->agg_stream) != cudaSuccess) return DECO_ERR_CUDA;
-    c->agg_pending = true;
+    c->agg_deferred = true;
+    c->agg_slot = si;
+    c->agg_dense = dense;
+    if (!behind_pass && launch_deferred_aggregate(c) != cudaSuccess) return DECO_ERR_CUDA;
     if (cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) return DECO_ERR_CUDA;
     finish_iteration(c);
     return DECO_OK;
@@ -574,6 +645,11 @@ extern "C" deco_status deco_set_policy(deco_ctx *c, double delta, uint32_t tau)
     if (c->phase != 0) return DECO_ERR_STATE;
     const uint64_t k = deco_k_from_delta(delta, c->d);
     if (tau > c->tau_max || k > c->k_cap) return DECO_ERR_CAPACITY;
+    if (c->agg_deferred) {
+        // the launch takes the length of the messages from the policy they were made under
+        DeviceGuard guard(c->device);
+        if (!guard.ok || launch_deferred_aggregate(c) != cudaSuccess) return DECO_ERR_CUDA;
+    }
     c->delta = delta;
     c->tau = tau;
     c->k = k;

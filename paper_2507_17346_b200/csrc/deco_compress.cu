@@ -2290,6 +2290,19 @@ cudaError_t query_fallback_grid(deco_ctx *c)
     return cudaSuccess;
 }
 
+// The staged-pair chain as one cooperative launch: short vectors only (one CTA walks the
+// chunks, all CTAs resident at once, few staged pairs).
+static bool chain_is_one_launch(const deco_ctx *c)
+{
+    return c->nchunks <= 256 && c->chain_grid >= c->n &&
+           static_cast<uint64_t>(c->n) * (2 * c->k + 65536) <= FUSED_CHAIN_MAX_PAIRS;
+}
+
+bool selection_is_separate_launches(const deco_ctx *c)
+{
+    return streaming_route(c) && !chain_is_one_launch(c);
+}
+
 cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
 {
     Sel p = make_sel(c);
@@ -2315,8 +2328,7 @@ cudaError_t launch_selection(deco_ctx *c, cudaStream_t s)
     const bool walk_here = c->nchunks <= 256;
     // the kernels from here on rewrite the messages and their directory, which the previous
     // iteration's aggregation may still be reading on the internal stream
-    if (walk_here && c->chain_grid >= c->n &&
-        static_cast<uint64_t>(c->n) * (2 * c->k + 65536) <= FUSED_CHAIN_MAX_PAIRS) {
+    if (chain_is_one_launch(c)) {
         // one cooperative launch for the whole chain: as many CTAs per worker as the separate
         // kernels would use, as far as they can all be resident at once
         if (wait_for_aggregate(c, s) != cudaSuccess) return cudaGetLastError();

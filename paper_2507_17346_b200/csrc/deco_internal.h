@@ -165,6 +165,15 @@ struct deco_ctx {
     // which rewrites the messages or reads the cache has to wait for ev_agg first
     cudaEvent_t ev_emit = nullptr, ev_agg = nullptr;
     bool agg_pending = false;
+    // deco_step does not launch the aggregation of its iteration at once: the slot is booked
+    // and the launch waits for the end of the next streaming pass (ev_pass), so that it runs
+    // beside the selection kernels, which leave most of the device idle, and not beside the
+    // pass, which does not.  Whatever needs the aggregate or rewrites the messages earlier
+    // launches it first (launch_deferred_aggregate).
+    cudaEvent_t ev_pass = nullptr;
+    bool agg_deferred = false;
+    uint32_t agg_slot = 0;              // ring slot the deferred aggregation fills
+    bool agg_dense = false;             // ... as a plain vector
     // optional event timing: 8 events per recorded iteration
     bool timing = false;
     std::vector<cudaEvent_t> events;
@@ -178,6 +187,9 @@ cudaError_t query_fallback_grid(deco_ctx *c);
 cudaError_t launch_begin_step(deco_ctx *c, const void *grads, cudaStream_t s);
 cudaError_t launch_accumulate(deco_ctx *c, const void *grads, cudaStream_t s);
 cudaError_t launch_selection(deco_ctx *c, cudaStream_t s);
+// streaming route with the staged-pair chain as a row of ordinary launches (not the multi-pass
+// route, not the single cooperative launch of short vectors)
+bool selection_is_separate_launches(const deco_ctx *c);
 
 // deco_init with the distance between gradient rows given (0: d)
 deco_status init_context(deco_ctx **out, uint64_t d, uint32_t n, double delta, uint32_t tau, float lr,
@@ -206,9 +218,17 @@ inline void set_message_layout(deco_ctx *c, uint64_t k)
     }
 }
 
-// Order stream s after the aggregation that deco_step left running on the internal stream.
+// Launch the aggregation that deco_step booked but has not launched yet, if there is one, on
+// the internal stream behind the messages it reads (deco_api.cu).
+cudaError_t launch_deferred_aggregate(deco_ctx *c);
+
+// Order stream s after the aggregation that deco_step left to the internal stream.
 inline cudaError_t wait_for_aggregate(deco_ctx *c, cudaStream_t s)
 {
+    if (c->agg_deferred) {
+        const cudaError_t err = launch_deferred_aggregate(c);
+        if (err != cudaSuccess) return err;
+    }
     if (!c->agg_pending) return cudaSuccess;
     c->agg_pending = false;
     return cudaStreamWaitEvent(s, c->ev_agg, 0);

@@ -28,7 +28,10 @@ __device__ __forceinline__ void latch(uint32_t *status, uint32_t code, uint32_t 
 }
 
 // One tile by the whole CTA: dense fp32 accumulator and touched-bit mask in shared memory (both
-// all-zero on entry and on exit), workers added in order, output in index order.
+// all-zero on entry and on exit), workers added in order, output in index order.  NW: how many
+// workers' ranges and entries a thread holds in registers at once (the code is unrolled NW
+// times, so callers pick the smallest NW >= n they have).
+template <uint32_t NW>
 __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, uint64_t k_cap,
                                            const uint32_t *__restrict__ tile_start, uint64_t dir_stride,
                                            uint32_t ntiles,
@@ -39,7 +42,23 @@ __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, ui
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     uint64_t out_off = 0;
     uint32_t cap = 0, longest = 0;
-    for (uint32_t i = 0; i < n; ++i) {
+    constexpr bool KEEP = NW <= 8;                         // ranges stay in registers for the loads below
+    constexpr uint32_t NR = KEEP ? NW : 1;
+    uint32_t ra[NR], rb[NR];
+    if (KEEP) {
+#pragma unroll
+        for (uint32_t i = 0; i < NR; ++i) {
+            ra[i] = rb[i] = 0;
+            if (i < n) {
+                ra[i] = tile_start[static_cast<size_t>(i) * dir_stride + tile];
+                rb[i] = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
+            }
+            out_off += ra[i];
+            cap += rb[i] - ra[i];
+            longest = max(longest, rb[i] - ra[i]);
+        }
+    }
+    for (uint32_t i = KEEP ? NW : 0; i < n; ++i) {
         const uint32_t a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
         const uint32_t b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
         out_off += a;
@@ -52,22 +71,29 @@ __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, ui
         return;
     }
     const uint32_t first = tile * static_cast<uint32_t>(TILE);
-    if (n <= PREFETCH_WORKERS && longest <= static_cast<uint32_t>(BLOCK)) {
+    if (n <= NW && longest <= static_cast<uint32_t>(BLOCK)) {
         // At most one entry per thread and worker.  All loads are issued before the first
         // barrier, then the workers are added in order from registers.
-        deco_pair pre[PREFETCH_WORKERS];
+        deco_pair pre[NW];
 #pragma unroll
-        for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
+        for (uint32_t i = 0; i < NW; ++i) {
             pre[i].idx = DECO_NO_INDEX;
             pre[i].val = 0.0f;
-            if (i < n) {
-                const uint32_t a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
-                const uint32_t b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
-                if (a + threadIdx.x < b) pre[i] = msg[static_cast<size_t>(i) * k_cap + a + threadIdx.x];
+            uint32_t a, b;
+            if (KEEP) {
+                a = ra[i < NR ? i : 0];
+                b = rb[i < NR ? i : 0];
+            } else {
+                a = b = 0;
+                if (i < n) {
+                    a = tile_start[static_cast<size_t>(i) * dir_stride + tile];
+                    b = tile_start[static_cast<size_t>(i) * dir_stride + tile + 1];
+                }
             }
+            if (a + threadIdx.x < b) pre[i] = msg[static_cast<size_t>(i) * k_cap + a + threadIdx.x];
         }
 #pragma unroll
-        for (uint32_t i = 0; i < PREFETCH_WORKERS; ++i) {
+        for (uint32_t i = 0; i < NW; ++i) {
             if (i >= n) break;
             if (pre[i].idx != DECO_NO_INDEX) {
                 const uint32_t loc = pre[i].idx - first;
@@ -149,6 +175,22 @@ __device__ __forceinline__ void dense_tile(const deco_pair *__restrict__ msg, ui
     __syncthreads();
 }
 
+// dense_tile with the smallest unrolling that holds all n workers (the branch is CTA-uniform)
+__device__ __forceinline__ void dense_tile_n(const deco_pair *__restrict__ msg, uint64_t k_cap,
+                                             const uint32_t *__restrict__ tile_start, uint64_t dir_stride,
+                                             uint32_t ntiles, uint32_t n, deco_pair *__restrict__ slot,
+                                             uint64_t positions, uint32_t *__restrict__ status,
+                                             uint32_t tile, float *acc, uint32_t *mask, uint32_t *s_w)
+{
+    if (n <= 4)
+        dense_tile<4>(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status, tile, acc, mask, s_w);
+    else if (n <= 8)
+        dense_tile<8>(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status, tile, acc, mask, s_w);
+    else
+        dense_tile<PREFETCH_WORKERS>(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status, tile,
+                                     acc, mask, s_w);
+}
+
 // Persistent CTAs, every tile by the whole CTA: for messages with many entries per tile.
 __global__ void __launch_bounds__(BLOCK)
 aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
@@ -163,7 +205,7 @@ aggregate_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     mask[threadIdx.x] = 0;
     __syncthreads();
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        dense_tile(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status, tile, acc, mask, s_w);
+        dense_tile_n(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status, tile, acc, mask, s_w);
 }
 
 // Dense messages (n k entries in all comparable with d): the aggregate is kept as the plain
@@ -467,7 +509,7 @@ aggregate_sparse_kernel(const deco_pair *__restrict__ msg, uint64_t k_cap,
     mask[threadIdx.x] = 0;
     __syncthreads();
     for (; heavy; heavy &= heavy - 1)
-        dense_tile(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status,
+        dense_tile_n(msg, k_cap, tile_start, dir_stride, ntiles, n, slot, positions, status,
                    blockIdx.x * WARPS + __ffs(heavy) - 1, acc, mask, s_w);
 }
 
@@ -489,7 +531,7 @@ aggregate_multi_kernel(const ServerLayer *__restrict__ table, const uint32_t *__
         const uint32_t tile = g - L.first_tile;
         const uint64_t positions = static_cast<uint64_t>(n) * L.k;
         if (tile == 0 && threadIdx.x == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
-        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles + 1, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
+        dense_tile_n(L.msg, L.k_cap, L.tile_start, L.ntiles + 1, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
                    positions, L.status, tile, acc, mask, s_w);
     }
 }
@@ -526,7 +568,7 @@ aggregate_sparse_multi_kernel(const ServerLayer *__restrict__ table, const uint3
     for (; heavy; heavy &= heavy - 1) {
         const uint32_t gh = blockIdx.x * WARPS + __ffs(heavy) - 1;
         const ServerLayer &L = table[tile_layer[gh]];
-        dense_tile(L.msg, L.k_cap, L.tile_start, L.ntiles + 1, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
+        dense_tile_n(L.msg, L.k_cap, L.tile_start, L.ntiles + 1, L.ntiles, n, L.slots + slot_write * (n * L.k_cap),
                    static_cast<uint64_t>(n) * L.k, L.status, gh - L.first_tile, acc, mask, s_w);
     }
 }
@@ -625,7 +667,7 @@ small_server_kernel(const SmallLayer *__restrict__ table, uint32_t n, uint32_t a
         mask[threadIdx.x] = 0;
         __syncthreads();
         const uint64_t positions = static_cast<uint64_t>(n) * L.k;
-        dense_tile(L.msg, L.k_cap, L.tile_start, 2, 1, n, L.slots + slot_write * slot_len, positions,
+        dense_tile_n(L.msg, L.k_cap, L.tile_start, 2, 1, n, L.slots + slot_write * slot_len, positions,
                    L.status, 0, acc, mask, s_w);
         if (threadIdx.x == 0) L.slot_pos[slot_write] = static_cast<uint32_t>(positions);
         __syncthreads();
