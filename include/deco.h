@@ -167,21 +167,24 @@ deco_status deco_apply_update(deco_ctx *ctx, void *stream);
 
 /*
  * The three calls above for callers that do not interleave other work.  With tau >= 1 the
- * server side runs on an internal stream next to the worker side:
+ * server side runs on internal streams:
  *   - the update of the aggregates that are due (it depends on neither e nor the messages) is
- *     forked from `stream` at the start of the call and joined back at its end, so e, the
- *     messages and the parameters are complete, in stream order, when `stream` passes the call;
+ *     forked from `stream` inside the call and joined back at its end, so e, the messages and
+ *     the parameters are complete, in stream order, when `stream` passes the call;
  *   - the aggregation S_t of this iteration's messages, which Algorithm 1 needs only tau
- *     iterations later, is left running on the internal stream.  It reads the messages and
- *     writes a cache slot only the library sees; every later library call orders itself after
- *     it (calls without a stream argument wait on the host), and deco_join does so explicitly.
+ *     iterations later, is left to the internal stream: it runs either right behind this call
+ *     or behind the streaming pass of the next one (the library picks by the size of the
+ *     problem).  It reads the messages and writes a cache slot only the library sees; every
+ *     later library call orders itself after it (calls without a stream argument wait on the
+ *     host), and deco_join does so explicitly.  The messages must not be overwritten by the
+ *     caller before deco_join or the next library call on this context.
  * With tau = 0 the three steps run strictly in order on `stream`.  Results are bit-identical
  * to the three calls in every case.
  */
 deco_status deco_step(deco_ctx *ctx, const void *grads /* DEVICE */, void *stream);
 
-/* Make `stream` wait for the aggregation a previous deco_step left on the internal stream
- * (no-op if there is none).  After it, all device work of the library is ordered before
+/* Launch the aggregation a previous deco_step left to the internal stream, if it has not been
+ * launched yet, and make `stream` wait for it (no-op if there is none).  After it, all device work of the library is ordered before
  * whatever is enqueued on `stream` next. */
 deco_status deco_join(deco_ctx *ctx, void *stream);
 
