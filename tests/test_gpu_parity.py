@@ -587,6 +587,77 @@ def test_fused_step_with_a_long_aggregation(tau):
         B.deco_destroy(b)
 
 
+@pytest.mark.parametrize("d,n,delta", [(6_000_000, 8, 0.05), (16_000_000, 16, 0.0065)])
+def test_fused_step_with_the_server_side_behind_the_pass(d, n, delta):
+    """With many staged pairs in all (n (2 k + 65536) above 4 Mi) the selection is a row of
+    ordinary launches, and deco_step then books the aggregation of an iteration and launches it
+    only behind the streaming pass of the next call, together with the update.  The first
+    shape keeps the aggregate as a vector, the second as pairs.  Bits must equal the strictly
+    sequential three calls: back to back without a host sync, across policy changes (which
+    have to launch a booked aggregation first, tau = 1 and tau = 0 included), with the three
+    calls mixed in, with a read of the cache in between, and through export / import while an
+    aggregation is booked."""
+    k = int(B.deco_k_from_delta(delta, d))
+    assert n * (2 * k + 65536) > (4 << 20)
+    kw = dict(tau_max=3, delta_max=delta)
+    a = B.deco_init(d, n, delta, 2, 0.1, **kw)
+    b = B.deco_init(d, n, delta, 2, 0.1, **kw)
+    c = B.deco_init(d, n, delta, 2, 0.1, **kw)
+    try:
+        pool = [_values("normal", n, d, t, torch.float32) for t in range(3)]
+        plan = {4: (delta, 1), 7: (delta * 0.9, 3), 10: (delta, 0), 12: (delta * 0.8, 2)}
+        steps = 16
+        for t in range(steps):
+            if t in plan:
+                B.deco_set_policy(a, *plan[t])
+            if t % 5 == 3:
+                B.deco_ef_compress(a, pool[t % 3])
+                B.deco_aggregate_stale(a)
+                B.deco_apply_update(a)
+            else:
+                B.deco_step(a, pool[t % 3])
+            if t == 8:
+                B.deco_get_aggregate_vector(a, 8) if 8 * n * B.deco_get_k(a) >= d else B.deco_get_aggregate(a, 8)
+            if t == 11:                                          # resume in another context
+                B.deco_import_state(c, B.deco_export_state(a))
+        for t in range(12, steps):
+            if t in plan:
+                B.deco_set_policy(c, *plan[t])
+            B.deco_step(c, pool[t % 3])
+        for t in range(steps):
+            if t in plan:
+                B.deco_set_policy(b, *plan[t])
+            B.deco_ef_compress(b, pool[t % 3])
+            B.deco_aggregate_stale(b)
+            B.deco_apply_update(b)
+        B.deco_join(a)
+        B.deco_join(c)
+        torch.cuda.synchronize()
+        bb = B.deco_get_buffers(b)
+        kk = B.deco_get_k(b)
+        for other in (a, c):
+            bo = B.deco_get_buffers(other)
+            assert torch.equal(B.view_i32(bo["params"], (d,)), B.view_i32(bb["params"], (d,)))
+            assert torch.equal(B.view_i32(bo["e"], (n, bo["e_stride"])), B.view_i32(bb["e"], (n, bb["e_stride"])))
+            assert torch.equal(B.view_i32(bo["msg"], (n, bo["k_cap"], 2))[:, :kk],
+                               B.view_i32(bb["msg"], (n, bb["k_cap"], 2))[:, :kk])
+            so, sb = B.deco_get_stats(other), B.deco_get_stats(b)
+            assert so["step"] == sb["step"] == steps and so["cached_aggregates"] == sb["cached_aggregates"]
+            assert so["device_status"] == 0
+            for s_ in range(steps - 2, steps):                   # the aggregates still cached (tau = 2)
+                if 8 * n * kk >= d:
+                    assert torch.equal(B.view_i32(B.deco_get_aggregate_vector(other, s_), (d,)),
+                                       B.view_i32(B.deco_get_aggregate_vector(b, s_), (d,)))
+                else:
+                    (pa, na), (pb, nb) = B.deco_get_aggregate(other, s_), B.deco_get_aggregate(b, s_)
+                    assert na == nb
+                    assert torch.equal(B.view_i32(pa, (na, 2)), B.view_i32(pb, (nb, 2)))
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
+        B.deco_destroy(c)
+
+
 def test_checkpoint_and_resume_give_the_same_bits():
     wl = W.make_workload("gpt2_small", 0.08)
     kw = dict(grad_dtype=B.DECO_BF16, tau_max=4, delta_max=0.01)
