@@ -658,6 +658,77 @@ def test_fused_step_with_the_server_side_behind_the_pass(d, n, delta):
         B.deco_destroy(c)
 
 
+@pytest.mark.parametrize("seed", range(700, 712))
+def test_fused_step_random_call_mixes(seed):
+    """deco_step against the strictly sequential three calls on seeded random shapes (up to
+    4 * 10^7 entries, 1 to 16 workers, both gradient types), policies that change at random
+    iterations (tau down to 0), and random mixes of calls between the steps: the three calls,
+    a join, a read of the statistics, and an export / import into a fresh context.  Parameters,
+    residuals, messages and the number of cached aggregates must agree bit for bit."""
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(1, 17))
+    d = int(rng.choice([rng.integers(200_000, 2_000_000), rng.integers(2_000_000, 12_000_000),
+                        rng.integers(12_000_000, 40_000_000)]))
+    d = min(d, 150_000_000 // n)
+    delta_max = float(min(1.0, 10.0 ** rng.uniform(-3, -0.7)))
+    tau_max = int(rng.integers(1, 5))
+    dtype = (torch.float32, torch.bfloat16)[int(rng.integers(0, 2))]
+
+    def policy():
+        return float(delta_max * 10.0 ** rng.uniform(-1.0, 0)), int(rng.integers(0, tau_max + 1))
+
+    first = policy()
+    steps = int(rng.integers(8, 16))
+    plan = {int(s_): policy() for s_ in rng.choice(np.arange(1, steps), size=int(rng.integers(0, 4)), replace=False)}
+    acts = [str(rng.choice(["step", "step", "step", "three", "step_join", "step_stats"])) for _ in range(steps)]
+    swap_at = int(rng.integers(2, steps - 1)) if rng.integers(0, 2) else -1
+    pool = [_values("normal", n, d, seed + t, dtype) for t in range(3)]
+    kw = dict(grad_dtype=B.DECO_F32 if dtype == torch.float32 else B.DECO_BF16, tau_max=tau_max,
+              delta_max=delta_max)
+    a = B.deco_init(d, n, first[0], first[1], 0.1, **kw)
+    b = B.deco_init(d, n, first[0], first[1], 0.1, **kw)
+    try:
+        for t in range(steps):
+            if t in plan:
+                B.deco_set_policy(a, *plan[t])
+                B.deco_set_policy(b, *plan[t])
+            g = pool[t % 3]
+            if acts[t] == "three":
+                B.deco_ef_compress(a, g)
+                B.deco_aggregate_stale(a)
+                B.deco_apply_update(a)
+            else:
+                B.deco_step(a, g)
+                if acts[t] == "step_join":
+                    B.deco_join(a)
+                if acts[t] == "step_stats":
+                    B.deco_get_stats(a)
+            B.deco_ef_compress(b, g)
+            B.deco_aggregate_stale(b)
+            B.deco_apply_update(b)
+            if t == swap_at:                                     # carry on in a fresh context
+                blob = B.deco_export_state(a)
+                B.deco_destroy(a)
+                a = B.deco_init(d, n, first[0], first[1], 0.1, **kw)
+                B.deco_import_state(a, blob)
+        B.deco_join(a)
+        torch.cuda.synchronize()
+        ba, bb = B.deco_get_buffers(a), B.deco_get_buffers(b)
+        k = B.deco_get_k(b)
+        assert torch.equal(B.view_i32(ba["params"], (d,)), B.view_i32(bb["params"], (d,)))
+        assert torch.equal(B.view_i32(ba["e"], (n, ba["e_stride"])), B.view_i32(bb["e"], (n, bb["e_stride"])))
+        assert torch.equal(B.view_i32(ba["msg"], (n, ba["k_cap"], 2))[:, :k],
+                           B.view_i32(bb["msg"], (n, bb["k_cap"], 2))[:, :k])
+        sa, sb = B.deco_get_stats(a), B.deco_get_stats(b)
+        assert sa["step"] == sb["step"] == steps and sa["cached_aggregates"] == sb["cached_aggregates"]
+        assert sa["device_status"] == 0 and sb["device_status"] == 0
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
+        del pool
+        torch.cuda.empty_cache()
+
+
 def test_checkpoint_and_resume_give_the_same_bits():
     wl = W.make_workload("gpt2_small", 0.08)
     kw = dict(grad_dtype=B.DECO_BF16, tau_max=4, delta_max=0.01)
