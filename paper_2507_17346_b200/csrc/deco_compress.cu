@@ -1184,10 +1184,9 @@ __global__ void __launch_bounds__(BLOCK) stage_hist_b_kernel(Sel p)
 }
 
 // One CTA: ties are granted to chunks in index order until ties_take are used up, then every
-// chunk gets its position in the message.  Per thread a contiguous range of chunks.  With
-// sums_ready the per-chunk sums were left in chunk_cnt/rej/eq by chunk_sums_kernel; otherwise
-// (few chunks) they are taken here from the CHUNK_TILES tile counters of each chunk.
-__device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, bool sums_ready)
+// chunk gets its position in the message.  Per thread a contiguous range of chunks.  The sums
+// of a chunk are taken here from its CHUNK_TILES tile counters (few chunks).
+__device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/)
 {
     uint32_t *ccnt = p.chunk_cnt + static_cast<size_t>(i) * p.nchunks;
     uint32_t *crej = p.chunk_rej + static_cast<size_t>(i) * p.nchunks;
@@ -1202,22 +1201,16 @@ __device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, 
     const uint32_t lo = min(p.nchunks, threadIdx.x * per), hi = min(p.nchunks, lo + per);
     uint32_t eq_sum = 0;
     for (uint32_t c = lo; c < hi; ++c) {
-        uint32_t q;
-        if (sums_ready) {
-            q = __ldcg(&ceq[c]);
-        } else {
-            uint32_t a = 0, b = 0;
-            q = 0;
-            const uint32_t t0 = c * CHUNK_TILES, t1 = min(p.ntiles, t0 + CHUNK_TILES);
-            for (uint32_t t = t0; t < t1; ++t) {
-                a += tcnt[t];
-                b += __ldcg(&rej[t]);
-                q += __ldcg(&eqc[t]);
-            }
-            ccnt[c] = a;
-            crej[c] = b;
-            ceq[c] = q;
+        uint32_t a = 0, b = 0, q = 0;
+        const uint32_t t0 = c * CHUNK_TILES, t1 = min(p.ntiles, t0 + CHUNK_TILES);
+        for (uint32_t t = t0; t < t1; ++t) {
+            a += tcnt[t];
+            b += __ldcg(&rej[t]);
+            q += __ldcg(&eqc[t]);
         }
+        ccnt[c] = a;
+        crej[c] = b;
+        ceq[c] = q;
         eq_sum += q;
     }
     uint32_t eq_total;
@@ -1242,6 +1235,71 @@ __device__ void chunk_walk(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/, 
     if (threadIdx.x == 0) {
         cstart[p.nchunks] = sel_total;
         if (sel_total != p.k) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x200u, i);
+    }
+    __syncthreads();
+}
+
+// The same walk over many chunks whose sums chunk_sums_kernel left in chunk_cnt/rej/eq: the
+// sums go through shared memory (sm.h, free in that kernel) in segments of WALK_SEG chunks,
+// fetched with coalesced loads in one round trip; a thread then owns WALK_PER consecutive
+// chunks of the segment, and the two running totals carry over from segment to segment.
+constexpr uint32_t WALK_PER = 8;
+constexpr uint32_t WALK_SEG = WALK_PER * BLOCK;
+static_assert(2 * WALK_SEG <= RADIX_BINS, "two words per chunk of a segment in sm.h");
+
+__device__ void chunk_walk_sums(const Sel &p, uint32_t i, uint32_t *s_scan /*[33]*/)
+{
+    const uint32_t *ccnt = p.chunk_cnt + static_cast<size_t>(i) * p.nchunks;
+    const uint32_t *crej = p.chunk_rej + static_cast<size_t>(i) * p.nchunks;
+    const uint32_t *ceq = p.chunk_eq + static_cast<size_t>(i) * p.nchunks;
+    uint32_t *cstart = p.chunk_start + static_cast<size_t>(i) * (p.nchunks + 1);
+    uint32_t *ceqb = p.chunk_eqb + static_cast<size_t>(i) * p.nchunks;
+    const uint32_t ties = p.sel[i].ties_take;
+    uint32_t *s_q = sm.h, *s_sel = sm.h + WALK_SEG;          // ties / entries surely selected, per chunk
+    uint32_t eq_carry = 0, pos_carry = 0;
+    for (uint32_t seg = 0; seg < p.nchunks; seg += WALK_SEG) {
+        const uint32_t m = min(WALK_SEG, p.nchunks - seg);
+        for (uint32_t c = threadIdx.x; c < WALK_SEG; c += BLOCK) {
+            uint32_t q = 0, surely = 0;
+            if (c < m) {
+                q = __ldcg(&ceq[seg + c]);
+                surely = __ldcg(&ccnt[seg + c]) - __ldcg(&crej[seg + c]) - q;
+            }
+            s_q[c] = q;
+            s_sel[c] = surely;
+        }
+        __syncthreads();
+        const uint32_t lo = threadIdx.x * WALK_PER;
+        uint32_t eq_sum = 0;
+#pragma unroll
+        for (uint32_t j = 0; j < WALK_PER; ++j) eq_sum += s_q[lo + j];
+        uint32_t eq_total;
+        uint32_t eq_before = eq_carry + block_excl_scan(eq_sum, s_scan, eq_total);
+        uint32_t sel_sum = 0;
+#pragma unroll
+        for (uint32_t j = 0; j < WALK_PER; ++j) {
+            const uint32_t q = s_q[lo + j];
+            const uint32_t left = ties > eq_before ? ties - eq_before : 0u;
+            if (lo + j < m) ceqb[seg + lo + j] = eq_before;
+            const uint32_t take = s_sel[lo + j] + min(q, left);
+            s_sel[lo + j] = take;                            // own words only
+            sel_sum += take;
+            eq_before += q;
+        }
+        uint32_t sel_total;
+        uint32_t pos = pos_carry + block_excl_scan(sel_sum, s_scan, sel_total);
+#pragma unroll
+        for (uint32_t j = 0; j < WALK_PER; ++j) {
+            if (lo + j < m) cstart[seg + lo + j] = pos;
+            pos += s_sel[lo + j];
+        }
+        eq_carry += eq_total;
+        pos_carry += sel_total;
+        __syncthreads();                                     // sm.h is refilled by the next segment
+    }
+    if (threadIdx.x == 0) {
+        cstart[p.nchunks] = pos_carry;
+        if (pos_carry != p.k) latch(p.status, DECO_ERR_DEVICE_CHECK, 0x200u, i);
     }
     __syncthreads();
 }
@@ -1274,7 +1332,7 @@ __device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i)
         }
     }
     if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 4], &sm.misc[2])) return;
-    chunk_walk(p, i, sm.scan, true);
+    chunk_walk_sums(p, i, sm.scan);
 }
 
 __global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p)
@@ -1325,7 +1383,7 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
     }
     // (the rejected entries get their value back in e from emit, which reads every staged pair anyway)
     if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &sm.misc[2])) return;
-    if (walk_here) chunk_walk(p, i, sm.scan, false);
+    if (walk_here) chunk_walk(p, i, sm.scan);
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_classify_kernel(Sel p, uint32_t walk_here)
