@@ -379,10 +379,73 @@ __device__ __forceinline__ uint32_t warp_merge(bool valid, uint32_t idx, float v
 
 // Sparse messages (a few entries per tile): one warp per tile, no accumulator.  Lane i first
 // holds worker i's range of the tile.  At most 32 entries in all are merged in one go;
-// otherwise the tile's index range is cut into SPARSE_WINDOWS windows that are merged one
-// after the other, each with at most 32 entries.  A tile that does not fit is left to the
-// whole CTA afterwards (dense_tile).
+// otherwise the tile's index range is cut into windows that are merged one after the other,
+// each with at most 32 entries: halves where that is enough (up to 64 entries), else
+// SPARSE_WINDOWS quarters.  A tile that does not fit is left to the whole CTA afterwards
+// (dense_tile).
 constexpr int SPARSE_WINDOWS = 4;
+
+// The entries of one tile, cut into windows of STEP quarters of its index range, merged window
+// after window (lane i holds worker i's range [a, a + len) and, in below[q], how many of its
+// entries lie below the end of quarter q - 1).  Returns false, with nothing written, if some
+// window holds more than 32 entries.
+template <int STEP>
+__device__ __forceinline__ bool merge_windows(const deco_pair *__restrict__ msg, uint64_t k_cap, uint32_t n,
+                                              uint32_t a, const uint32_t (&below)[SPARSE_WINDOWS + 1],
+                                              uint32_t first, deco_pair *__restrict__ out, uint32_t cap,
+                                              uint32_t *__restrict__ status)
+{
+    constexpr int NWIN = SPARSE_WINDOWS / STEP;
+    const int lane = threadIdx.x & 31;
+    // per window: entries of the workers before lane's own, and in all
+    uint32_t before[NWIN], total[NWIN];
+    bool fits = true;
+#pragma unroll
+    for (int q = 0; q < NWIN; ++q) {
+        const uint32_t mine = below[(q + 1) * STEP] - below[q * STEP];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(FULL, incl, o);
+            if (lane >= o) incl += t;
+        }
+        before[q] = incl - mine;
+        total[q] = __shfl_sync(FULL, incl, 31);
+        fits = fits && total[q] <= 32;
+    }
+    if (!fits) return false;
+    uint32_t uniq = 0;
+#pragma unroll
+    for (int q = 0; q < NWIN; ++q) {
+        if (total[q] == 0) continue;
+        const uint32_t part_a = a + below[q * STEP], part_len = below[(q + 1) * STEP] - below[q * STEP];
+        deco_pair pr;
+        pr.idx = DECO_NO_INDEX;
+        pr.val = 0.0f;
+        bool valid = false;
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint32_t pb = __shfl_sync(FULL, before[q], i);
+            const uint32_t pl = __shfl_sync(FULL, part_len, i);
+            const uint32_t pa = __shfl_sync(FULL, part_a, i);
+            if (static_cast<uint32_t>(lane) >= pb && static_cast<uint32_t>(lane) < pb + pl) {
+                pr = msg[static_cast<size_t>(i) * k_cap + pa + (lane - pb)];
+                valid = true;
+            }
+        }
+        if (valid && pr.idx - first >= static_cast<uint32_t>(TILE)) {
+            latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pr.idx);
+            valid = false;
+        }
+        uniq += warp_merge(valid, pr.idx, pr.val, out + uniq);
+    }
+    for (uint32_t q = uniq + lane; q < cap; q += 32) {
+        deco_pair pr;
+        pr.idx = DECO_NO_INDEX;
+        pr.val = 0.0f;
+        out[q] = pr;
+    }
+    return true;
+}
 
 // One tile by one warp.  Returns true (to every lane) if the tile does not fit and has to be
 // done by the whole CTA with the dense accumulator.
@@ -414,74 +477,29 @@ __device__ __forceinline__ bool sparse_tile_warp(const deco_pair *__restrict__ m
         return false;
     }
     if (cap > 32u * SPARSE_WINDOWS || longest > 32) return true;
-    // lane i: how many of worker i's entries lie below the end of each window
-    // (every lane looks at one entry of each worker in turn: ranges are at most 32 long)
+    deco_pair *out = slot + out_off;
     uint32_t below[SPARSE_WINDOWS + 1];
     below[0] = 0;
 #pragma unroll
     for (int q = 1; q <= SPARSE_WINDOWS; ++q) below[q] = len;
-    if (cap > 32) {
-        for (uint32_t i = 0; i < n; ++i) {
-            const uint32_t ai = __shfl_sync(FULL, a, i), li = __shfl_sync(FULL, len, i);
-            uint32_t loc = DECO_NO_INDEX;
-            if (static_cast<uint32_t>(lane) < li)
-                loc = msg[static_cast<size_t>(i) * k_cap + ai + lane].idx - first;
+    // at most 32 entries in all: one window
+    if (cap <= 32) return !merge_windows<SPARSE_WINDOWS>(msg, k_cap, n, a, below, first, out, cap, status);
+    // lane i: how many of worker i's entries lie below the end of each quarter
+    // (every lane looks at one entry of each worker in turn: ranges are at most 32 long)
+    for (uint32_t i = 0; i < n; ++i) {
+        const uint32_t ai = __shfl_sync(FULL, a, i), li = __shfl_sync(FULL, len, i);
+        uint32_t loc = DECO_NO_INDEX;
+        if (static_cast<uint32_t>(lane) < li)
+            loc = msg[static_cast<size_t>(i) * k_cap + ai + lane].idx - first;
 #pragma unroll
-            for (int q = 1; q < SPARSE_WINDOWS; ++q) {
-                const uint32_t cnt = __popc(__ballot_sync(FULL, loc < q * (TILE / SPARSE_WINDOWS)));
-                if (static_cast<uint32_t>(lane) == i) below[q] = cnt;
-            }
+        for (int q = 1; q < SPARSE_WINDOWS; ++q) {
+            const uint32_t cnt = __popc(__ballot_sync(FULL, loc < q * (TILE / SPARSE_WINDOWS)));
+            if (static_cast<uint32_t>(lane) == i) below[q] = cnt;
         }
     }
-    // per window: entries of the workers before lane's own, and in all
-    uint32_t before[SPARSE_WINDOWS], total[SPARSE_WINDOWS];
-    bool fits = true;
-#pragma unroll
-    for (int q = 0; q < SPARSE_WINDOWS; ++q) {
-        const uint32_t mine = below[q + 1] - below[q];
-        uint32_t incl = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t t = __shfl_up_sync(FULL, incl, o);
-            if (lane >= o) incl += t;
-        }
-        before[q] = incl - mine;
-        total[q] = __shfl_sync(FULL, incl, 31);
-        fits = fits && total[q] <= 32;
-    }
-    if (!fits) return true;
-    deco_pair *out = slot + out_off;
-    uint32_t uniq = 0;
-#pragma unroll
-    for (int q = 0; q < SPARSE_WINDOWS; ++q) {
-        if (total[q] == 0) continue;
-        const uint32_t part_a = a + below[q], part_len = below[q + 1] - below[q];
-        deco_pair pr;
-        pr.idx = DECO_NO_INDEX;
-        pr.val = 0.0f;
-        bool valid = false;
-        for (uint32_t i = 0; i < n; ++i) {
-            const uint32_t pb = __shfl_sync(FULL, before[q], i);
-            const uint32_t pl = __shfl_sync(FULL, part_len, i);
-            const uint32_t pa = __shfl_sync(FULL, part_a, i);
-            if (static_cast<uint32_t>(lane) >= pb && static_cast<uint32_t>(lane) < pb + pl) {
-                pr = msg[static_cast<size_t>(i) * k_cap + pa + (lane - pb)];
-                valid = true;
-            }
-        }
-        if (valid && pr.idx - first >= static_cast<uint32_t>(TILE)) {
-            latch(status, DECO_ERR_DEVICE_CHECK, 0x401u, pr.idx);
-            valid = false;
-        }
-        uniq += warp_merge(valid, pr.idx, pr.val, out + uniq);
-    }
-    for (uint32_t q = uniq + lane; q < cap; q += 32) {
-        deco_pair pr;
-        pr.idx = DECO_NO_INDEX;
-        pr.val = 0.0f;
-        out[q] = pr;
-    }
-    return false;
+    // halves if they hold at most 32 entries each, else quarters
+    if (cap <= 64 && merge_windows<2>(msg, k_cap, n, a, below, first, out, cap, status)) return false;
+    return !merge_windows<1>(msg, k_cap, n, a, below, first, out, cap, status);
 }
 
 __global__ void __launch_bounds__(BLOCK)
