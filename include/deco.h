@@ -192,8 +192,11 @@ deco_status deco_join(deco_ctx *ctx, void *stream);
  * One iteration with HOST buffers: copies grads_host ([n][d], grad_dtype) to the device,
  * runs deco_step, and copies back what a deployment would move: the n messages
  * (msg_host_out, [n][k] pairs, may be NULL) and the parameters (params_host_out, [d] fp32,
- * may be NULL).  Copies are asynchronous on `stream`; use pinned host memory and
- * synchronise the stream before reading the outputs.
+ * may be NULL).  Use pinned host memory.  The copy of grads_host runs on a stream of the
+ * library's own into one of two device buffers, so that it overlaps the kernels of the previous
+ * call: grads_host must hold the gradients when the call is made (the copy does not wait for
+ * earlier work on `stream`) and must stay unchanged until `stream` has passed the call.  The
+ * step and the copies back are ordered on `stream`; synchronise it before reading the outputs.
  */
 deco_status deco_step_host(deco_ctx *ctx, const void *grads_host, deco_pair *msg_host_out,
                            float *params_host_out, void *stream);

@@ -67,7 +67,12 @@ void free_all(deco_ctx *c)
     cudaFree(c->sample_win);
     cudaFree(c->done);
     cudaFree(c->dev_status);
-    cudaFree(c->grads_staging);
+    for (int b = 0; b < 2; ++b) {
+        cudaFree(c->grads_staging[b]);
+        if (c->ev_copied[b]) cudaEventDestroy(c->ev_copied[b]);
+        if (c->ev_consumed[b]) cudaEventDestroy(c->ev_consumed[b]);
+    }
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
     c->events.clear();
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -606,20 +611,34 @@ extern "C" deco_status deco_step_host(deco_ctx *c, const void *grads_host, deco_
     if (!guard.ok) return DECO_ERR_CUDA;
     cudaStream_t s = as_stream(stream);
     const uint64_t gbytes = static_cast<uint64_t>(c->n) * c->d * (c->grad_dtype == DECO_BF16 ? 2 : 4);
-    if (!c->grads_staging) {
+    const int b = static_cast<int>(c->host_calls & 1);
+    if (!c->copy_stream && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
+        return DECO_ERR_CUDA;
+    if (!c->grads_staging[b]) {
         void *q = nullptr;
         cudaError_t err = cudaMalloc(&q, gbytes);
+        if (err == cudaSuccess) err = cudaEventCreateWithFlags(&c->ev_copied[b], cudaEventDisableTiming);
+        if (err == cudaSuccess) err = cudaEventCreateWithFlags(&c->ev_consumed[b], cudaEventDisableTiming);
         if (err != cudaSuccess) {
             cudaGetLastError();
+            cudaFree(q);
             return err == cudaErrorMemoryAllocation ? DECO_ERR_OOM : DECO_ERR_CUDA;
         }
-        c->grads_staging = q;
+        c->grads_staging[b] = q;
         c->device_bytes += gbytes;
+    } else if (cudaStreamWaitEvent(c->copy_stream, c->ev_consumed[b], 0) != cudaSuccess) {
+        return DECO_ERR_CUDA;              // the step of two calls ago still reads this buffer
     }
-    if (cudaMemcpyAsync(c->grads_staging, grads_host, gbytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    if (cudaMemcpyAsync(c->grads_staging[b], grads_host, gbytes, cudaMemcpyHostToDevice, c->copy_stream) !=
+            cudaSuccess ||
+        cudaEventRecord(c->ev_copied[b], c->copy_stream) != cudaSuccess ||
+        cudaStreamWaitEvent(s, c->ev_copied[b], 0) != cudaSuccess)
         return DECO_ERR_CUDA;
     c->launches += 1;
-    deco_status st = deco_step(c, c->grads_staging, stream);
+    c->host_calls += 1;
+    deco_status st = deco_step(c, c->grads_staging[b], stream);
+    // (recorded also after a step that failed to enqueue: the buffer is free either way)
+    if (cudaEventRecord(c->ev_consumed[b], s) != cudaSuccess) return DECO_ERR_CUDA;
     if (st != DECO_OK) return st;
     if (msg_out) {
         // rows of k pairs, packed: [n][k]

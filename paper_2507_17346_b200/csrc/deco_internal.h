@@ -148,7 +148,13 @@ struct deco_ctx {
     uint32_t *chunk_eqb = nullptr;      // [n][nchunks] ties in earlier chunks
     uint32_t *chunk_start = nullptr;    // [n][nchunks + 1] message position of each chunk
     uint32_t *dev_status = nullptr;     // [4]: status, two detail words, fallback flag
-    void *grads_staging = nullptr;      // device copy of host gradients (deco_step_host)
+    // deco_step_host: two device copies of host gradients, filled in turn on a stream of their
+    // own, so that the copy for one call runs while the previous call's kernels do
+    void *grads_staging[2] = {nullptr, nullptr};
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr};      // the buffer holds the call's gradients
+    cudaEvent_t ev_consumed[2] = {nullptr, nullptr};    // the step that read the buffer is through
+    uint64_t host_calls = 0;
     uint64_t device_bytes = 0;
     // host bookkeeping
     uint64_t t = 0;

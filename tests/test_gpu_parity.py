@@ -837,3 +837,40 @@ def test_host_buffer_step_matches_device_step():
     finally:
         B.deco_destroy(a)
         B.deco_destroy(b)
+
+
+def test_host_buffer_steps_back_to_back():
+    """deco_step_host copies the gradients on a stream of the library's own into one of two device
+    buffers: calls made back to back, without a host sync in between, must each see their own
+    gradients (a buffer is not refilled before the step that read it is through) and give the
+    bits of the device-buffer steps, message by message."""
+    wl = W.make_workload("resnet18", 0.25)
+    k = B.deco_k_from_delta(wl.delta, wl.d)
+    steps = 7
+    a = B.deco_init(wl.d, wl.n, wl.delta, wl.tau, wl.lr)
+    b = B.deco_init(wl.d, wl.n, wl.delta, wl.tau, wl.lr)
+    try:
+        grads = [W.gradients(wl, t, "cuda") for t in range(steps)]
+        hosts = [g.cpu().pin_memory() for g in grads]
+        msgs = [torch.empty((wl.n, k, 2), dtype=torch.int32).pin_memory() for _ in range(steps)]
+        xs = [torch.empty(wl.d, dtype=torch.float32).pin_memory() for _ in range(steps)]
+        torch.cuda.synchronize()
+        for t in range(steps):
+            B.deco_step_host(b, hosts[t], msgs[t], xs[t] if t % 2 == 0 else None)
+        B.deco_join(b)
+        torch.cuda.synchronize()
+        buf = B.deco_get_buffers(a)
+        for t in range(steps):
+            B.deco_step(a, grads[t])
+            torch.cuda.synchronize()
+            assert torch.equal(msgs[t], B.view_i32(buf["msg"], (wl.n, buf["k_cap"], 2))[:, :k].cpu()), t
+            if t % 2 == 0:
+                assert torch.equal(xs[t].view(torch.int32),
+                                   B.view_i32(buf["params"], (wl.d,)).cpu()), t
+        bb = B.deco_get_buffers(b)
+        assert torch.equal(B.view_i32(bb["e"], (wl.n, bb["e_stride"])), B.view_i32(buf["e"], (wl.n, buf["e_stride"])))
+        assert B.deco_get_stats(b)["device_status"] == 0
+    finally:
+        B.deco_destroy(a)
+        B.deco_destroy(b)
+
