@@ -610,6 +610,14 @@ def run_ours(args):
     # replicas: every rank steps the whole workload; sharded: the ranks share one workload
     value = whole_job_value(gbytes, 1 if sharded else world, res["ms_per_step"])
 
+    # the oracle's sample on the host cores comes next: ten seconds in which the card rests
+    # between the 1.1 G workload and the smaller ones
+    cpu_base = None
+    if not args.no_cpu_baseline and world == 1:
+        gbs, ms, sample = oracle_throughput(wl, 2, 1)
+        cpu_base = {"value": gbs, "unit": UNIT, "cores": 1, "host_cores": host_cores(),
+                    "kind": "oracle", "sample": sample, "ms_per_step_sample": ms}
+
     others = None
     if world == 1 and not args.no_others and args.workload == DEFAULT_WORKLOAD and args.scale == 1.0:
         others = {}
@@ -648,11 +656,9 @@ def run_ours(args):
             "roofline": res["roofline"], "clocks": res["clocks"], "gpu_launches": res["launches"]}
     if res["e2e"] is not None:
         line["e2e"] = res["e2e"]
-    if not args.no_cpu_baseline and world == 1:
-        gbs, ms, sample = oracle_throughput(wl, 2, 1)
-        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": 1, "host_cores": host_cores(),
-                                "kind": "oracle", "sample": sample, "ms_per_step_sample": ms}
-        line["config"]["cpu_baseline_sample"] = sample
+    if cpu_base is not None:
+        line["cpu_baseline"] = cpu_base
+        line["config"]["cpu_baseline_sample"] = cpu_base["sample"]
     if others is not None:
         line["other_workloads"] = others
     print(json.dumps(line), flush=True)
