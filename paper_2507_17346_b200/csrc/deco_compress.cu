@@ -369,7 +369,7 @@ __device__ __forceinline__ void pick_body(SelectState &s, const uint32_t *h, uin
     __syncthreads();
 }
 
-// true for exactly one CTA per counter: the last of gridDim.x to get here (nothing waits)
+// true for exactly one CTA per counter: the last of `ctas` to get here (nothing waits)
 __device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *s_flag, uint32_t ctas)
 {
     __threadfence();
@@ -379,11 +379,6 @@ __device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *
     const bool last = *s_flag != 0;
     if (last) __threadfence();
     return last;
-}
-
-__device__ __forceinline__ bool last_cta_to_arrive(uint32_t *counter, uint32_t *s_flag)
-{
-    return last_cta_to_arrive(counter, s_flag, gridDim.x);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1020,16 +1015,15 @@ __device__ __forceinline__ uint32_t emit_items_of(uint32_t cnt, bool whole_tiles
 }
 
 // Work list of a worker: one (tile, slice) entry per slice; every thread looks at one tile, a
-// warp reserves its entries with one atomic.  Called by all threads of the CTAs of a kernel
-// that runs between the streaming pass and emit.
-__device__ __forceinline__ void build_emit_work(const Sel &p, uint32_t i)
+// warp reserves its entries with one atomic.  Called by all threads of the `nctas` CTAs that a
+// kernel between the streaming pass and emit has for the worker.
+__device__ __forceinline__ void build_emit_work(const Sel &p, uint32_t i, const uint32_t cta, const uint32_t nctas)
 {
     const int lane = threadIdx.x & 31;
     uint32_t *count = &p.done[i * DONE_SLOTS + 5];
     uint2 *work = p.work + static_cast<size_t>(i) * p.work_cap;
     const uint32_t tiles_up = (p.ntiles + 31u) & ~31u;       // whole warps stay together
-    for (uint32_t tile = blockIdx.x * BLOCK + threadIdx.x; tile < tiles_up;
-         tile += gridDim.x * BLOCK) {
+    for (uint32_t tile = cta * BLOCK + threadIdx.x; tile < tiles_up; tile += nctas * BLOCK) {
         const uint32_t items =
             tile < p.ntiles ? emit_items_of(p.tile_cnt[static_cast<size_t>(i) * p.ntiles + tile], p.use_band != 0) : 0u;
         const uint32_t incl = warp_incl_scan(items);
@@ -1066,7 +1060,8 @@ __shared__ SelectShared sm;
 // rank k - (candidates above the band).  If the set is not usable, or the threshold falls into
 // the shared top bin, the worker is handed to the multi-pass route.
 template <bool COH>
-__device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i)
+__device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i, const uint32_t cta,
+                                                  const uint32_t nctas)
 {
     SelectState &s = p.sel[i];
     if (ldq<COH>(&s.exact)) return;
@@ -1080,8 +1075,8 @@ __device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i
     if (valid) {
         for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
         __syncthreads();
-        for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
-             base += gridDim.x * (4 * BLOCK)) {
+        for (uint32_t base = cta * (4 * BLOCK); base < n_band;
+             base += nctas * (4 * BLOCK)) {
             deco_pair v[4];
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
@@ -1100,7 +1095,7 @@ __device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i
         for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
             if (h[b]) atomicAdd(&out[b], h[b]);
     }
-    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 0], &sm.misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 0], &sm.misc[2], nctas)) return;
     uint32_t a_sel = REL_TOP, above_a = 0;
     if (valid) pick_bin(hist_of(p, i, 0, 0), p.k - n_cert, sm.scan, sm.misc, a_sel, above_a);
     if (threadIdx.x == 0) {
@@ -1118,13 +1113,14 @@ __device__ __forceinline__ void stage_hist_a_body(const Sel &p, const uint32_t i
 
 __global__ void __launch_bounds__(BLOCK) stage_hist_a_kernel(Sel p)
 {
-    stage_hist_a_body<false>(p, blockIdx.y);
+    stage_hist_a_body<false>(p, blockIdx.y, blockIdx.x, gridDim.x);
 }
 
 // Level B: histogram of the low bits of the band keys that fell into the chosen A bin; the
 // last CTA of a worker to arrive fixes the threshold key and the number of ties to take.
 template <bool COH>
-__device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i)
+__device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i, const uint32_t cta,
+                                                  const uint32_t nctas)
 {
     SelectState &s = p.sel[i];
     if (ldq<COH>(&s.exact)) return;
@@ -1137,10 +1133,10 @@ __device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i
     const uint32_t low_mask = (1u << shift) - 1u;
     const deco_pair *src = select_list(p, i, n_staged, n_band);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK) h[b] = 0;
-    build_emit_work(p, i);                              // independent of the histogram
+    build_emit_work(p, i, cta, nctas);                  // independent of the histogram
     __syncthreads();
-    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
-         base += gridDim.x * (4 * BLOCK)) {
+    for (uint32_t base = cta * (4 * BLOCK); base < n_band;
+         base += nctas * (4 * BLOCK)) {
         deco_pair v[4];
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
@@ -1160,7 +1156,7 @@ __device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i
     uint32_t *out = hist_of(p, i, 0, 1);
     for (int b = threadIdx.x; b < RADIX_BINS; b += BLOCK)
         if (h[b]) atomicAdd(&out[b], h[b]);
-    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 1], &sm.misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 1], &sm.misc[2], nctas)) return;
     uint32_t bin, above;
     pick_bin(hist_of(p, i, 0, 1), k_rem, sm.scan, sm.misc, bin, above);
     if (threadIdx.x == 0) {
@@ -1180,7 +1176,7 @@ __device__ __forceinline__ void stage_hist_b_body(const Sel &p, const uint32_t i
 
 __global__ void __launch_bounds__(BLOCK) stage_hist_b_kernel(Sel p)
 {
-    stage_hist_b_body<false>(p, blockIdx.y);
+    stage_hist_b_body<false>(p, blockIdx.y, blockIdx.x, gridDim.x);
 }
 
 // One CTA: ties are granted to chunks in index order until ties_take are used up, then every
@@ -1307,11 +1303,12 @@ __device__ void chunk_walk_sums(const Sel &p, uint32_t i, uint32_t *s_scan /*[33
 // Many chunks: their sums are taken in parallel, one warp per chunk (three coalesced loads
 // and a warp reduction; the CTAs stride over the chunks), and the last CTA of a worker to
 // arrive walks the chunks.
-__device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i)
+__device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i, const uint32_t cta,
+                                                const uint32_t nctas)
 {
     if (p.sel[i].exact) return;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    for (uint32_t chunk = blockIdx.x * WARPS + w; chunk < p.nchunks; chunk += gridDim.x * WARPS) {
+    for (uint32_t chunk = cta * WARPS + w; chunk < p.nchunks; chunk += nctas * WARPS) {
         const uint32_t tile = chunk * CHUNK_TILES + lane;
         const size_t ti = static_cast<size_t>(i) * p.ntiles + tile;
         uint32_t a = 0, b = 0, q = 0;
@@ -1331,13 +1328,13 @@ __device__ __forceinline__ void chunk_sums_body(const Sel &p, const uint32_t i)
             p.chunk_eq[static_cast<size_t>(i) * p.nchunks + chunk] = q;
         }
     }
-    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 4], &sm.misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 4], &sm.misc[2], nctas)) return;
     chunk_walk_sums(p, i, sm.scan);
 }
 
 __global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p)
 {
-    chunk_sums_body(p, blockIdx.y);
+    chunk_sums_body(p, blockIdx.y, blockIdx.x, gridDim.x);
 }
 
 // Classification.  With the threshold known every band entry below it is rejected: counted
@@ -1347,7 +1344,8 @@ __global__ void __launch_bounds__(BLOCK) chunk_sums_kernel(Sel p)
 // (The per-tile positions follow from these inside the emit step, so nothing here is serial
 // in the number of tiles.)
 template <bool COH>
-__device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t i, uint32_t walk_here)
+__device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t i, uint32_t walk_here,
+                                                    const uint32_t cta, const uint32_t nctas)
 {
     const SelectState &s = p.sel[i];
     if (ldq<COH>(&s.exact)) return;
@@ -1358,8 +1356,8 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
     uint32_t *rej = p.tile_rej + static_cast<size_t>(i) * p.ntiles;
     uint32_t *eqc = p.tile_eq + static_cast<size_t>(i) * p.ntiles;
     const int lane = threadIdx.x & 31;
-    for (uint32_t base = blockIdx.x * (4 * BLOCK); base < n_band;
-         base += gridDim.x * (4 * BLOCK)) {
+    for (uint32_t base = cta * (4 * BLOCK); base < n_band;
+         base += nctas * (4 * BLOCK)) {
         deco_pair prs[4];
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
@@ -1382,13 +1380,13 @@ __device__ __forceinline__ void stage_classify_body(const Sel &p, const uint32_t
         }
     }
     // (the rejected entries get their value back in e from emit, which reads every staged pair anyway)
-    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &sm.misc[2])) return;
+    if (!last_cta_to_arrive(&p.done[i * DONE_SLOTS + 2], &sm.misc[2], nctas)) return;
     if (walk_here) chunk_walk(p, i, sm.scan);
 }
 
 __global__ void __launch_bounds__(BLOCK) stage_classify_kernel(Sel p, uint32_t walk_here)
 {
-    stage_classify_body<false>(p, blockIdx.y, walk_here);
+    stage_classify_body<false>(p, blockIdx.y, walk_here, blockIdx.x, gridDim.x);
 }
 
 // What a warp learns about the CHUNK_TILES tiles of one chunk from three coalesced loads and
@@ -1582,16 +1580,17 @@ __device__ __forceinline__ void emit_items_part(const Sel &p, const uint32_t i, 
 
 // Emit as a launch of its own: CTAs [0, dir_ctas) of a worker do the directory part, the
 // remaining CTAs the work list.
-__device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, uint32_t dir_ctas)
+__device__ __forceinline__ void emit_stage_body(const Sel &p, const uint32_t i, const uint32_t cta,
+                                                const uint32_t nctas, uint32_t dir_ctas)
 {
     if (p.sel[i].exact) return;
-    if (blockIdx.x < dir_ctas) emit_directory_part<false>(p, i, blockIdx.x, dir_ctas);
-    else emit_items_part<false>(p, i, blockIdx.x - dir_ctas, gridDim.x - dir_ctas);
+    if (cta < dir_ctas) emit_directory_part<false>(p, i, cta, dir_ctas);
+    else emit_items_part<false>(p, i, cta - dir_ctas, nctas - dir_ctas);
 }
 
 __global__ void __launch_bounds__(BLOCK) emit_stage_kernel(Sel p, uint32_t dir_ctas)
 {
-    emit_stage_body(p, blockIdx.y, dir_ctas);
+    emit_stage_body(p, blockIdx.y, blockIdx.x, gridDim.x, dir_ctas);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1973,11 +1972,11 @@ __global__ void __launch_bounds__(BLOCK, 3) select_chain_kernel(Sel p)
 {
     cg::grid_group grid = cg::this_grid();
     const uint32_t i = blockIdx.y;
-    stage_hist_a_body<true>(p, i);
+    stage_hist_a_body<true>(p, i, blockIdx.x, gridDim.x);
     grid.sync();
-    stage_hist_b_body<true>(p, i);
+    stage_hist_b_body<true>(p, i, blockIdx.x, gridDim.x);
     grid.sync();
-    stage_classify_body<true>(p, i, 1u);
+    stage_classify_body<true>(p, i, 1u, blockIdx.x, gridDim.x);
     grid.sync();
     if (!__ldcg(&p.sel[i].exact)) {
         emit_directory_part<true>(p, i, blockIdx.x, gridDim.x);
@@ -1990,11 +1989,13 @@ __global__ void __launch_bounds__(BLOCK, 3) select_chain_kernel(Sel p)
 
 // ------------------------------------------------------------------------------------------
 // Many contexts in one launch (per-layer Top-k: one context per layer, all with n workers).
-// Row y of the grid is worker y % n of layer y / n; the layer's parameters come from a table
-// in device memory.  Every selection kernel above strides over its work by gridDim.x and
-// counts gridDim.x arrivals per worker, so one grid width serves layers of any size; the
-// sampling kernel is told how many CTAs each layer uses, and the streaming pass, which has one
-// CTA per tile, finds its layer from the tile number.
+// The layer's parameters come from a table in device memory.  The sampling and carry kernels
+// have grid row y = worker y % n of layer y / n.  The kernels that work on the staged pairs give
+// every layer a number of CTAs in proportion to its work (a layer of half a million entries next
+// to one of sixty-five million): grid row y is the worker, and a map in device memory says which
+// layer CTA x belongs to; the layer's record says where its CTAs start and how many they are,
+// and the bodies stride over their work and count arrivals by that number.  The streaming pass,
+// which has one CTA per tile, finds its layer from the tile number.
 // ------------------------------------------------------------------------------------------
 struct MultiLayer {
     Sel p;
@@ -2003,7 +2004,12 @@ struct MultiLayer {
     uint32_t walk_here;      // classification walks the chunks itself (few chunks)
     uint32_t rows_aligned;   // the layer's gradient rows start on 16-byte boundaries
     uint32_t carry;          // the layer's bound is carried over between iterations (short layers)
+    // first CTA and number of CTAs per worker: levels A, B and classification / chunk sums
+    // (0 CTAs where the classification walks the chunks) / emit, of which emit_dir do the
+    // directory part
+    uint32_t sel_first, sel_ctas, cs_first, cs_ctas, emit_first, emit_ctas, emit_dir;
 };
+constexpr uint32_t MULTI_MAP_CAP = 8192;        // CTAs per worker and kernel that the maps hold at least
 
 // With hundreds of (layer, worker) rows the sampling kernel is bound by the number of CTAs it
 // has to get through, so each thread takes several sample groups.
@@ -2129,38 +2135,45 @@ ef_accumulate_multi_kernel(const __grid_constant__ AccTable tab, const void *__r
                                                  m.tile_off, m.tile_cnt, m.tile_rej, m.tile_eq, m.ntiles);
 }
 
-__global__ void __launch_bounds__(BLOCK) stage_hist_a_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
+__global__ void __launch_bounds__(BLOCK)
+stage_hist_a_multi_kernel(const MultiLayer *__restrict__ table, const uint32_t *__restrict__ map)
 {
-    const Sel p = table[blockIdx.y / n].p;
-    stage_hist_a_body<false>(p, blockIdx.y % n);
-}
-
-__global__ void __launch_bounds__(BLOCK) stage_hist_b_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
-{
-    const Sel p = table[blockIdx.y / n].p;
-    stage_hist_b_body<false>(p, blockIdx.y % n);
-}
-
-__global__ void __launch_bounds__(BLOCK) stage_classify_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
-{
-    const MultiLayer &m = table[blockIdx.y / n];
+    const MultiLayer &m = table[map[blockIdx.x]];
     const Sel p = m.p;
-    stage_classify_body<false>(p, blockIdx.y % n, m.walk_here);
-}
-
-__global__ void __launch_bounds__(BLOCK) chunk_sums_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n)
-{
-    const MultiLayer &m = table[blockIdx.y / n];
-    if (m.walk_here) return;                                 // the classification did the walk
-    const Sel p = m.p;
-    chunk_sums_body(p, blockIdx.y % n);
+    stage_hist_a_body<false>(p, blockIdx.y, blockIdx.x - m.sel_first, m.sel_ctas);
 }
 
 __global__ void __launch_bounds__(BLOCK)
-emit_stage_multi_kernel(const MultiLayer *__restrict__ table, uint32_t n, uint32_t dir_ctas)
+stage_hist_b_multi_kernel(const MultiLayer *__restrict__ table, const uint32_t *__restrict__ map)
 {
-    const Sel p = table[blockIdx.y / n].p;
-    emit_stage_body(p, blockIdx.y % n, dir_ctas);
+    const MultiLayer &m = table[map[blockIdx.x]];
+    const Sel p = m.p;
+    stage_hist_b_body<false>(p, blockIdx.y, blockIdx.x - m.sel_first, m.sel_ctas);
+}
+
+__global__ void __launch_bounds__(BLOCK)
+stage_classify_multi_kernel(const MultiLayer *__restrict__ table, const uint32_t *__restrict__ map)
+{
+    const MultiLayer &m = table[map[blockIdx.x]];
+    const Sel p = m.p;
+    stage_classify_body<false>(p, blockIdx.y, m.walk_here, blockIdx.x - m.sel_first, m.sel_ctas);
+}
+
+// (only the layers whose classification does not walk the chunks itself are on this map)
+__global__ void __launch_bounds__(BLOCK)
+chunk_sums_multi_kernel(const MultiLayer *__restrict__ table, const uint32_t *__restrict__ map)
+{
+    const MultiLayer &m = table[map[blockIdx.x]];
+    const Sel p = m.p;
+    chunk_sums_body(p, blockIdx.y, blockIdx.x - m.cs_first, m.cs_ctas);
+}
+
+__global__ void __launch_bounds__(BLOCK)
+emit_stage_multi_kernel(const MultiLayer *__restrict__ table, const uint32_t *__restrict__ map)
+{
+    const MultiLayer &m = table[map[blockIdx.x]];
+    const Sel p = m.p;
+    emit_stage_body(p, blockIdx.y, blockIdx.x - m.emit_first, m.emit_ctas, m.emit_dir);
 }
 
 // Cooperative: the layers with a rejected staged set, one after the other.  Which layers those
@@ -2459,8 +2472,12 @@ struct MultiPlan {
         bool any_aligned = false, any_unaligned = false;
     };
     std::vector<AccGroup> acc;
-    // grid widths shared by all layers
-    uint32_t begin_ctas = 1, stage_ctas = 1, chunk_ctas = 0, dir_ctas = 1, item_ctas = 1;
+    // grid width of the sampling kernel (shared by all layers); CTAs per worker of the kernels
+    // on the staged pairs, and their maps CTA -> layer in device memory (map_cap words each)
+    uint32_t begin_ctas = 1, sel_total = 1, cs_total = 0, emit_total = 1;
+    uint32_t *maps = nullptr;
+    uint32_t map_cap = 0;
+    std::vector<uint32_t> maps_host;
 };
 
 MultiPlan *multi_plan_create(const std::vector<deco_ctx *> &layers, const std::vector<uint64_t> &g_off,
@@ -2484,6 +2501,11 @@ MultiPlan *multi_plan_create(const std::vector<deco_ctx *> &layers, const std::v
         mp->fallback_grid = static_cast<uint32_t>((per_sm > 4 ? 4 : per_sm) * sms);
         if (cudaMalloc(reinterpret_cast<void **>(&mp->dev), sizeof(MultiLayer) * layers.size()) != cudaSuccess)
             throw 2;
+        // every layer has at least one CTA on a map and at most two by that rule alone
+        mp->map_cap = std::max<uint32_t>(MULTI_MAP_CAP, 2 * static_cast<uint32_t>(layers.size()));
+        if (cudaMalloc(reinterpret_cast<void **>(&mp->maps), sizeof(uint32_t) * 3 * mp->map_cap) != cudaSuccess)
+            throw 2;
+        mp->maps_host.resize(3 * static_cast<size_t>(mp->map_cap));
     } catch (...) {
         cudaGetLastError();
         multi_plan_destroy(mp);
@@ -2496,6 +2518,7 @@ void multi_plan_destroy(MultiPlan *mp)
 {
     if (!mp) return;
     cudaFree(mp->dev);
+    cudaFree(mp->maps);
     delete mp;
 }
 
@@ -2509,7 +2532,8 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
 {
     const uint32_t L = static_cast<uint32_t>(mp->layers.size());
     const uint64_t esz = mp->grad_dtype == DECO_BF16 ? 2 : 4;
-    uint64_t begin_max = 1, stage_max = 1, chunk_max = 0, dir_max = 1, item_max = 1, dir_sum = 0;
+    uint64_t begin_max = 1;
+    std::vector<uint64_t> want_sel(L), want_cs(L), want_dir(L), want_items(L);
     for (uint32_t l = 0; l < L; ++l) {
         const deco_ctx *c = mp->layers[l];
         MultiLayer &m = mp->host[l];
@@ -2522,13 +2546,51 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
         m.rows_aligned = ((mp->g_off[l] * esz) % 16 == 0 && (c->g_stride * esz) % 16 == 0) ? 1u : 0u;
         begin_max = std::max<uint64_t>(begin_max, (m.S + MULTI_BEGIN_GROUPS * BEGIN_BLOCK - 1) /
                                                       (MULTI_BEGIN_GROUPS * BEGIN_BLOCK));
-        stage_max = std::max<uint64_t>(stage_max, (2 * c->k + 65536 + BLOCK * 4 - 1) / (BLOCK * 4));
-        if (!m.walk_here) chunk_max = std::max<uint64_t>(chunk_max, (c->nchunks + WARPS - 1) / WARPS);
-        dir_max = std::max<uint64_t>(dir_max, (c->nchunks + WARPS - 1) / WARPS);
-        dir_sum += (c->nchunks + WARPS - 1) / WARPS;
+        // what the layer would use by itself: a CTA per trip over about 2 k staged pairs, a warp
+        // per chunk, a warp per expected emit work item
+        want_sel[l] = (2 * c->k + 1024 + BLOCK * 4 - 1) / (BLOCK * 4);
+        want_cs[l] = m.walk_here ? 0 : (c->nchunks + WARPS - 1) / WARPS;
+        want_dir[l] = (c->nchunks + WARPS - 1) / WARPS;
         const uint64_t staged = 13 * c->k / 10, many = staged / (EMIT_LANE_MAX + 1);
         const uint64_t est_items = staged / EMIT_SLICE + (many < c->ntiles ? many : c->ntiles);
-        item_max = std::max<uint64_t>(item_max, (est_items + WARPS - 1) / WARPS + 1);
+        want_items[l] = (est_items + WARPS - 1) / WARPS + 1;
+    }
+    // Shares of a budget of CTAs per worker (two waves of the device over all workers; the maps'
+    // capacity at most): in proportion to what the layers want, at least one each where they
+    // want any.  The bodies stride over their work, so fewer CTAs than wanted only means trips.
+    const uint64_t budget = std::min<uint64_t>(mp->map_cap / 2, std::max<uint64_t>(1, 148ull * 8 * 2 / mp->n));
+    auto share = [&](const std::vector<uint64_t> &want, std::vector<uint32_t> &got, uint64_t room) {
+        uint64_t sum = 0;
+        for (uint64_t w : want) sum += w;
+        got.assign(L, 0);
+        for (uint32_t l = 0; l < L; ++l) {
+            if (want[l] == 0) continue;
+            const uint64_t g = sum <= room ? want[l] : want[l] * room / sum;
+            got[l] = static_cast<uint32_t>(g < 1 ? 1 : g);
+        }
+    };
+    std::vector<uint32_t> got_sel, got_cs, got_dir, got_items;
+    share(want_sel, got_sel, budget);
+    share(want_cs, got_cs, budget);
+    share(want_dir, got_dir, budget / 2);
+    share(want_items, got_items, budget);
+    uint32_t *map_sel = mp->maps_host.data(), *map_cs = map_sel + mp->map_cap, *map_emit = map_cs + mp->map_cap;
+    mp->sel_total = mp->cs_total = mp->emit_total = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        MultiLayer &m = mp->host[l];
+        m.sel_first = mp->sel_total;
+        m.sel_ctas = got_sel[l];
+        m.cs_first = mp->cs_total;
+        m.cs_ctas = got_cs[l];
+        m.emit_first = mp->emit_total;
+        m.emit_dir = got_dir[l];
+        m.emit_ctas = got_dir[l] + got_items[l];
+        if (mp->sel_total + m.sel_ctas > mp->map_cap || mp->cs_total + m.cs_ctas > mp->map_cap ||
+            mp->emit_total + m.emit_ctas > mp->map_cap)
+            return cudaErrorInvalidValue;          // cannot happen: the shares fit the budget
+        for (uint32_t q = 0; q < m.sel_ctas; ++q) map_sel[mp->sel_total++] = l;
+        for (uint32_t q = 0; q < m.cs_ctas; ++q) map_cs[mp->cs_total++] = l;
+        for (uint32_t q = 0; q < m.emit_ctas; ++q) map_emit[mp->emit_total++] = l;
     }
     mp->acc.assign((L + ACC_LAYERS_MAX - 1) / ACC_LAYERS_MAX, MultiPlan::AccGroup());
     for (uint32_t l = 0; l < L; ++l) {
@@ -2555,20 +2617,14 @@ static cudaError_t multi_plan_refresh(MultiPlan *mp, const void *grads, cudaStre
         grp.tab.pad = 0;
         (m.rows_aligned ? grp.any_aligned : grp.any_unaligned) = true;
     }
-    // a few waves of the device in all: rows = layers * n
-    const uint64_t rows = static_cast<uint64_t>(L) * mp->n;
-    const uint64_t cap = std::max<uint64_t>(1, (148ull * 8 * 4 + rows - 1) / rows);
     mp->begin_ctas = static_cast<uint32_t>(begin_max);
-    mp->stage_ctas = static_cast<uint32_t>(std::min(stage_max, cap));
-    mp->chunk_ctas = static_cast<uint32_t>(chunk_max);
-    // directory CTAs stride over the chunks: the longest layer may take four trips, so that the
-    // many short layers do not each bring a grid row full of idle CTAs
-    mp->dir_ctas = static_cast<uint32_t>(std::max<uint64_t>({1, (dir_max + 3) / 4, (dir_sum + L - 1) / L}));
-    mp->item_ctas = static_cast<uint32_t>(std::min(item_max, std::max<uint64_t>(1, 2 * cap)));
     (void)grads;
-    // the host table is pageable: the copy has left it when the call returns
-    const cudaError_t err = cudaMemcpyAsync(mp->dev, mp->host.data(), sizeof(MultiLayer) * L,
-                                            cudaMemcpyHostToDevice, s);
+    // the host tables are pageable: the copies have left them when the calls return
+    cudaError_t err = cudaMemcpyAsync(mp->dev, mp->host.data(), sizeof(MultiLayer) * L,
+                                      cudaMemcpyHostToDevice, s);
+    if (err == cudaSuccess)
+        err = cudaMemcpyAsync(mp->maps, mp->maps_host.data(), sizeof(uint32_t) * 3 * mp->map_cap,
+                              cudaMemcpyHostToDevice, s);
     if (err == cudaSuccess) {
         mp->dirty = false;
         mp->age = 0;
@@ -2609,12 +2665,13 @@ cudaError_t multi_compress(MultiPlan *mp, const void *grads, float alpha, cudaSt
             else ef_accumulate_multi_kernel<0, false><<<agrid, BLOCK, 0, s>>>(grp.tab, grads, g_stride, alpha);
         }
     }
-    const dim3 sgrid(mp->stage_ctas, rows);
-    stage_hist_a_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, n);
-    stage_hist_b_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, n);
-    stage_classify_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, n);
-    if (mp->chunk_ctas) chunk_sums_multi_kernel<<<dim3(mp->chunk_ctas, rows), BLOCK, 0, s>>>(mp->dev, n);
-    emit_stage_multi_kernel<<<dim3(mp->dir_ctas + mp->item_ctas, rows), BLOCK, 0, s>>>(mp->dev, n, mp->dir_ctas);
+    const uint32_t *map_sel = mp->maps, *map_cs = map_sel + mp->map_cap, *map_emit = map_cs + mp->map_cap;
+    const dim3 sgrid(mp->sel_total, n);
+    stage_hist_a_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, map_sel);
+    stage_hist_b_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, map_sel);
+    stage_classify_multi_kernel<<<sgrid, BLOCK, 0, s>>>(mp->dev, map_sel);
+    if (mp->cs_total) chunk_sums_multi_kernel<<<dim3(mp->cs_total, n), BLOCK, 0, s>>>(mp->dev, map_cs);
+    emit_stage_multi_kernel<<<dim3(mp->emit_total, n), BLOCK, 0, s>>>(mp->dev, map_emit);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     const MultiLayer *tab = mp->dev;
@@ -2622,7 +2679,7 @@ cudaError_t multi_compress(MultiPlan *mp, const void *grads, float alpha, cudaSt
     void *args[] = {&tab, &layers};
     err = cudaLaunchCooperativeKernel(reinterpret_cast<void *>(exact_fallback_multi_kernel),
                                       dim3(mp->fallback_grid), dim3(BLOCK), args, 0, s);
-    mp->layers[0]->launches += mp->chunk_ctas ? 9 : 8;
+    mp->layers[0]->launches += mp->cs_total ? 9 : 8;
     return err;
 }
 
