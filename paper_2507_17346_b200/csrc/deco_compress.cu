@@ -2501,8 +2501,9 @@ MultiPlan *multi_plan_create(const std::vector<deco_ctx *> &layers, const std::v
         mp->fallback_grid = static_cast<uint32_t>((per_sm > 4 ? 4 : per_sm) * sms);
         if (cudaMalloc(reinterpret_cast<void **>(&mp->dev), sizeof(MultiLayer) * layers.size()) != cudaSuccess)
             throw 2;
-        // every layer has at least one CTA on a map and at most two by that rule alone
-        mp->map_cap = std::max<uint32_t>(MULTI_MAP_CAP, 2 * static_cast<uint32_t>(layers.size()));
+        // a map holds a share of the budget (at most 1.5 times 148 * 8 * 2 CTAs: emit's two parts)
+        // plus the one CTA that every layer gets in any case (two on emit's map)
+        mp->map_cap = std::max<uint32_t>(MULTI_MAP_CAP, 4096u + 4u * static_cast<uint32_t>(layers.size()));
         if (cudaMalloc(reinterpret_cast<void **>(&mp->maps), sizeof(uint32_t) * 3 * mp->map_cap) != cudaSuccess)
             throw 2;
         mp->maps_host.resize(3 * static_cast<size_t>(mp->map_cap));

@@ -263,6 +263,21 @@ def test_per_layer_topk_short_layers_batch(kind):
                            tau_max=3, delta_max=1.0)
 
 
+def test_per_layer_thousands_of_layers():
+    """4400 layers just above one tile (8200 entries each) with one worker: the kernels on the
+    staged pairs share a CTA budget out over the layers, and with more layers than the budget
+    every layer still gets its one CTA (two for emit) - the map from CTA to layer has to hold
+    them all.  Two layers of 300 K entries take the long end of the shares."""
+    lengths = [8200] * 2200 + [300_000] + [8200] * 2200 + [300_001]
+    offsets = [0]
+    for ln in lengths:
+        offsets.append(offsets[-1] + ln)
+    n = 1
+    run_layered_parity(offsets, n, 0.01, 1, 0.1,
+                       lambda t: _values("normal", n, offsets[-1], t, torch.float32), steps=3,
+                       grad_dtype="f32", tau_max=1, delta_max=0.01)
+
+
 def test_per_layer_bound_carried_over_between_iterations():
     """After a few iterations under one policy the per-layer path takes its speculative bound
     from the previous iterations' exact thresholds instead of a sample.  Stationary gradients:
